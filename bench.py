@@ -1,0 +1,353 @@
+#!/usr/bin/env python
+"""Benchmark of the quantized-linear + LoRA layer, forward + backward, at the LLaMA-7B q_proj shape.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" = qlora_fwd + qlora_bwd_input + qlora_bwd_lora on one projection (K = N = 4096, INT4, group 128,
+LoRA r = 8, alpha = 16, M = 2048 bf16 tokens; synthetic seeded inputs).  Consecutive steps rotate through several
+independent copies of the layer (own weights, activations and outputs) whose combined footprint exceeds the L2
+cache, so no step finds its operands cached by the previous one.  Prints ONE JSON line (rank 0).
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs an independent replica of the
+same work: the layer has no exchange step, so there is no data-path collective; the time is the max over ranks.
+
+--impl reference times the CPU oracle (oracle/qlora_oracle.py, as it stands) on the host cores on a bounded
+sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "fwd+bwd TFLOP/s & % roofline, INTn dequant-GEMM+LoRA at LLaMA-7B shapes"
+UNIT = "TFLOP/s"
+WORKLOAD = dict(K=4096, N=4096, bits=4, group_size=128, r=8, alpha=16.0, M=2048)
+WORKLOAD_NAME = "configs[1]: LLaMA-7B q_proj K=N=4096, INT4 group 128, LoRA r=8 alpha=16, M=2048 (4x512) bf16 tokens, fwd+bwd"
+ROTATION = 4                      # independent layer copies cycled through (4 x ~73 MiB > 126 MB of L2)
+KERNELS_PER_STEP = None           # filled from the library's dispatch (see launches_per_step)
+
+# DRAM traffic per launch of the dominant kernel, from an ncu capture (profiles/); None until one is recorded.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def layer_flops(M, K, N, r):
+    """Algorithmic flops of one step: fwd 2MNK + 2MKr + 2MNr, bwd 2MNK + 4MNr + 4MKr  ->  4MNK + 6Mr(K+N)."""
+    return 4.0 * M * N * K + 6.0 * M * r * (K + N)
+
+
+def fwd_flops(M, K, N, r):
+    return 2.0 * M * N * K + 2.0 * M * r * (K + N)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(bf16_burst=float(p["bf16_tflops"]), bf16_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    hbm=float(p["hbm_gbs"]), source="measured")
+    return dict(bf16_burst=1590.0, bf16_sustained=1400.0, hbm=6650.0, source="fallback")
+
+
+# --------------------------------------------------------------------------------------------------------------
+# clocks sampled while the timed region runs (read-only NVML queries)
+# --------------------------------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+               0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+
+    def __init__(self, index: int, period_s: float = 0.05):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+                for bit, name in self.REASONS.items():
+                    if mask & bit and name != "gpu_idle":
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------------------------------------------
+# CPU oracle timing (the cpu_baseline leg and --impl reference)
+# --------------------------------------------------------------------------------------------------------------
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [int(p.get("num_threads", 1)) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_sample_step(sample):
+    """One pass of the whole hot path in the oracle on `sample` (a layer dict): unpack + dequant + fwd + bwd."""
+    from oracle import qlora_oracle as orc
+    return orc.layer_reference(sample)
+
+
+def make_sample(M_s, N_s, seed=0):
+    """A bounded sample of the workload: the first N_s output features and M_s token rows, all K input features."""
+    import qlora_inputs as qi
+    w = WORKLOAD
+    return qi.make_layer(K=w["K"], N=N_s, bits=w["bits"], group_size=w["group_size"], r=w["r"], alpha=w["alpha"],
+                         M=M_s, seed=1000 + seed)
+
+
+def time_oracle(target_seconds: float, steps: int, warmup: int):
+    """Choose a sample size so that (steps + warmup) oracle passes take about target_seconds; time `steps` of them."""
+    w = WORKLOAD
+    # calibrate on a small sample
+    probe = make_sample(32, 128)
+    t0 = time.perf_counter()
+    oracle_sample_step(probe)
+    oracle_sample_step(probe)
+    t_probe = (time.perf_counter() - t0) / 2
+    f_probe = layer_flops(32, w["K"], 128, w["r"])
+    rate = f_probe / max(t_probe, 1e-6)                      # conservative: small problems run below peak
+    budget = target_seconds / max(steps + warmup, 1)
+    M_s, N_s = 32, 128
+    for cand in ((64, 256), (128, 512), (256, 1024), (512, 2048), (1024, 4096), (2048, 4096)):
+        if layer_flops(cand[0], w["K"], cand[1], w["r"]) / rate <= budget:
+            M_s, N_s = cand
+    sample = make_sample(M_s, N_s)
+    for _ in range(warmup):
+        oracle_sample_step(sample)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_sample_step(sample)
+    dt = time.perf_counter() - t0
+    flops = layer_flops(M_s, w["K"], N_s, w["r"]) * steps
+    return dict(value=flops / dt / 1e12, seconds=dt, ms_per_step=dt / steps * 1e3, M_s=M_s, N_s=N_s,
+                sample=f"{steps} oracle passes (unpack+dequant+fwd+bwd, float64 numpy) over a sub-layer of the workload: "
+                       f"first {N_s} of {w['N']} output features, {M_s} of {w['M']} token rows, all K={w['K']}")
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    res = time_oracle(target_seconds=120.0, steps=args.steps, warmup=args.warmup)
+    cores = oracle_threads()
+    line = {"impl": "reference", "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": res["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD_NAME, "sample": res["sample"]},
+            "cpu_baseline": {"value": res["value"], "unit": UNIT, "cores": cores, "kind": "oracle", "sample": res["sample"]},
+            "e2e": {"value": res["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+# --------------------------------------------------------------------------------------------------------------
+# the GPU arm
+# --------------------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2306_08162_b200 as ql
+    import qlora_inputs as qi
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    ql.library()  # fail loudly if the CUDA library is missing
+
+    w = WORKLOAD
+    M, K, N, r = w["M"], w["K"], w["N"], w["r"]
+    d = ql.desc(w["bits"], w["group_size"], K, N, r, w["alpha"])
+    ws = torch.empty(ql.qlora_workspace_bytes(d, M), dtype=torch.uint8, device=dev)
+
+    def bf16(bits16):
+        return torch.from_numpy(np.ascontiguousarray(bits16).view(np.int16)).to(dev).view(torch.bfloat16)
+
+    layers, host = [], []
+    for i in range(ROTATION):
+        L = qi.config2(seed=10 * rank + i)
+        codes = torch.from_numpy(L["codes"]).to(dev)
+        Q = torch.empty((K * w["bits"] // 32, N), dtype=torch.int32, device=dev)
+        ql.qlora_pack(w["bits"], K, N, codes, Q)
+        del codes
+        layers.append(dict(Q=Q, scales=torch.from_numpy(L["scales"]).to(dev), zeros=torch.from_numpy(L["zeros"]).to(dev),
+                           A=bf16(L["A"]), B=bf16(L["B"]), X=bf16(L["X"]), dY=bf16(L["dY"]),
+                           Y=torch.empty((M, N), dtype=torch.bfloat16, device=dev),
+                           dX=torch.empty((M, K), dtype=torch.bfloat16, device=dev),
+                           H=torch.empty((M, r), dtype=torch.float32, device=dev),
+                           G=torch.empty((M, r), dtype=torch.float32, device=dev),
+                           dA=torch.zeros((r, K), dtype=torch.float32, device=dev),
+                           dB=torch.zeros((N, r), dtype=torch.float32, device=dev)))
+        host.append(dict(X=torch.from_numpy(L["X"].view(np.int16)).pin_memory(),
+                         dY=torch.from_numpy(L["dY"].view(np.int16)).pin_memory()))
+    host_out = dict(Y=torch.empty((M, N), dtype=torch.int16).pin_memory(), dX=torch.empty((M, K), dtype=torch.int16).pin_memory(),
+                    dA=torch.empty((r, K), dtype=torch.float32).pin_memory(), dB=torch.empty((N, r), dtype=torch.float32).pin_memory())
+
+    def step(L, events=None):
+        if events is not None:
+            events[0].record()
+        ql.qlora_fwd(d, M, L["X"], L["Q"], L["scales"], L["zeros"], L["A"], L["B"], L["Y"], L["H"], ws)
+        if events is not None:
+            events[1].record()
+        ql.qlora_bwd_input(d, M, L["dY"], L["Q"], L["scales"], L["zeros"], L["A"], L["B"], L["dX"], L["G"], ws)
+        if events is not None:
+            events[2].record()
+        ql.qlora_bwd_lora(d, M, L["X"], L["dY"], L["A"], L["B"], L["H"], L["G"], L["dA"], L["dB"], 0, ws)
+        if events is not None:
+            events[3].record()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing -------------------------------------------------------------------------
+    for i in range(args.warmup):
+        step(layers[i % ROTATION])
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    for i in range(args.steps):
+        step(layers[i % ROTATION], ev[i])
+    barrier()
+    clocks = sampler.stop()
+    total_ms = ev[0][0].elapsed_time(ev[-1][3])
+    call_ms = [float(np.mean([ev[i][c].elapsed_time(ev[i][c + 1]) for i in range(args.steps)])) for c in range(3)]
+
+    # ---- end to end: pinned host inputs copied in, results copied out, every step --------------------------
+    e2e_steps = max(3, min(args.steps, 50))
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def e2e_step(i):
+        L, Hs = layers[i % ROTATION], host[i % ROTATION]
+        L["X"].view(torch.int16).copy_(Hs["X"], non_blocking=True)
+        L["dY"].view(torch.int16).copy_(Hs["dY"], non_blocking=True)
+        step(L)
+        host_out["Y"].copy_(L["Y"].view(torch.int16), non_blocking=True)
+        host_out["dX"].copy_(L["dX"].view(torch.int16), non_blocking=True)
+        host_out["dA"].copy_(L["dA"], non_blocking=True)
+        host_out["dB"].copy_(L["dB"], non_blocking=True)
+
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    s0.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    s1.record()
+    barrier()
+    e2e_ms = s0.elapsed_time(s1)
+    h2d = 2 * M * (K + N)
+    d2h = 2 * M * (K + N) + 4 * r * (K + N)
+
+    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = float(times[0]), float(times[1])
+
+    if rank == 0:
+        flops_step = layer_flops(M, K, N, r)
+        value = flops_step * args.steps * world / (total_ms * 1e-3) / 1e12
+        e2e_value = flops_step * e2e_steps * world / (e2e_ms * 1e-3) / 1e12
+        peaks = measured_peaks()
+        # dominant kernel: the dequant-GEMM of the forward or backward-input call, whichever takes longer
+        dom = 0 if call_ms[0] >= call_ms[1] else 1
+        dom_name = ("qlora_fwd", "qlora_bwd_input")[dom]
+        achieved = fwd_flops(M, K, N, r) / (call_ms[dom] * 1e-3) / 1e12
+        long_run = total_ms > 1000.0
+        peak = peaks["bf16_sustained"] if long_run else peaks["bf16_burst"]
+        cpu = time_oracle(target_seconds=20.0, steps=3, warmup=1)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD_NAME, "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "l2": f"inputs larger than L2: steps rotate through {ROTATION} independent layer copies (~{ROTATION * 73} MiB)",
+                       "calls_ms": {"qlora_fwd": call_ms[0], "qlora_bwd_input": call_ms[1], "qlora_bwd_lora": call_ms[2]}},
+            "roofline": {"bound": "tensor", "kernel": dom_name, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                         "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                         "peak_kind": f"{peaks['source']} cuBLAS bf16 {'sustained' if long_run else 'burst'}",
+                         "step_frac_of_peak": value / world / peak},
+            "cpu_baseline": {"value": cpu["value"], "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": cpu["sample"]},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
+            "gpu_launches": launches_per_step(r) * args.steps,
+            "clocks": clocks,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def launches_per_step(r: int) -> int:
+    """Kernels the library launches for one fwd + bwd_input + bwd_lora at the benchmark shape: the LoRA
+    down-projection and the dequant-GEMM for each of fwd and bwd_input, and two (partial, reduce) for each of dA, dB."""
+    return (2 + 2 + 4) if r > 0 else 2
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,111 @@
+/*
+ * qlora.h -- C ABI of the B200 (sm_100a) library for the frozen-quantized linear layer with a trainable
+ * LoRA branch, forward and backward: the per-projection hot path of EMEF / LREC fine-tuning
+ * (INT2.1 paper, Section 3.1 and Figure 1).
+ *
+ * Notation.  M tokens, K input features, N output features, LoRA rank r, s = alpha / r.
+ *   X  bf16 [M, K]      activations               dY bf16 [M, N]   upstream gradient
+ *   Q  int32 [K*bits/32, N]  packed codes (frozen) scales, zeros fp16 [K/g, N]  per-group parameters
+ *   W  = dequant(Q) [N, K],  W[n,k] = scales[k/g, n] * (q[k,n] - zeros[k/g, n])
+ *   A  bf16 [r, K]  LoRA down-projection           B  bf16 [N, r]   LoRA up-projection
+ *   H  = X A^T  fp32 [M, r]                        G  = dY B  fp32 [M, r]
+ * (Appendix B of the paper names the pair the other way round; this header follows
+ *  Y = X W^T + s (X A^T) B^T, i.e. A is the matrix applied to the input first.)
+ *
+ * Packed format (Section 3.1, "Implementation Details": the frozen weights are a bit-packed INT32 matrix;
+ * the bit layout is this library's definition).  For each output column n the K codes form a little-endian
+ * bit stream: code k occupies stream bits [k*bits, k*bits+bits), LSB first, and word i of the column
+ * (element Q[i*N + n]) holds stream bits [32i, 32i+32).  bits = 2, 4, 8: 16, 8, 4 codes per word.  bits = 3:
+ * every 32 codes fill three consecutive words of the column; codes 10 and 21 of each block straddle two words.
+ * Words are to be read as unsigned.  Zero-points are fp16 values holding integers in [0, 2^bits - 1].
+ * Groups are contiguous along K: group(k) = k / group_size.
+ *
+ * General rules for every entry point below.
+ *   - All tensor pointers are DEVICE pointers owned by the caller, dense row-major, 16-byte aligned.  The
+ *     descriptor is a HOST pointer.  The library allocates no device memory, keeps no per-call state and never
+ *     frees anything.  Q, scales, zeros, A, B are read-only (theta_q is frozen and there is no gradient for it;
+ *     Section 3.1).
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = the legacy default stream) of
+ *     the current device.  No call synchronises the device; outputs are valid in stream order.
+ *   - Return value: QLORA_OK or a negative QLORA_ERR_* code.  Arguments are validated before anything is
+ *     launched; on error nothing has been enqueued.  Nothing is printed, nothing throws.
+ *   - Same inputs give bitwise the same outputs on every run (fixed-order reductions, no floating-point atomics).
+ *   - Supported shapes: M >= 1 (M = 0 is accepted and does nothing); K % 32 == 0; group_size % 32 == 0 and
+ *     K % group_size == 0; N % 8 == 0; r in {0, 8, 16, 24, ..., 64}.  Anything else: QLORA_ERR_UNSUPPORTED.
+ *     r = 0 means "no LoRA branch" (A, B may be NULL).
+ */
+#ifndef QLORA_H_
+#define QLORA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    QLORA_OK = 0,
+    QLORA_ERR_INVALID_ARG = -1, /* NULL where a pointer is required, negative size, bad flag */
+    QLORA_ERR_UNSUPPORTED = -2, /* shape / bits / group size / rank outside the supported set */
+    QLORA_ERR_ALIGNMENT = -3,   /* a tensor pointer is not 16-byte aligned */
+    QLORA_ERR_WORKSPACE = -4,   /* workspace missing or smaller than qlora_workspace_bytes() */
+    QLORA_ERR_CUDA = -5,        /* a CUDA runtime / driver call failed (launch, tensor-map encoding, ...) */
+    QLORA_ERR_TIMEOUT = -6      /* reserved: a bounded device-side wait gave up (see qlora_last_device_status) */
+};
+
+/* Layer descriptor (host memory). */
+typedef struct {
+    int bits;       /* 2, 3, 4 or 8 */
+    int group_size; /* g: codes per (scale, zero) pair along K */
+    int K;          /* input features */
+    int N;          /* output features */
+    int r;          /* LoRA rank (0 = no branch) */
+    float alpha;    /* LoRA "linear stretch"; the branch is scaled by alpha / r (Appendix B: 16 with r = 8) */
+} qlora_desc;
+
+/* Bytes of scratch the three layer calls may need for M tokens (the maximum over the calls, so one buffer
+ * serves all).  `out` is a host pointer.  The scratch holds H / G when the caller does not keep them, the
+ * split partial sums of the LoRA gradients and of small-M products.  Contents are undefined between calls. */
+int qlora_workspace_bytes(const qlora_desc* desc, int M, size_t* out);
+
+/* Forward (Figure 1, forward path):  Y = X W^T + s (X A^T) B^T,  bf16 output, fp32 accumulation.
+ * H_out: optional fp32 [M, r]; when non-NULL receives H = X A^T for reuse by qlora_bwd_lora. */
+int qlora_fwd(const qlora_desc* desc, int M, const void* X, const int32_t* Q, const void* scales,
+              const void* zeros, const void* A, const void* B, void* Y, float* H_out, void* workspace,
+              size_t workspace_bytes, void* cuda_stream);
+
+/* Backward through the frozen weight (Section 3.1: transposition of the packed matrix, unpacking and the matrix
+ * product fused in one kernel; Figure 1, backward path):  dX = dY W + s (dY B) A,  bf16 output.
+ * G_out: optional fp32 [M, r]; when non-NULL receives G = dY B for reuse by qlora_bwd_lora. */
+int qlora_bwd_input(const qlora_desc* desc, int M, const void* dY, const int32_t* Q, const void* scales,
+                    const void* zeros, const void* A, const void* B, void* dX, float* G_out, void* workspace,
+                    size_t workspace_bytes, void* cuda_stream);
+
+/* Gradients of the trainable pair (Section 3.1: only theta_l is updated; Figure 1, arrows into the LoRA blocks):
+ *   dA = s (dY B)^T X  fp32 [r, K],     dB = s dY^T (X A^T)  fp32 [N, r].
+ * H, G: fp32 [M, r] saved by the calls above, or NULL to recompute them here (the case under gradient
+ * checkpointing, Section 4.1).  accumulate = 0 overwrites dA / dB, 1 adds to their current contents
+ * (micro-batch accumulation, Appendix B). */
+int qlora_bwd_lora(const qlora_desc* desc, int M, const void* X, const void* dY, const void* A, const void* B,
+                   const float* H, const float* G, float* dA, float* dB, int accumulate, void* workspace,
+                   size_t workspace_bytes, void* cuda_stream);
+
+/* Format utilities (Section 3.1: bit-packed INT32 storage).  codes: uint8 [K, N], one code per byte.
+ * qlora_pack rejects nothing about code values: only the low `bits` bits of each byte are used. */
+int qlora_pack(int bits, int K, int N, const uint8_t* codes, int32_t* Q, void* cuda_stream);
+int qlora_unpack(int bits, int K, int N, const int32_t* Q, uint8_t* codes, void* cuda_stream);
+
+/* Full dequantisation to the bf16 weight the tensor-core kernels stage:  W[n,k] = bf16_rne(fp32(scale) * (q - zero)),
+ * bf16 [N, K].  The fp32 product is exact (an 11-bit significand times an integer of at most 9 bits), so the result
+ * is a single rounding of the closed form.  desc->r and desc->alpha are ignored. */
+int qlora_dequant(const qlora_desc* desc, const int32_t* Q, const void* scales, const void* zeros, void* W,
+                  void* cuda_stream);
+
+/* Human-readable name of a status code (static storage; never NULL). */
+const char* qlora_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QLORA_H_ */

@@ -1,0 +1,190 @@
+// The C ABI declared in qlora.h: argument validation, workspace carving and kernel dispatch.  No kernel lives here.
+#include <cuda_runtime.h>
+
+#include "launch.h"
+#include "qlora.h"
+
+namespace {
+
+using namespace qlora;
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int check_bits(int bits) { return (bits == 2 || bits == 3 || bits == 4 || bits == 8) ? QLORA_OK : QLORA_ERR_UNSUPPORTED; }
+
+int check_format(int bits, int K, int N) {
+    if (K < 0 || N < 0) return QLORA_ERR_INVALID_ARG;
+    if (check_bits(bits) != QLORA_OK) return QLORA_ERR_UNSUPPORTED;
+    if (K % 32 != 0 || N % 8 != 0) return QLORA_ERR_UNSUPPORTED;
+    return QLORA_OK;
+}
+
+int check_desc(const qlora_desc* d, bool need_lora) {
+    if (d == nullptr) return QLORA_ERR_INVALID_ARG;
+    const int rc = check_format(d->bits, d->K, d->N);
+    if (rc != QLORA_OK) return rc;
+    if (d->group_size <= 0) return QLORA_ERR_INVALID_ARG;
+    if (d->group_size % 32 != 0 || d->K % d->group_size != 0) return QLORA_ERR_UNSUPPORTED;
+    if (need_lora) {
+        if (d->r < 0) return QLORA_ERR_INVALID_ARG;
+        if (d->r % 8 != 0 || d->r > 64) return QLORA_ERR_UNSUPPORTED;
+        if (!(d->alpha == d->alpha)) return QLORA_ERR_INVALID_ARG;   // NaN
+    }
+    return QLORA_OK;
+}
+
+struct Workspace {
+    size_t p0_off, p1_off, grad_off, total;
+};
+
+Workspace carve(const qlora_desc& d, int M) {
+    Workspace w{};
+    const size_t p = align_up((size_t)M * (size_t)d.r * sizeof(float), 256);
+    w.p0_off = 0;
+    w.p1_off = p;
+    w.grad_off = 2 * p;
+    const size_t ga = lora_grad_scratch_bytes(M, d.K, d.r), gb = lora_grad_scratch_bytes(M, d.N, d.r);
+    w.total = w.grad_off + align_up(ga > gb ? ga : gb, 256);
+    if (w.total == 0) w.total = 256;
+    return w;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* qlora_status_string(int status) {
+    switch (status) {
+        case QLORA_OK: return "ok";
+        case QLORA_ERR_INVALID_ARG: return "invalid argument";
+        case QLORA_ERR_UNSUPPORTED: return "unsupported shape, bit width, group size or rank";
+        case QLORA_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+        case QLORA_ERR_WORKSPACE: return "workspace missing or too small";
+        case QLORA_ERR_CUDA: return "CUDA call failed";
+        case QLORA_ERR_TIMEOUT: return "bounded device-side wait gave up";
+        default: return "unknown status";
+    }
+}
+
+int qlora_workspace_bytes(const qlora_desc* desc, int M, size_t* out) {
+    if (out == nullptr || M < 0) return QLORA_ERR_INVALID_ARG;
+    const int rc = check_desc(desc, true);
+    if (rc != QLORA_OK) return rc;
+    *out = carve(*desc, M).total;
+    return QLORA_OK;
+}
+
+int qlora_pack(int bits, int K, int N, const uint8_t* codes, int32_t* Q, void* cuda_stream) {
+    const int rc = check_format(bits, K, N);
+    if (rc != QLORA_OK) return rc;
+    if (K == 0 || N == 0) return QLORA_OK;
+    if (codes == nullptr || Q == nullptr) return QLORA_ERR_INVALID_ARG;
+    if (!aligned16(codes) || !aligned16(Q)) return QLORA_ERR_ALIGNMENT;
+    return launch_pack(bits, K, N, codes, Q, (cudaStream_t)cuda_stream);
+}
+
+int qlora_unpack(int bits, int K, int N, const int32_t* Q, uint8_t* codes, void* cuda_stream) {
+    const int rc = check_format(bits, K, N);
+    if (rc != QLORA_OK) return rc;
+    if (K == 0 || N == 0) return QLORA_OK;
+    if (codes == nullptr || Q == nullptr) return QLORA_ERR_INVALID_ARG;
+    if (!aligned16(codes) || !aligned16(Q)) return QLORA_ERR_ALIGNMENT;
+    return launch_unpack(bits, K, N, Q, codes, (cudaStream_t)cuda_stream);
+}
+
+int qlora_dequant(const qlora_desc* desc, const int32_t* Q, const void* scales, const void* zeros, void* W,
+                  void* cuda_stream) {
+    const int rc = check_desc(desc, false);
+    if (rc != QLORA_OK) return rc;
+    if (desc->K == 0 || desc->N == 0) return QLORA_OK;
+    if (!Q || !scales || !zeros || !W) return QLORA_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(scales) || !aligned16(zeros) || !aligned16(W)) return QLORA_ERR_ALIGNMENT;
+    return launch_dequant(*desc, Q, scales, zeros, W, (cudaStream_t)cuda_stream);
+}
+
+int qlora_fwd(const qlora_desc* desc, int M, const void* X, const int32_t* Q, const void* scales, const void* zeros,
+              const void* A, const void* B, void* Y, float* H_out, void* workspace, size_t workspace_bytes,
+              void* cuda_stream) {
+    int rc = check_desc(desc, true);
+    if (rc != QLORA_OK) return rc;
+    if (M < 0) return QLORA_ERR_INVALID_ARG;
+    const qlora_desc& d = *desc;
+    if (M == 0 || d.N == 0) return QLORA_OK;
+    if (!X || !Q || !scales || !zeros || !Y) return QLORA_ERR_INVALID_ARG;
+    if (d.r > 0 && (!A || !B)) return QLORA_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(Q) || !aligned16(scales) || !aligned16(zeros) || !aligned16(Y) ||
+        !aligned16(A) || !aligned16(B) || !aligned16(H_out) || !aligned16(workspace))
+        return QLORA_ERR_ALIGNMENT;
+    const Workspace w = carve(d, M);
+    if (workspace == nullptr || workspace_bytes < w.total) return QLORA_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    float* H = H_out ? H_out : reinterpret_cast<float*>(static_cast<char*>(workspace) + w.p0_off);
+    if (d.r > 0) {
+        rc = launch_lora_down(M, d.K, d.r, true, X, A, H, st);
+        if (rc != QLORA_OK) return rc;
+    }
+    return launch_simt_gemm(d, M, false, X, Q, scales, zeros, B, H, Y, st);
+}
+
+int qlora_bwd_input(const qlora_desc* desc, int M, const void* dY, const int32_t* Q, const void* scales,
+                    const void* zeros, const void* A, const void* B, void* dX, float* G_out, void* workspace,
+                    size_t workspace_bytes, void* cuda_stream) {
+    int rc = check_desc(desc, true);
+    if (rc != QLORA_OK) return rc;
+    if (M < 0) return QLORA_ERR_INVALID_ARG;
+    const qlora_desc& d = *desc;
+    if (M == 0 || d.K == 0) return QLORA_OK;
+    if (!dY || !Q || !scales || !zeros || !dX) return QLORA_ERR_INVALID_ARG;
+    if (d.r > 0 && (!A || !B)) return QLORA_ERR_INVALID_ARG;
+    if (!aligned16(dY) || !aligned16(Q) || !aligned16(scales) || !aligned16(zeros) || !aligned16(dX) ||
+        !aligned16(A) || !aligned16(B) || !aligned16(G_out) || !aligned16(workspace))
+        return QLORA_ERR_ALIGNMENT;
+    const Workspace w = carve(d, M);
+    if (workspace == nullptr || workspace_bytes < w.total) return QLORA_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    float* G = G_out ? G_out : reinterpret_cast<float*>(static_cast<char*>(workspace) + w.p0_off);
+    if (d.r > 0) {
+        rc = launch_lora_down(M, d.N, d.r, false, dY, B, G, st);
+        if (rc != QLORA_OK) return rc;
+    }
+    return launch_simt_gemm(d, M, true, dY, Q, scales, zeros, A, G, dX, st);
+}
+
+int qlora_bwd_lora(const qlora_desc* desc, int M, const void* X, const void* dY, const void* A, const void* B,
+                   const float* H, const float* G, float* dA, float* dB, int accumulate, void* workspace,
+                   size_t workspace_bytes, void* cuda_stream) {
+    int rc = check_desc(desc, true);
+    if (rc != QLORA_OK) return rc;
+    if (M < 0 || (accumulate != 0 && accumulate != 1)) return QLORA_ERR_INVALID_ARG;
+    const qlora_desc& d = *desc;
+    if (d.r == 0) return QLORA_OK;
+    if (!dA || !dB) return QLORA_ERR_INVALID_ARG;
+    if (M > 0 && (!X || !dY)) return QLORA_ERR_INVALID_ARG;
+    if (M > 0 && ((!H && !A) || (!G && !B))) return QLORA_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(dY) || !aligned16(A) || !aligned16(B) || !aligned16(H) || !aligned16(G) ||
+        !aligned16(dA) || !aligned16(dB) || !aligned16(workspace))
+        return QLORA_ERR_ALIGNMENT;
+    const Workspace w = carve(d, M);
+    if (workspace == nullptr || workspace_bytes < w.total) return QLORA_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    char* ws = static_cast<char*>(workspace);
+    const float s = d.alpha / (float)d.r;
+    if (M > 0 && !H) {
+        float* Hs = reinterpret_cast<float*>(ws + w.p0_off);
+        rc = launch_lora_down(M, d.K, d.r, true, X, A, Hs, st);
+        if (rc != QLORA_OK) return rc;
+        H = Hs;
+    }
+    if (M > 0 && !G) {
+        float* Gs = reinterpret_cast<float*>(ws + w.p1_off);
+        rc = launch_lora_down(M, d.N, d.r, false, dY, B, Gs, st);
+        if (rc != QLORA_OK) return rc;
+        G = Gs;
+    }
+    rc = launch_lora_grad(M, d.N, d.r, s, true, dY, H, dB, accumulate, ws + w.grad_off, st);
+    if (rc != QLORA_OK) return rc;
+    return launch_lora_grad(M, d.K, d.r, s, false, X, G, dA, accumulate, ws + w.grad_off, st);
+}
+
+}  // extern "C"

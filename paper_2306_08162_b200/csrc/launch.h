@@ -1,0 +1,30 @@
+// Host-side launch functions of the individual kernels (internal; the public boundary is include/qlora.h).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "qlora.h"
+
+namespace qlora {
+
+// format_kernels.cu
+int launch_pack(int bits, int K, int N, const uint8_t* codes, int32_t* Q, cudaStream_t st);
+int launch_unpack(int bits, int K, int N, const int32_t* Q, uint8_t* codes, cudaStream_t st);
+int launch_dequant(const qlora_desc& d, const int32_t* Q, const void* scales, const void* zeros, void* W,
+                   cudaStream_t st);
+
+// simt_kernels.cu -- CUDA-core kernels, correct for every supported shape
+// In [M, T] bf16 times the dequantised weight, plus s * P L.  transposed = false: forward (T = K, C = N);
+// true: backward-input (T = N, C = K).  P fp32 [M, r] (H or G) may be NULL when r == 0.
+int launch_simt_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q,
+                     const void* scales, const void* zeros, const void* L, const float* P, void* Out,
+                     cudaStream_t st);
+// P[m, j] = sum_t In[m, t] * L(j, t);  l_is_A: L = A [r, K] (t = k) else L = B [N, r] (t = n).
+int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const void* L, float* P, cudaStream_t st);
+// Out = s * sum_m In[m, c] * P[m, j]; out_is_dB: Out[c * r + j] (dB [N, r]) else Out[j * C + c] (dA [r, K]).
+size_t lora_grad_scratch_bytes(int M, int C, int r);
+int launch_lora_grad(int M, int C, int r, float s, bool out_is_dB, const void* In, const float* P, float* Out,
+                     int accumulate, void* scratch, cudaStream_t st);
+
+}  // namespace qlora

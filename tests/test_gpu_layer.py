@@ -1,0 +1,128 @@
+"""Parity of qlora_fwd / qlora_bwd_input / qlora_bwd_lora with the CPU oracle on seeded inputs (needs a B200).
+
+Gate: max relative error 2e-2 per output tensor (helpers.rel_err), bf16 inputs and fp32 accumulation on the GPU."""
+import numpy as np
+import pytest
+import torch
+
+import qlora_inputs as qi
+from oracle import qlora_oracle as orc
+from gpu_util import GpuLayer, to_f64
+from helpers import REL_TOL, rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+def check_layer(layer, rows=None, tol=REL_TOL, **run_kw):
+    gl = GpuLayer(layer)
+    out = gl.run(**run_kw)
+    ref = orc.layer_reference(layer, rows=rows)
+    sel = slice(None) if rows is None else np.asarray(rows)
+    errs = {"Y": rel_err(to_f64(out["Y"])[sel], ref["Y"]), "dX": rel_err(to_f64(out["dX"])[sel], ref["dX"])}
+    if layer["r"]:
+        errs["dA"] = rel_err(to_f64(out["dA"]), ref["dA"])
+        errs["dB"] = rel_err(to_f64(out["dB"]), ref["dB"])
+        if out["H"] is not None:
+            errs["H"] = rel_err(to_f64(out["H"])[sel], ref["H"])
+            errs["G"] = rel_err(to_f64(out["G"])[sel], ref["G"])
+    for name, e in errs.items():
+        assert e <= tol, (name, e, errs)
+    # the packed matrix produced by the library equals the oracle's
+    assert np.array_equal(gl.Q.cpu().numpy(), ref["Q"])
+    return errs, out, gl
+
+
+def sample_rows(M, n=48, seed=0):
+    if M <= n:
+        return None
+    rng = np.random.default_rng(seed)
+    rows = set(rng.choice(M, size=n - 4, replace=False).tolist()) | {0, 1, M - 2, M - 1}
+    return sorted(rows)
+
+
+def test_config1_full():
+    errs, _, _ = check_layer(qi.config1())
+    assert errs["Y"] < 1e-2 and errs["dX"] < 1e-2   # expected a few 2^-9; larger would point at a bug
+
+
+def test_config2_q_proj_int4():
+    check_layer(qi.config2())
+
+
+@pytest.mark.parametrize("which", ["gate", "up", "down"])
+def test_config3_mlp_int2_outliers(which):
+    layer = qi.config3(which)
+    check_layer(layer, rows=sample_rows(layer["M"], seed=1))
+
+
+@pytest.mark.parametrize("bits", [3, 8])
+@pytest.mark.parametrize("M", qi.CONFIG4_M)
+def test_config4_int3_int8_sweep(bits, M):
+    layer = qi.config4(bits, M)
+    check_layer(layer, rows=sample_rows(M, seed=M))
+
+
+@pytest.mark.parametrize("M", [1, 16, 17, 127, 129, 300])
+@pytest.mark.parametrize("bits,g", [(4, 128), (3, 32), (2, 64), (8, 64)])
+def test_edge_token_counts(M, bits, g):
+    check_layer(qi.random_codes_layer(K=256, N=264, bits=bits, group_size=g, r=8, alpha=16.0, M=M, seed=M + bits))
+
+
+@pytest.mark.parametrize("K,N", [(11008, 128), (128, 11008), (352, 8), (32, 4096)])
+def test_edge_feature_counts(K, N):
+    g = 32 if K % 64 else 64
+    check_layer(qi.random_codes_layer(K=K, N=N, bits=2, group_size=g, r=16, alpha=32.0, M=40, seed=K + N))
+
+
+@pytest.mark.parametrize("r", [0, 8, 16, 24, 32, 64])
+def test_ranks(r):
+    check_layer(qi.random_codes_layer(K=256, N=384, bits=4, group_size=128, r=r, alpha=2.0 * max(r, 1), M=70, seed=r))
+
+
+def test_group_equals_k_and_small_group():
+    check_layer(qi.random_codes_layer(K=512, N=128, bits=4, group_size=512, r=8, alpha=16.0, M=33, seed=1))
+    check_layer(qi.random_codes_layer(K=512, N=128, bits=8, group_size=32, r=8, alpha=16.0, M=33, seed=2))
+
+
+def test_recompute_h_g_matches_saved():
+    layer = qi.random_codes_layer(K=512, N=256, bits=4, group_size=128, r=8, alpha=16.0, M=200, seed=3)
+    _, saved, gl = check_layer(layer, save_hg=True)
+    recomputed = gl.run(save_hg=False)
+    assert torch.equal(saved["dA"], recomputed["dA"]) and torch.equal(saved["dB"], recomputed["dB"])
+
+
+def test_accumulate_adds_to_existing_gradients():
+    layer = qi.random_codes_layer(K=256, N=256, bits=4, group_size=128, r=8, alpha=16.0, M=96, seed=4)
+    gl = GpuLayer(layer)
+    first = gl.run()
+    dA0 = torch.full_like(first["dA"], 3.0)
+    dB0 = torch.full_like(first["dB"], -2.0)
+    second = gl.run(accumulate=1, dA=dA0.clone(), dB=dB0.clone())
+    assert torch.equal(second["dA"], dA0 + first["dA"]) and torch.equal(second["dB"], dB0 + first["dB"])
+
+
+def test_bitwise_deterministic():
+    layer = qi.config1(seed=2)
+    gl = GpuLayer(layer)
+    a = gl.run()
+    b = gl.run()
+    for k in ("Y", "dX", "dA", "dB"):
+        assert torch.equal(a[k].view(torch.int16) if a[k].dtype == torch.bfloat16 else a[k],
+                           b[k].view(torch.int16) if b[k].dtype == torch.bfloat16 else b[k]), k
+
+
+def test_b_zero_gives_pure_quantized_layer():
+    layer = qi.random_codes_layer(K=256, N=128, bits=4, group_size=128, r=8, alpha=16.0, M=64, seed=5)
+    layer["B"] = np.zeros_like(layer["B"])
+    errs, out, gl = check_layer(layer)
+    W = orc.dequant(orc.pack(layer["codes"], 4), layer["scales"], layer["zeros"], 4, 128)
+    X = orc.bf16_bits_to_f64(layer["X"])
+    assert rel_err(to_f64(out["Y"]), X @ W.T) <= REL_TOL
+    assert float(out["dA"].abs().max()) == 0.0
+
+
+def test_empty_batch_is_a_no_op():
+    layer = qi.random_codes_layer(K=64, N=64, bits=4, group_size=32, r=8, alpha=16.0, M=4, seed=6)
+    gl = GpuLayer(layer)
+    out = gl.run(X=gl.X[:0], dY=gl.dY[:0], check_canaries=True)
+    assert float(out["dA"].abs().max()) == 0.0 and float(out["dB"].abs().max()) == 0.0
