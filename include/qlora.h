@@ -51,7 +51,7 @@ enum {
     QLORA_ERR_ALIGNMENT = -3,   /* a tensor pointer is not 16-byte aligned */
     QLORA_ERR_WORKSPACE = -4,   /* workspace missing or smaller than qlora_workspace_bytes() */
     QLORA_ERR_CUDA = -5,        /* a CUDA runtime / driver call failed (launch, tensor-map encoding, ...) */
-    QLORA_ERR_TIMEOUT = -6      /* reserved: a bounded device-side wait gave up (see qlora_last_device_status) */
+    QLORA_ERR_TIMEOUT = -6      /* a bounded device-side wait gave up (reported by qlora_device_status) */
 };
 
 /* Layer descriptor (host memory). */
@@ -101,6 +101,13 @@ int qlora_unpack(int bits, int K, int N, const int32_t* Q, uint8_t* codes, void*
  * is a single rounding of the closed form.  desc->r and desc->alpha are ignored. */
 int qlora_dequant(const qlora_desc* desc, const int32_t* Q, const void* scales, const void* zeros, void* W,
                   void* cuda_stream);
+
+/* Health check of the kernels enqueued so far on the current device.  Every wait inside the tensor-core kernels (on a
+ * TMA transfer, on another warp, on the tensor cores) is bounded; if one ever runs out, the kernel stops early, leaves
+ * its outputs incomplete and sets a sticky per-device status word instead of hanging the GPU.  This call SYNCHRONISES
+ * the device, copies the word to *status_out (host pointer; 0 = healthy), clears it when `clear` is non-zero, and
+ * returns QLORA_OK or QLORA_ERR_TIMEOUT.  The paper has no counterpart; it exists so that a synchronisation fault cannot hang a device. */
+int qlora_device_status(unsigned int* status_out, int clear);
 
 /* Human-readable name of a status code (static storage; never NULL). */
 const char* qlora_status_string(int status);

@@ -50,8 +50,9 @@ def library() -> ctypes.CDLL:
     lib.qlora_pack.argtypes = [i32, i32, i32, vp, vp, vp]
     lib.qlora_unpack.argtypes = [i32, i32, i32, vp, vp, vp]
     lib.qlora_dequant.argtypes = [dp, vp, vp, vp, vp, vp]
+    lib.qlora_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint), i32]
     for name in ("qlora_workspace_bytes", "qlora_fwd", "qlora_bwd_input", "qlora_bwd_lora", "qlora_pack",
-                 "qlora_unpack", "qlora_dequant"):
+                 "qlora_unpack", "qlora_dequant", "qlora_device_status"):
         getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -127,3 +128,12 @@ def qlora_unpack(bits, K, N, Q, codes, stream=None):
 def qlora_dequant(d, Q, scales, zeros, W, stream=None):
     _check(library().qlora_dequant(ctypes.byref(d), _ptr(Q), _ptr(scales), _ptr(zeros), _ptr(W), _stream(stream)),
            "qlora_dequant")
+
+
+def qlora_device_status(clear: bool = True) -> int:
+    """Synchronise the device and return its sticky health word (0 = healthy).  Raises QloraError on a recorded timeout."""
+    out = ctypes.c_uint(0)
+    rc = library().qlora_device_status(ctypes.byref(out), 1 if clear else 0)
+    if rc != 0:
+        raise QloraError(rc, f"qlora_device_status (word {out.value:#x})")
+    return int(out.value)

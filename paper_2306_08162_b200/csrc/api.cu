@@ -67,6 +67,14 @@ const char* qlora_status_string(int status) {
     }
 }
 
+int qlora_device_status(unsigned int* status_out, int clear) {
+    if (status_out == nullptr) return QLORA_ERR_INVALID_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return QLORA_ERR_CUDA;
+    const int rc = read_device_status(status_out, clear);
+    if (rc != QLORA_OK) return rc;
+    return *status_out == 0 ? QLORA_OK : QLORA_ERR_TIMEOUT;
+}
+
 int qlora_workspace_bytes(const qlora_desc* desc, int M, size_t* out) {
     if (out == nullptr || M < 0) return QLORA_ERR_INVALID_ARG;
     const int rc = check_desc(desc, true);
@@ -124,6 +132,7 @@ int qlora_fwd(const qlora_desc* desc, int M, const void* X, const int32_t* Q, co
         rc = launch_lora_down(M, d.K, d.r, true, X, A, H, st);
         if (rc != QLORA_OK) return rc;
     }
+    if (umma_supported(d, M)) return launch_umma_gemm(d, M, false, X, Q, scales, zeros, B, H, Y, st);
     return launch_simt_gemm(d, M, false, X, Q, scales, zeros, B, H, Y, st);
 }
 
@@ -148,6 +157,7 @@ int qlora_bwd_input(const qlora_desc* desc, int M, const void* dY, const int32_t
         rc = launch_lora_down(M, d.N, d.r, false, dY, B, G, st);
         if (rc != QLORA_OK) return rc;
     }
+    if (umma_supported(d, M)) return launch_umma_gemm(d, M, true, dY, Q, scales, zeros, A, G, dX, st);
     return launch_simt_gemm(d, M, true, dY, Q, scales, zeros, A, G, dX, st);
 }
 

@@ -27,4 +27,11 @@ size_t lora_grad_scratch_bytes(int M, int C, int r);
 int launch_lora_grad(int M, int C, int r, float s, bool out_is_dB, const void* In, const float* P, float* Out,
                      int accumulate, void* scratch, cudaStream_t st);
 
+// umma_kernel.cu -- tcgen05 tensor-core kernel (both directions); same contract as launch_simt_gemm
+bool umma_supported(const qlora_desc& d, int M);
+int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q,
+                     const void* scales, const void* zeros, const void* L, const float* P, void* Out,
+                     cudaStream_t st);
+int read_device_status(unsigned int* out, int clear);
+
 }  // namespace qlora

@@ -1,0 +1,558 @@
+// Tensor-core kernel of the quantized-linear + LoRA layer for sm_100a: TMA-staged packed codes and group parameters,
+// register-level unpack + dequantisation to bf16 in shared memory, tcgen05 MMA with fp32 accumulators in tensor
+// memory, LoRA update fused as one extra MMA per tile, bf16 epilogue.
+//
+// One kernel template serves both directions (Figure 1 of the paper):
+//   forward        Out[m, n] = sum_k X[m, k]  W[n, k] + s sum_j H[m, j] B[n, j]      contraction over k
+//   backward-input Out[m, k] = sum_n dY[m, n] W[n, k] + s sum_j G[m, j] A[j, k]      contraction over n
+// The backward direction is the paper's fused "transpose + unpack + matmul" (Section 3.1): nothing is transposed in
+// memory.  The packed word still yields consecutive-k codes; they are written as one 16-byte chunk of a shared-memory
+// operand whose *non-contraction* dimension is contiguous, and the MMA descriptor's major-ness bit does the rest.
+//
+// Orientation: the dequantised weight tile is the MMA's A operand (128 rows), the activation tile is the B operand
+// (up to 256 token rows), so every dequantised weight is reused by up to 256 tokens inside one CTA.  The accumulator
+// D[weight row, token] lives in tensor memory (two buffers of 256 columns, so the epilogue of one tile overlaps the
+// main loop of the next).
+//
+// Warp roles (480 threads): warp 0 = TMA producer of activation tiles, warp 1 = MMA issuer (+ tensor-memory
+// allocation), warp 2 = TMA producer of packed codes + group parameters (its ring runs ahead of the activation ring),
+// warps 3-6 = epilogue (+ LoRA operand staging), warps 7-14 = unpack/dequant.
+// Every mbarrier wait is bounded; on a timeout the kernel records a status word, drains and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "launch.h"
+
+namespace qlora {
+
+__device__ unsigned int g_device_status = 0;   // sticky; bit 0: an mbarrier wait timed out
+
+namespace {
+
+constexpr int kThreads = 480;
+constexpr int kDequantWarp0 = 7, kDequantWarps = 8, kDequantThreads = kDequantWarps * 32;
+constexpr int kEpiWarp0 = 3, kEpiWarps = 4;
+constexpr int kWRows = 128;          // weight rows (MMA M) per tile: n in forward, k in backward
+constexpr int kStepC = 64;           // contraction elements per pipeline stage
+constexpr int kWStageBytes = kWRows * kStepC * 2;   // 16 KiB of bf16 per stage
+constexpr int kAccStride = 256;      // tensor-memory columns per accumulator buffer
+constexpr uint32_t kSpinLimit = 1u << 23;
+
+struct Params {
+    int M, N, K, bits, g, r, r_pad;
+    int C;               // output columns (N forward, K backward)
+    int BT;              // token rows per tile (MMA N): 32, 64, 128 or 256
+    int n_tok_tiles, n_tiles, steps;
+    int S, P;            // stages of the activation/weight ring and of the packed ring
+    int packed_cols;     // 128 forward, 64 backward
+    int packed_rows;     // int32 rows per stage
+    int scale_rows;      // group rows per stage
+    uint32_t words_bytes, scale_bytes, packed_slot_bytes, x_stage_bytes;
+    uint32_t off_x, off_w, off_p, off_lora_a, off_lora_p, off_bar;   // offsets from the 1024-aligned smem base
+    float s;
+    const float* Pmat;               // H (forward) or G (backward), fp32 [M, r]
+    const __nv_bfloat16* L;          // B [N, r] (forward) or A [r, K] (backward)
+    __nv_bfloat16* Out;
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+// Bounded wait.  Returns false when the kernel is aborting (this wait or another one ran out of polls).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 63u) == 63u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    atomicOr(&g_device_status, 1u);
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor (version 1).  Offsets in bytes; layout 0 = no swizzle, 2 = 128-byte swizzle.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo, uint32_t layout) {
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo >> 4) & 0x3FFFu) << 32) | (1ull << 46) | ((uint64_t)layout << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = n_mma; majors: 0 = contraction-contiguous, 1 = other.
+__device__ __forceinline__ uint32_t instr_desc(uint32_t n_mma, uint32_t a_mn_major, uint32_t b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn_major << 15) | (b_mn_major << 16) | ((n_mma >> 3) << 17) |
+           ((128u >> 4) << 24);
+}
+
+// 32 consecutive-k codes of one column (BITS words) -> 16 registers of packed bf16 pairs, canonical rounding:
+// bf16_rne(fp32(scale) * (q - zero)); the fp32 product is exact.  The integer -> float step ORs the code into the
+// mantissa of 2^23 and subtracts 2^23 + zero, which is exact.
+template <int BITS>
+__device__ __forceinline__ void dequant32(const uint32_t (&w)[BITS], float scale, float zero, uint32_t (&out)[16]) {
+    const float bias = 8388608.0f + zero;
+    constexpr uint32_t mask = (1u << BITS) - 1u;
+#pragma unroll
+    for (int j = 0; j < 32; j += 2) {
+        float f[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int bitpos = (j + h) * BITS, wi = bitpos >> 5, sh = bitpos & 31;
+            uint32_t q = w[wi] >> sh;
+            if (sh + BITS > 32) q |= w[(wi + 1) % BITS] << (32 - sh);   // only reached for BITS == 3
+            q = (q & mask) | 0x4B000000u;
+            f[h] = (__uint_as_float(q) - bias) * scale;
+        }
+        __nv_bfloat162 p = __floats2bfloat162_rn(f[0], f[1]);
+        out[j / 2] = *reinterpret_cast<uint32_t*>(&p);
+    }
+}
+
+template <int BITS, bool TRANSPOSED>
+__global__ void __launch_bounds__(kThreads, 1)
+umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_q,
+                 const __grid_constant__ CUtensorMap tm_scales, const __grid_constant__ CUtensorMap tm_zeros,
+                 const Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag_s;
+    volatile int* abort_flag = &abort_flag_s;
+
+    const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem0 - smem_u32(smem_raw));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // barrier addresses
+    const uint32_t bar0 = smem0 + p.off_bar;
+    const uint32_t bar_full_x = bar0;                       // [S]
+    const uint32_t bar_full_w = bar_full_x + 8 * p.S;       // [S]
+    const uint32_t bar_empty = bar_full_w + 8 * p.S;        // [S]
+    const uint32_t bar_full_p = bar_empty + 8 * p.S;        // [P]
+    const uint32_t bar_empty_p = bar_full_p + 8 * p.P;      // [P]
+    const uint32_t bar_acc_full = bar_empty_p + 8 * p.P;    // [2]
+    const uint32_t bar_acc_empty = bar_acc_full + 16;       // [2]
+    const uint32_t bar_lora_full = bar_acc_empty + 16;      // [1]
+
+    if (threadIdx.x == 0) {
+        abort_flag_s = 0;
+        for (int i = 0; i < p.S; ++i) {
+            mbar_init(bar_full_x + 8 * i, 1);
+            mbar_init(bar_full_w + 8 * i, kDequantWarps);
+            mbar_init(bar_empty + 8 * i, 1);
+        }
+        for (int i = 0; i < p.P; ++i) {
+            mbar_init(bar_full_p + 8 * i, 1);
+            mbar_init(bar_empty_p + 8 * i, kDequantWarps);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar_acc_full + 8 * i, 1);
+            mbar_init(bar_acc_empty + 8 * i, kEpiWarps);
+        }
+        mbar_init(bar_lora_full, kEpiWarps);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {   // whole warp: allocate all 512 tensor-memory columns (one CTA per SM owns them)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    const int first_tile = blockIdx.x, tile_stride = gridDim.x;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer: activation tiles
+        if (lane == 0) {
+            uint32_t it = 0;   // running stage counter (continues across tiles)
+            bool ok = true;
+            for (int tile = first_tile; tile < p.n_tiles && ok; tile += tile_stride) {
+                const int m0 = (tile % p.n_tok_tiles) * p.BT;
+                for (int step = 0; step < p.steps; ++step, ++it) {
+                    const uint32_t slot = it % p.S, par = ((it / p.S) & 1u) ^ 1u;
+                    if (!mbar_wait(bar_empty + 8 * slot, par, abort_flag)) { ok = false; break; }
+                    const uint32_t bar = bar_full_x + 8 * slot;
+                    mbar_expect_tx(bar, p.x_stage_bytes);
+                    tma_load_2d(smem0 + p.off_x + slot * p.x_stage_bytes, &tm_act, bar, step * kStepC, m0);
+                }
+            }
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ TMA producer: packed codes, scales, zeros
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = first_tile; tile < p.n_tiles && ok; tile += tile_stride) {
+                const int w0 = (tile / p.n_tok_tiles) * kWRows;
+                for (int step = 0; step < p.steps; ++step, ++it) {
+                    const uint32_t slot = it % p.P, par = ((it / p.P) & 1u) ^ 1u;
+                    if (!mbar_wait(bar_empty_p + 8 * slot, par, abort_flag)) { ok = false; break; }
+                    const uint32_t dst = smem0 + p.off_p + slot * p.packed_slot_bytes;
+                    const uint32_t bar = bar_full_p + 8 * slot;
+                    mbar_expect_tx(bar, p.words_bytes + 2 * p.scale_bytes);
+                    const int c0 = step * kStepC;
+                    if (!TRANSPOSED) {   // weight rows n = w0.., contraction k = c0..
+                        tma_load_2d(dst, &tm_q, bar, w0, c0 * BITS / 32);
+                        tma_load_2d(dst + p.words_bytes, &tm_scales, bar, w0, c0 / p.g);
+                        tma_load_2d(dst + p.words_bytes + p.scale_bytes, &tm_zeros, bar, w0, c0 / p.g);
+                    } else {             // weight rows k = w0.., contraction n = c0..
+                        tma_load_2d(dst, &tm_q, bar, c0, w0 * BITS / 32);
+                        tma_load_2d(dst + p.words_bytes, &tm_scales, bar, c0, w0 / p.g);
+                        tma_load_2d(dst + p.words_bytes + p.scale_bytes, &tm_zeros, bar, c0, w0 / p.g);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc((uint32_t)p.BT, TRANSPOSED ? 1u : 0u, 0u);
+            const uint32_t idesc_lora = instr_desc((uint32_t)p.BT, 0u, 0u);
+            uint32_t it = 0, tile_it = 0;
+            bool ok = true;
+            for (int tile = first_tile; tile < p.n_tiles && ok; tile += tile_stride, ++tile_it) {
+                const uint32_t buf = tile_it & 1u;
+                const uint32_t d_tmem = tmem_base + buf * kAccStride;
+                if (!mbar_wait(bar_acc_empty + 8 * buf, ((tile_it >> 1) & 1u) ^ 1u, abort_flag)) break;
+                tc_fence_after();
+                for (int step = 0; step < p.steps; ++step, ++it) {
+                    const uint32_t slot = it % p.S, par = (it / p.S) & 1u;
+                    if (!mbar_wait(bar_full_x + 8 * slot, par, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(bar_full_w + 8 * slot, par, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t xa = smem0 + p.off_x + slot * p.x_stage_bytes;
+                    const uint32_t wa = smem0 + p.off_w + slot * kWStageBytes;
+#pragma unroll
+                    for (int k16 = 0; k16 < kStepC / 16; ++k16) {
+                        // activation tile: contraction-contiguous rows of 128 B, 128-byte swizzle, 8-row groups 1024 B apart
+                        const uint64_t b_desc = smem_desc(xa + k16 * 32, 16, 1024, 2);
+                        // weight tile: forward = same layout (rows n); backward = rows are contraction (n), 64 k contiguous:
+                        // MN-major, 64-element atoms 8192 B apart (LBO), 8-row contraction groups 1024 B apart (SBO)
+                        const uint64_t a_desc = TRANSPOSED ? smem_desc(wa + k16 * 2048, 8192, 1024, 2)
+                                                           : smem_desc(wa + k16 * 32, 16, 1024, 2);
+                        tc_mma(d_tmem, a_desc, b_desc, idesc, (step | k16) != 0 ? 1u : 0u);
+                    }
+                    tc_commit(bar_empty + 8 * slot);
+                }
+                if (!ok) break;
+                if (p.r > 0) {
+                    if (!mbar_wait(bar_lora_full, tile_it & 1u, abort_flag)) break;
+                    tc_fence_after();
+                    for (int jb = 0; jb < p.r_pad / 16; ++jb) {
+                        // un-swizzled operands: 8-row x 16-byte core matrices 128 B apart (SBO), contraction halves LBO apart
+                        const uint64_t a_desc = smem_desc(smem0 + p.off_lora_a + jb * 2 * (kWRows * 16), kWRows * 16, 128, 0);
+                        const uint64_t b_desc = smem_desc(smem0 + p.off_lora_p + jb * 2 * (p.BT * 16), p.BT * 16, 128, 0);
+                        tc_mma(d_tmem, a_desc, b_desc, idesc_lora, 1u);
+                    }
+                }
+                tc_commit(bar_acc_full + 8 * buf);
+            }
+        }
+    } else if (warp >= kEpiWarp0 && warp < kDequantWarp0) {
+        // ------------------------------------------------------------------ epilogue (+ LoRA operand staging)
+        const int q = warp & 3;                      // tensor-memory lane quarter this warp may read
+        const int et = threadIdx.x - kEpiWarp0 * 32; // 0..127
+        uint32_t tile_it = 0;
+        for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride, ++tile_it) {
+            const int wt = tile / p.n_tok_tiles, tt = tile % p.n_tok_tiles;
+            const int w0 = wt * kWRows, m0 = tt * p.BT;
+            const uint32_t buf = tile_it & 1u;
+            if (p.r > 0) {
+                // (the previous tile's LoRA MMA has completed: its accumulator-full barrier was observed below)
+                uint8_t* la = smem_gen + p.off_lora_a;
+                uint8_t* lp = smem_gen + p.off_lora_p;
+                const int row = et, wrow = w0 + row;
+                for (int jc = 0; jc < p.r_pad / 8; ++jc) {
+                    uint4 v = make_uint4(0, 0, 0, 0);
+                    if (jc * 8 < p.r && wrow < p.C) {
+                        if (!TRANSPOSED) {
+                            v = __ldg(reinterpret_cast<const uint4*>(p.L + (size_t)wrow * p.r + jc * 8));      // B[n, j..j+7]
+                        } else {
+                            uint32_t e[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                e[j] = __bfloat16_as_ushort(__ldg(p.L + (size_t)(jc * 8 + j) * p.K + wrow));     // A[j, k]
+                            v = make_uint4(e[0] | (e[1] << 16), e[2] | (e[3] << 16), e[4] | (e[5] << 16), e[6] | (e[7] << 16));
+                        }
+                    }
+                    *reinterpret_cast<uint4*>(la + jc * (kWRows * 16) + (row >> 3) * 128 + (row & 7) * 16) = v;
+                }
+                for (int row_t = et; row_t < p.BT; row_t += 128) {
+                    const int m = m0 + row_t;
+                    for (int jc = 0; jc < p.r_pad / 8; ++jc) {
+                        uint4 v = make_uint4(0, 0, 0, 0);
+                        if (jc * 8 < p.r && m < p.M) {
+                            const float4 a = __ldg(reinterpret_cast<const float4*>(p.Pmat + (size_t)m * p.r + jc * 8));
+                            const float4 b = __ldg(reinterpret_cast<const float4*>(p.Pmat + (size_t)m * p.r + jc * 8 + 4));
+                            __nv_bfloat162 h0 = __floats2bfloat162_rn(p.s * a.x, p.s * a.y), h1 = __floats2bfloat162_rn(p.s * a.z, p.s * a.w);
+                            __nv_bfloat162 h2 = __floats2bfloat162_rn(p.s * b.x, p.s * b.y), h3 = __floats2bfloat162_rn(p.s * b.z, p.s * b.w);
+                            v = make_uint4(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1),
+                                           *reinterpret_cast<uint32_t*>(&h2), *reinterpret_cast<uint32_t*>(&h3));
+                        }
+                        *reinterpret_cast<uint4*>(lp + jc * (p.BT * 16) + (row_t >> 3) * 128 + (row_t & 7) * 16) = v;
+                    }
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_lora_full);
+            }
+            bool ok = mbar_wait(bar_acc_full + 8 * buf, (tile_it >> 1) & 1u, abort_flag);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const int c = w0 + q * 32 + lane;                 // output column owned by this thread
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccStride;
+            for (int cb = 0; cb < p.BT; cb += 32) {
+                uint32_t v[32];
+                tc_ld32(taddr + cb, v);
+                tc_wait_ld();
+                if (c < p.C) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int m = m0 + cb + j;
+                        if (m < p.M) p.Out[(size_t)m * p.C + c] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
+        }
+    } else {
+        // ------------------------------------------------------------------ unpack + dequant
+        const int dt = threadIdx.x - kDequantWarp0 * 32;          // 0..255
+        const int col = dt % p.packed_cols;                       // column of the packed tile (n in both directions)
+        const int kb = dt / p.packed_cols;                        // 32-code block along k: 0..1 forward, 0..3 backward
+        // destination of this thread's four 16-byte chunks inside a weight stage
+        const int row = col;                                      // forward: row n; backward: row n (contraction) of a 64-k half
+        const uint32_t row_off = (TRANSPOSED ? (uint32_t)(kb >> 1) * 8192u : 0u) + (uint32_t)(row >> 3) * 1024u + (uint32_t)(row & 7) * 128u;
+        const int chunk0 = (TRANSPOSED ? (kb & 1) : kb) * 4;
+        const int srow = TRANSPOSED ? ((kb * 32) / p.g) % p.scale_rows : 0;   // group row inside the stage's scale tile
+        uint32_t it = 0, it_p = 0;
+        bool ok = true;
+        for (int tile = first_tile; tile < p.n_tiles && ok; tile += tile_stride) {
+            for (int step = 0; step < p.steps; ++step, ++it, ++it_p) {
+                const uint32_t pslot = it_p % p.P, ppar = (it_p / p.P) & 1u;
+                ok = mbar_wait(bar_full_p + 8 * pslot, ppar, abort_flag);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                const uint8_t* pk = smem_gen + p.off_p + pslot * p.packed_slot_bytes;
+                uint32_t w[BITS];
+#pragma unroll
+                for (int i = 0; i < BITS; ++i)
+                    w[i] = reinterpret_cast<const uint32_t*>(pk)[(kb * BITS + i) * p.packed_cols + col];
+                const float scale = __half2float(reinterpret_cast<const __half*>(pk + p.words_bytes)[srow * p.packed_cols + col]);
+                const float zero = __half2float(reinterpret_cast<const __half*>(pk + p.words_bytes + p.scale_bytes)[srow * p.packed_cols + col]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_empty_p + 8 * pslot);
+
+                uint32_t out[16];
+                dequant32<BITS>(w, scale, zero, out);
+
+                const uint32_t slot = it % p.S, par = ((it / p.S) & 1u) ^ 1u;
+                ok = mbar_wait(bar_empty + 8 * slot, par, abort_flag);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                uint8_t* ws = smem_gen + p.off_w + slot * kWStageBytes + row_off;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int chunk = (chunk0 + c) ^ (row & 7);
+                    *reinterpret_cast<uint4*>(ws + chunk * 16) = make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_full_w + 8 * slot);
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {   // give copies that may still be in flight time to land before the CTA's memory is released
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            f = nullptr;
+        return (EncodeTiledFn)f;
+    }();
+    return fn;
+}
+
+bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const void* base, uint64_t inner, uint64_t outer,
+                 uint32_t box_inner, uint32_t box_outer, CUtensorMapSwizzle sw) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {inner * (uint64_t)elem_bytes};
+    cuuint32_t box[2] = {box_inner, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+    static int n = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
+        return v;
+    }();
+    return n;
+}
+
+template <int BITS, bool TRANSPOSED>
+int launch_impl(const CUtensorMap& ta, const CUtensorMap& tq, const CUtensorMap& ts, const CUtensorMap& tz, const Params& p,
+                size_t smem_bytes, int grid, cudaStream_t st) {
+    static bool configured = false;   // raising the dynamic shared-memory limit is a per-function, per-process setting
+    auto kern = umma_gemm_kernel<BITS, TRANSPOSED>;
+    if (!configured) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024) != cudaSuccess) return QLORA_ERR_CUDA;
+        configured = true;
+    }
+    kern<<<grid, kThreads, smem_bytes, st>>>(ta, tq, ts, tz, p);
+    return cudaGetLastError() == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
+}
+
+}  // namespace
+
+bool umma_supported(const qlora_desc& d, int M) {
+    if (M < 1) return false;
+    if (d.K % 64 != 0 || d.N % 64 != 0) return false;              // contraction steps of 64 in both directions
+    if (!(d.group_size == 64 || d.group_size % 128 == 0)) return false;
+    if (d.r > 64) return false;
+    return true;
+}
+
+int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
+                     const void* zeros, const void* L, const float* Pmat, void* Out, cudaStream_t st) {
+    Params p{};
+    p.M = M; p.N = d.N; p.K = d.K; p.bits = d.bits; p.g = d.group_size; p.r = d.r; p.r_pad = (d.r + 15) / 16 * 16;
+    p.C = transposed ? d.K : d.N;
+    const int T = transposed ? d.N : d.K;
+    p.BT = M > 128 ? 256 : (M > 64 ? 128 : (M > 32 ? 64 : 32));
+    p.n_tok_tiles = (M + p.BT - 1) / p.BT;
+    const int n_w_tiles = (p.C + kWRows - 1) / kWRows;
+    p.n_tiles = p.n_tok_tiles * n_w_tiles;
+    p.steps = T / kStepC;
+    p.packed_cols = transposed ? 64 : 128;
+    p.packed_rows = (transposed ? 128 : 64) * d.bits / 32;
+    p.scale_rows = transposed ? (d.group_size >= 128 ? 1 : 128 / d.group_size) : 1;
+    p.words_bytes = (uint32_t)(p.packed_rows * p.packed_cols * 4);
+    p.scale_bytes = (uint32_t)(p.scale_rows * p.packed_cols * 2);
+    p.packed_slot_bytes = (p.words_bytes + 2 * p.scale_bytes + 127u) / 128u * 128u;
+    p.x_stage_bytes = (uint32_t)(p.BT * 128);
+    p.s = d.r > 0 ? d.alpha / (float)d.r : 0.f;
+    p.Pmat = Pmat; p.L = (const __nv_bfloat16*)L; p.Out = (__nv_bfloat16*)Out;
+
+    // shared-memory plan (offsets from a 1024-byte aligned base)
+    const uint32_t lora_a = (uint32_t)(kWRows * p.r_pad * 2), lora_p = (uint32_t)(p.BT * p.r_pad * 2);
+    const uint32_t budget = 232448 - 1024 /*alignment slack*/ - 2048 /*static, barriers, padding*/;
+    p.P = 4;
+    const uint32_t fixed = lora_a + lora_p + p.P * p.packed_slot_bytes + 512;
+    const uint32_t per_stage = p.x_stage_bytes + kWStageBytes;
+    int S = (int)((budget - fixed) / per_stage);
+    if (S > 8) S = 8;
+    if (S < 2) return QLORA_ERR_UNSUPPORTED;
+    p.S = S;
+    p.off_x = 0;
+    p.off_w = p.off_x + S * p.x_stage_bytes;
+    p.off_p = p.off_w + S * kWStageBytes;
+    p.off_lora_a = p.off_p + p.P * p.packed_slot_bytes;
+    p.off_lora_p = p.off_lora_a + lora_a;
+    p.off_bar = (p.off_lora_p + lora_p + 127u) / 128u * 128u;
+    const size_t smem_bytes = (size_t)p.off_bar + 512 + 1024;
+
+    CUtensorMap ta, tq, ts, tz;
+    if (!make_map_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, In, (uint64_t)T, (uint64_t)M, 64, (uint32_t)p.BT, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_2d(&tq, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, Q, (uint64_t)d.N, (uint64_t)(d.K * d.bits / 32), (uint32_t)p.packed_cols, (uint32_t)p.packed_rows, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_map_2d(&ts, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, scales, (uint64_t)d.N, (uint64_t)(d.K / d.group_size), (uint32_t)p.packed_cols, (uint32_t)p.scale_rows, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_map_2d(&tz, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, zeros, (uint64_t)d.N, (uint64_t)(d.K / d.group_size), (uint32_t)p.packed_cols, (uint32_t)p.scale_rows, CU_TENSOR_MAP_SWIZZLE_NONE))
+        return QLORA_ERR_CUDA;
+
+    const int grid = p.n_tiles < sm_count() ? p.n_tiles : sm_count();
+#define QLORA_LAUNCH(B)                                                                              \
+    return transposed ? launch_impl<B, true>(ta, tq, ts, tz, p, smem_bytes, grid, st)                \
+                      : launch_impl<B, false>(ta, tq, ts, tz, p, smem_bytes, grid, st)
+    switch (d.bits) {
+        case 2: QLORA_LAUNCH(2);
+        case 3: QLORA_LAUNCH(3);
+        case 4: QLORA_LAUNCH(4);
+        case 8: QLORA_LAUNCH(8);
+    }
+#undef QLORA_LAUNCH
+    return QLORA_ERR_UNSUPPORTED;
+}
+
+int read_device_status(unsigned int* out, int clear) {
+    unsigned int v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_device_status, sizeof(v)) != cudaSuccess) return QLORA_ERR_CUDA;
+    if (clear && v != 0) {
+        const unsigned int zero = 0;
+        if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(zero)) != cudaSuccess) return QLORA_ERR_CUDA;
+    }
+    *out = v;
+    return QLORA_OK;
+}
+
+}  // namespace qlora

@@ -67,6 +67,7 @@ class GpuLayer:
         ql.qlora_bwd_input(self.desc, M, dY, self.Q, self.scales, self.zeros, self.A, self.B, dX, G, self.ws)
         ql.qlora_bwd_lora(self.desc, M, X, dY, self.A, self.B, H, G, dA, dB, accumulate, self.ws)
         torch.cuda.synchronize()
+        assert ql.qlora_device_status() == 0
         if check_canaries:
             assert canaries_intact(Yraw, (M, self.N), torch.bfloat16), "write outside Y"
             assert canaries_intact(dXraw, (M, self.K), torch.bfloat16), "write outside dX"
