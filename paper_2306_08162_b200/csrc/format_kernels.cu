@@ -32,26 +32,25 @@ __global__ void unpack_kernel(int bits, int K, int N, const uint32_t* __restrict
     codes[idx] = (uint8_t)load_code(Q, N, bits, k, n);
 }
 
-// W[n, k] for a 32(k) x 32(n) tile per block: reads are coalesced along n, the tile is transposed through shared
-// memory so that the bf16 writes are coalesced along k.
-__global__ void dequant_kernel(int bits, int g, int K, int N, const uint32_t* __restrict__ Q,
-                               const __half* __restrict__ scales, const __half* __restrict__ zeros,
-                               __nv_bfloat16* __restrict__ W) {
-    __shared__ __nv_bfloat16 tile[32][33];
-    const int n0 = blockIdx.x * 32, k0 = blockIdx.y * 32;
-    const int tx = threadIdx.x, ty = threadIdx.y;          // 32 x 8
-    for (int i = ty; i < 32; i += 8) {
-        const int k = k0 + i, n = n0 + tx;
-        if (n < N) {
-            const size_t gi = (size_t)(k / g) * N + n;
-            tile[i][tx] = dequant_one(load_code(Q, N, bits, k, n), scales[gi], zeros[gi]);
-        }
-    }
-    __syncthreads();
-    for (int i = ty; i < 32; i += 8) {
-        const int n = n0 + i, k = k0 + tx;
-        if (n < N) W[(size_t)n * K + k] = tile[tx][i];
-    }
+// Full dequantisation.  One thread turns the 32 consecutive-k codes of one column (BITS words) into 32 bf16 with the same
+// routine the tensor-core kernel uses, and writes them as 64 contiguous bytes of row n of W.
+template <int BITS>
+__global__ void dequant_kernel(int g, int K, int N, const uint32_t* __restrict__ Q, const __half* __restrict__ scales,
+                               const __half* __restrict__ zeros, __nv_bfloat16* __restrict__ W) {
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int blocks = K / 32;
+    if (idx >= (size_t)blocks * N) return;
+    const int kb = (int)(idx / N), n = (int)(idx % N);
+    uint32_t w[BITS];
+#pragma unroll
+    for (int i = 0; i < BITS; ++i) w[i] = __ldg(Q + (size_t)(kb * BITS + i) * N + n);
+    const size_t gi = (size_t)((kb * 32) / g) * N + n;
+    const GroupParams gp = group_params(scales[gi], zeros[gi]);
+    uint32_t out[16];
+    dequant32<BITS>(w, gp, out);
+    uint4* dst = reinterpret_cast<uint4*>(W + (size_t)n * K + (size_t)kb * 32);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) dst[c] = make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
 }
 
 int launch_pack(int bits, int K, int N, const uint8_t* codes, int32_t* Q, cudaStream_t st) {
@@ -72,9 +71,19 @@ int launch_unpack(int bits, int K, int N, const int32_t* Q, uint8_t* codes, cuda
 int launch_dequant(const qlora_desc& d, const int32_t* Q, const void* scales, const void* zeros, void* W,
                    cudaStream_t st) {
     if (d.K == 0 || d.N == 0) return QLORA_OK;
-    dim3 grid((d.N + 31) / 32, d.K / 32), block(32, 8);
-    dequant_kernel<<<grid, block, 0, st>>>(d.bits, d.group_size, d.K, d.N, (const uint32_t*)Q, (const __half*)scales,
-                                           (const __half*)zeros, (__nv_bfloat16*)W);
+    const size_t total = (size_t)(d.K / 32) * d.N;
+    const unsigned grid = (unsigned)((total + 255) / 256);
+    const uint32_t* q = (const uint32_t*)Q;
+    const __half* s = (const __half*)scales;
+    const __half* z = (const __half*)zeros;
+    __nv_bfloat16* w = (__nv_bfloat16*)W;
+    switch (d.bits) {
+        case 2: dequant_kernel<2><<<grid, 256, 0, st>>>(d.group_size, d.K, d.N, q, s, z, w); break;
+        case 3: dequant_kernel<3><<<grid, 256, 0, st>>>(d.group_size, d.K, d.N, q, s, z, w); break;
+        case 4: dequant_kernel<4><<<grid, 256, 0, st>>>(d.group_size, d.K, d.N, q, s, z, w); break;
+        case 8: dequant_kernel<8><<<grid, 256, 0, st>>>(d.group_size, d.K, d.N, q, s, z, w); break;
+        default: return QLORA_ERR_UNSUPPORTED;
+    }
     return cudaGetLastError() == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
 }
 

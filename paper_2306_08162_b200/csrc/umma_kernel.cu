@@ -16,7 +16,7 @@
 //
 // Warp roles (480 threads): warp 0 = TMA producer of activation tiles, warp 1 = MMA issuer (+ tensor-memory
 // allocation), warp 2 = TMA producer of packed codes + group parameters (its ring runs ahead of the activation ring),
-// warps 3-6 = epilogue (+ LoRA operand staging), warps 7-14 = unpack/dequant.
+// warps 3-6 = epilogue (+ LoRA operand staging), warps 7-14 = unpack/dequant (two groups taking alternate stages).
 // Every mbarrier wait is bounded; on a timeout the kernel records a status word, drains and returns.
 #include <cuda.h>
 
@@ -30,7 +30,7 @@ __device__ unsigned int g_device_status = 0;   // sticky; bit 0: an mbarrier wai
 namespace {
 
 constexpr int kThreads = 480;
-constexpr int kDequantWarp0 = 7, kDequantWarps = 8, kDequantThreads = kDequantWarps * 32;
+constexpr int kDequantWarp0 = 7, kGroupWarps = 4;   // two dequant groups of four warps
 constexpr int kEpiWarp0 = 3, kEpiWarps = 4;
 constexpr int kWRows = 128;          // weight rows (MMA M) per tile: n in forward, k in backward
 constexpr int kStepC = 64;           // contraction elements per pipeline stage
@@ -86,6 +86,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     atomicOr(&g_device_status, 1u);
     return false;
 }
+// Whole-warp wait: lane 0 polls (so a waiting warp costs one lane's issue slots), the outcome is broadcast, and every
+// lane then observes the completed phase itself before touching the data the barrier guards.
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int lane) {
+    uint32_t ok = 1;
+    if (lane == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1u : 0u;
+    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+    if (ok) (void)mbar_try_wait(bar, parity);
+    return ok != 0;
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
                  ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
@@ -103,15 +112,12 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
 }
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
         : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -127,28 +133,11 @@ __device__ __forceinline__ uint32_t instr_desc(uint32_t n_mma, uint32_t a_mn_maj
            ((128u >> 4) << 24);
 }
 
-// 32 consecutive-k codes of one column (BITS words) -> 16 registers of packed bf16 pairs, canonical rounding:
-// bf16_rne(fp32(scale) * (q - zero)); the fp32 product is exact.  The integer -> float step ORs the code into the
-// mantissa of 2^23 and subtracts 2^23 + zero, which is exact.
-template <int BITS>
-__device__ __forceinline__ void dequant32(const uint32_t (&w)[BITS], float scale, float zero, uint32_t (&out)[16]) {
-    const float bias = 8388608.0f + zero;
-    constexpr uint32_t mask = (1u << BITS) - 1u;
-#pragma unroll
-    for (int j = 0; j < 32; j += 2) {
-        float f[2];
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const int bitpos = (j + h) * BITS, wi = bitpos >> 5, sh = bitpos & 31;
-            uint32_t q = w[wi] >> sh;
-            if (sh + BITS > 32) q |= w[(wi + 1) % BITS] << (32 - sh);   // only reached for BITS == 3
-            q = (q & mask) | 0x4B000000u;
-            f[h] = (__uint_as_float(q) - bias) * scale;
-        }
-        __nv_bfloat162 p = __floats2bfloat162_rn(f[0], f[1]);
-        out[j / 2] = *reinterpret_cast<uint32_t*>(&p);
-    }
-}
+// Ring position: slot index plus the phase bit of the current lap (no division in the hot loops).
+struct Ring {
+    uint32_t slot = 0, phase = 0;
+    __device__ __forceinline__ void advance(uint32_t n) { if (++slot == n) { slot = 0; phase ^= 1u; } }
+};
 
 template <int BITS, bool TRANSPOSED>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -163,28 +152,28 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem0 - smem_u32(smem_raw));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t S = (uint32_t)p.S, P = (uint32_t)p.P;
 
     // barrier addresses
-    const uint32_t bar0 = smem0 + p.off_bar;
-    const uint32_t bar_full_x = bar0;                       // [S]
-    const uint32_t bar_full_w = bar_full_x + 8 * p.S;       // [S]
-    const uint32_t bar_empty = bar_full_w + 8 * p.S;        // [S]
-    const uint32_t bar_full_p = bar_empty + 8 * p.S;        // [P]
-    const uint32_t bar_empty_p = bar_full_p + 8 * p.P;      // [P]
-    const uint32_t bar_acc_full = bar_empty_p + 8 * p.P;    // [2]
-    const uint32_t bar_acc_empty = bar_acc_full + 16;       // [2]
-    const uint32_t bar_lora_full = bar_acc_empty + 16;      // [1]
+    const uint32_t bar_full_x = smem0 + p.off_bar;          // [S]  activation tile landed (TMA)
+    const uint32_t bar_full_w = bar_full_x + 8 * S;         // [S]  weight tile written by one dequant group
+    const uint32_t bar_empty = bar_full_w + 8 * S;          // [S]  MMAs reading the stage have completed
+    const uint32_t bar_full_p = bar_empty + 8 * S;          // [P]  packed words + group parameters landed (TMA)
+    const uint32_t bar_empty_p = bar_full_p + 8 * P;        // [P]  the dequant group has read them into registers
+    const uint32_t bar_acc_full = bar_empty_p + 8 * P;      // [2]  accumulator buffer complete
+    const uint32_t bar_acc_empty = bar_acc_full + 16;       // [2]  accumulator buffer drained by the epilogue
+    const uint32_t bar_lora_full = bar_acc_empty + 16;      // [1]  LoRA operand tiles staged
 
     if (threadIdx.x == 0) {
         abort_flag_s = 0;
-        for (int i = 0; i < p.S; ++i) {
+        for (uint32_t i = 0; i < S; ++i) {
             mbar_init(bar_full_x + 8 * i, 1);
-            mbar_init(bar_full_w + 8 * i, kDequantWarps);
+            mbar_init(bar_full_w + 8 * i, kGroupWarps);
             mbar_init(bar_empty + 8 * i, 1);
         }
-        for (int i = 0; i < p.P; ++i) {
+        for (uint32_t i = 0; i < P; ++i) {
             mbar_init(bar_full_p + 8 * i, 1);
-            mbar_init(bar_empty_p + 8 * i, kDequantWarps);
+            mbar_init(bar_empty_p + 8 * i, kGroupWarps);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar_acc_full + 8 * i, 1);
@@ -207,79 +196,84 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer: activation tiles
         if (lane == 0) {
-            uint32_t it = 0;   // running stage counter (continues across tiles)
-            bool ok = true;
-            for (int tile = first_tile; tile < p.n_tiles && ok; tile += tile_stride) {
+            Ring ring;
+            for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride) {
                 const int m0 = (tile % p.n_tok_tiles) * p.BT;
-                for (int step = 0; step < p.steps; ++step, ++it) {
-                    const uint32_t slot = it % p.S, par = ((it / p.S) & 1u) ^ 1u;
-                    if (!mbar_wait(bar_empty + 8 * slot, par, abort_flag)) { ok = false; break; }
-                    const uint32_t bar = bar_full_x + 8 * slot;
+                for (int step = 0; step < p.steps; ++step) {
+                    if (!mbar_wait(bar_empty + 8 * ring.slot, ring.phase ^ 1u, abort_flag)) goto done;
+                    const uint32_t bar = bar_full_x + 8 * ring.slot;
                     mbar_expect_tx(bar, p.x_stage_bytes);
-                    tma_load_2d(smem0 + p.off_x + slot * p.x_stage_bytes, &tm_act, bar, step * kStepC, m0);
+                    tma_load_2d(smem0 + p.off_x + ring.slot * p.x_stage_bytes, &tm_act, bar, step * kStepC, m0);
+                    ring.advance(S);
                 }
             }
         }
     } else if (warp == 2) {
         // ------------------------------------------------------------------ TMA producer: packed codes, scales, zeros
         if (lane == 0) {
-            uint32_t it = 0;
-            bool ok = true;
-            for (int tile = first_tile; tile < p.n_tiles && ok; tile += tile_stride) {
+            Ring ring;
+            const uint32_t tx_bytes = p.words_bytes + 2 * p.scale_bytes;
+            for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride) {
                 const int w0 = (tile / p.n_tok_tiles) * kWRows;
-                for (int step = 0; step < p.steps; ++step, ++it) {
-                    const uint32_t slot = it % p.P, par = ((it / p.P) & 1u) ^ 1u;
-                    if (!mbar_wait(bar_empty_p + 8 * slot, par, abort_flag)) { ok = false; break; }
-                    const uint32_t dst = smem0 + p.off_p + slot * p.packed_slot_bytes;
-                    const uint32_t bar = bar_full_p + 8 * slot;
-                    mbar_expect_tx(bar, p.words_bytes + 2 * p.scale_bytes);
+                // forward: weight rows n = w0.., contraction k = c0..;  backward: weight rows k = w0.., contraction n = c0..
+                const int g_row = TRANSPOSED ? w0 / p.g : 0;
+                for (int step = 0; step < p.steps; ++step) {
+                    if (!mbar_wait(bar_empty_p + 8 * ring.slot, ring.phase ^ 1u, abort_flag)) goto done;
+                    const uint32_t dst = smem0 + p.off_p + ring.slot * p.packed_slot_bytes;
+                    const uint32_t bar = bar_full_p + 8 * ring.slot;
+                    mbar_expect_tx(bar, tx_bytes);
                     const int c0 = step * kStepC;
-                    if (!TRANSPOSED) {   // weight rows n = w0.., contraction k = c0..
+                    if (!TRANSPOSED) {
+                        const int gr = c0 / p.g;
                         tma_load_2d(dst, &tm_q, bar, w0, c0 * BITS / 32);
-                        tma_load_2d(dst + p.words_bytes, &tm_scales, bar, w0, c0 / p.g);
-                        tma_load_2d(dst + p.words_bytes + p.scale_bytes, &tm_zeros, bar, w0, c0 / p.g);
-                    } else {             // weight rows k = w0.., contraction n = c0..
+                        tma_load_2d(dst + p.words_bytes, &tm_scales, bar, w0, gr);
+                        tma_load_2d(dst + p.words_bytes + p.scale_bytes, &tm_zeros, bar, w0, gr);
+                    } else {
                         tma_load_2d(dst, &tm_q, bar, c0, w0 * BITS / 32);
-                        tma_load_2d(dst + p.words_bytes, &tm_scales, bar, c0, w0 / p.g);
-                        tma_load_2d(dst + p.words_bytes + p.scale_bytes, &tm_zeros, bar, c0, w0 / p.g);
+                        tma_load_2d(dst + p.words_bytes, &tm_scales, bar, c0, g_row);
+                        tma_load_2d(dst + p.words_bytes + p.scale_bytes, &tm_zeros, bar, c0, g_row);
                     }
+                    ring.advance(P);
                 }
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------------ MMA issuer (one thread)
         if (lane == 0) {
             const uint32_t idesc = instr_desc((uint32_t)p.BT, TRANSPOSED ? 1u : 0u, 0u);
             const uint32_t idesc_lora = instr_desc((uint32_t)p.BT, 0u, 0u);
-            uint32_t it = 0, tile_it = 0;
-            bool ok = true;
-            for (int tile = first_tile; tile < p.n_tiles && ok; tile += tile_stride, ++tile_it) {
+            // Descriptors of slot 0; the start-address field (16-byte units) is advanced per slot and per 16-wide MMA step.
+            // activation tile: contraction-contiguous rows of 128 B, 128-byte swizzle, 8-row groups 1024 B apart.
+            // weight tile: forward = the same layout (rows n); backward = rows are the contraction (n) with 64 k contiguous:
+            //   MN-major, 64-element atoms 8192 B apart (LBO), 8-row contraction groups 1024 B apart (SBO).
+            const uint64_t b_desc0 = smem_desc(smem0 + p.off_x, 16, 1024, 2);
+            const uint64_t a_desc0 = TRANSPOSED ? smem_desc(smem0 + p.off_w, 8192, 1024, 2) : smem_desc(smem0 + p.off_w, 16, 1024, 2);
+            constexpr uint32_t a_k16 = TRANSPOSED ? (2048u >> 4) : (32u >> 4);
+            const uint32_t x_step = p.x_stage_bytes >> 4;
+            Ring ring;
+            uint32_t tile_it = 0;
+            for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride, ++tile_it) {
                 const uint32_t buf = tile_it & 1u;
                 const uint32_t d_tmem = tmem_base + buf * kAccStride;
-                if (!mbar_wait(bar_acc_empty + 8 * buf, ((tile_it >> 1) & 1u) ^ 1u, abort_flag)) break;
+                if (!mbar_wait(bar_acc_empty + 8 * buf, ((tile_it >> 1) & 1u) ^ 1u, abort_flag)) goto done;
                 tc_fence_after();
-                for (int step = 0; step < p.steps; ++step, ++it) {
-                    const uint32_t slot = it % p.S, par = (it / p.S) & 1u;
-                    if (!mbar_wait(bar_full_x + 8 * slot, par, abort_flag)) { ok = false; break; }
-                    if (!mbar_wait(bar_full_w + 8 * slot, par, abort_flag)) { ok = false; break; }
+                uint32_t acc = 0;
+                for (int step = 0; step < p.steps; ++step) {
+                    if (!mbar_wait(bar_full_x + 8 * ring.slot, ring.phase, abort_flag)) goto done;
+                    if (!mbar_wait(bar_full_w + 8 * ring.slot, ring.phase, abort_flag)) goto done;
                     tc_fence_after();
-                    const uint32_t xa = smem0 + p.off_x + slot * p.x_stage_bytes;
-                    const uint32_t wa = smem0 + p.off_w + slot * kWStageBytes;
+                    const uint64_t b_desc = b_desc0 + ring.slot * x_step;
+                    const uint64_t a_desc = a_desc0 + ring.slot * (uint32_t)(kWStageBytes >> 4);
 #pragma unroll
                     for (int k16 = 0; k16 < kStepC / 16; ++k16) {
-                        // activation tile: contraction-contiguous rows of 128 B, 128-byte swizzle, 8-row groups 1024 B apart
-                        const uint64_t b_desc = smem_desc(xa + k16 * 32, 16, 1024, 2);
-                        // weight tile: forward = same layout (rows n); backward = rows are contraction (n), 64 k contiguous:
-                        // MN-major, 64-element atoms 8192 B apart (LBO), 8-row contraction groups 1024 B apart (SBO)
-                        const uint64_t a_desc = TRANSPOSED ? smem_desc(wa + k16 * 2048, 8192, 1024, 2)
-                                                           : smem_desc(wa + k16 * 32, 16, 1024, 2);
-                        tc_mma(d_tmem, a_desc, b_desc, idesc, (step | k16) != 0 ? 1u : 0u);
+                        tc_mma(d_tmem, a_desc + k16 * a_k16, b_desc + k16 * 2, idesc, acc);
+                        acc = 1;
                     }
-                    tc_commit(bar_empty + 8 * slot);
+                    tc_commit(bar_empty + 8 * ring.slot);
+                    ring.advance(S);
                 }
-                if (!ok) break;
                 if (p.r > 0) {
-                    if (!mbar_wait(bar_lora_full, tile_it & 1u, abort_flag)) break;
+                    if (!mbar_wait(bar_lora_full, tile_it & 1u, abort_flag)) goto done;
                     tc_fence_after();
                     for (int jb = 0; jb < p.r_pad / 16; ++jb) {
                         // un-swizzled operands: 8-row x 16-byte core matrices 128 B apart (SBO), contraction halves LBO apart
@@ -339,21 +333,22 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_lora_full);
             }
-            bool ok = mbar_wait(bar_acc_full + 8 * buf, (tile_it >> 1) & 1u, abort_flag);
-            ok = __all_sync(0xFFFFFFFFu, ok);
-            if (!ok) break;
+            if (!warp_wait(bar_acc_full + 8 * buf, (tile_it >> 1) & 1u, abort_flag, lane)) break;
             tc_fence_after();
             const int c = w0 + q * 32 + lane;                 // output column owned by this thread
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccStride;
-            for (int cb = 0; cb < p.BT; cb += 32) {
-                uint32_t v[32];
-                tc_ld32(taddr + cb, v);
+#pragma unroll 1
+            for (int cb = 0; cb < p.BT; cb += 16) {
+                uint32_t v[16];
+                tc_ld16(taddr + cb, v);
                 tc_wait_ld();
                 if (c < p.C) {
+                    __nv_bfloat16* optr = p.Out + (size_t)(m0 + cb) * p.C + c;
+                    const int rows_left = p.M - (m0 + cb);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int m = m0 + cb + j;
-                        if (m < p.M) p.Out[(size_t)m * p.C + c] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                    for (int j = 0; j < 16; ++j) {
+                        if (j < rows_left) *optr = __float2bfloat16_rn(__uint_as_float(v[j]));
+                        optr += p.C;
                     }
                 }
             }
@@ -361,54 +356,71 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
         }
-    } else {
+    } else if (warp >= kDequantWarp0) {
         // ------------------------------------------------------------------ unpack + dequant
-        const int dt = threadIdx.x - kDequantWarp0 * 32;          // 0..255
-        const int col = dt % p.packed_cols;                       // column of the packed tile (n in both directions)
-        const int kb = dt / p.packed_cols;                        // 32-code block along k: 0..1 forward, 0..3 backward
-        // destination of this thread's four 16-byte chunks inside a weight stage
-        const int row = col;                                      // forward: row n; backward: row n (contraction) of a 64-k half
-        const uint32_t row_off = (TRANSPOSED ? (uint32_t)(kb >> 1) * 8192u : 0u) + (uint32_t)(row >> 3) * 1024u + (uint32_t)(row & 7) * 128u;
-        const int chunk0 = (TRANSPOSED ? (kb & 1) : kb) * 4;
-        const int srow = TRANSPOSED ? ((kb * 32) / p.g) % p.scale_rows : 0;   // group row inside the stage's scale tile
-        uint32_t it = 0, it_p = 0;
-        bool ok = true;
-        for (int tile = first_tile; tile < p.n_tiles && ok; tile += tile_stride) {
-            for (int step = 0; step < p.steps; ++step, ++it, ++it_p) {
-                const uint32_t pslot = it_p % p.P, ppar = (it_p / p.P) & 1u;
-                ok = mbar_wait(bar_full_p + 8 * pslot, ppar, abort_flag);
-                ok = __all_sync(0xFFFFFFFFu, ok);
-                if (!ok) break;
-                const uint8_t* pk = smem_gen + p.off_p + pslot * p.packed_slot_bytes;
-                uint32_t w[BITS];
+        // Two groups of four warps take alternate pipeline stages, so each group has two stage times for its serial chain
+        // (wait, shared-memory loads, arithmetic, wait, stores, fence, arrive).  Inside a group a thread owns one column of
+        // the packed tile and two blocks of 32 consecutive-k codes.
+        const int group = (warp - kDequantWarp0) / kGroupWarps;    // 0 or 1
+        const int gt = threadIdx.x - (kDequantWarp0 + group * kGroupWarps) * 32;   // 0..127 inside the group
+        const int col = gt % p.packed_cols;                       // column of the packed tile (n in both directions)
+        const int kb0 = gt / p.packed_cols;                       // forward: 0; backward: 0..1
+        const int kb_stride = TRANSPOSED ? 2 : 1;                 // the thread's two code blocks are kb0 and kb0 + kb_stride
+        const uint32_t row_base = (uint32_t)(col >> 3) * 1024u + (uint32_t)(col & 7) * 128u;   // row `col` of a swizzled tile
+        const uint32_t sw = (uint32_t)(col & 7);
+        uint32_t w_off[2], chunk0[2], srow[2];
 #pragma unroll
-                for (int i = 0; i < BITS; ++i)
-                    w[i] = reinterpret_cast<const uint32_t*>(pk)[(kb * BITS + i) * p.packed_cols + col];
-                const float scale = __half2float(reinterpret_cast<const __half*>(pk + p.words_bytes)[srow * p.packed_cols + col]);
-                const float zero = __half2float(reinterpret_cast<const __half*>(pk + p.words_bytes + p.scale_bytes)[srow * p.packed_cols + col]);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_empty_p + 8 * pslot);
-
-                uint32_t out[16];
-                dequant32<BITS>(w, scale, zero, out);
-
-                const uint32_t slot = it % p.S, par = ((it / p.S) & 1u) ^ 1u;
-                ok = mbar_wait(bar_empty + 8 * slot, par, abort_flag);
-                ok = __all_sync(0xFFFFFFFFu, ok);
-                if (!ok) break;
-                uint8_t* ws = smem_gen + p.off_w + slot * kWStageBytes + row_off;
+        for (int b = 0; b < 2; ++b) {
+            const int kb = kb0 + b * kb_stride;                   // 32-code block along k: 0..1 forward, 0..3 backward
+            w_off[b] = row_base + (TRANSPOSED ? (uint32_t)(kb >> 1) * 8192u : 0u);
+            chunk0[b] = (uint32_t)((TRANSPOSED ? (kb & 1) : kb) * 4);
+            srow[b] = TRANSPOSED ? (uint32_t)(((kb * 32) / p.g) % p.scale_rows) : 0u;
+        }
+        const uint32_t pcols = (uint32_t)p.packed_cols;
+        const int my_tiles = first_tile < p.n_tiles ? (p.n_tiles - first_tile + tile_stride - 1) / tile_stride : 0;
+        const int total = my_tiles * p.steps;
+        Ring ring_w, ring_p;
+        if (group == 1) { ring_w.advance(S); ring_p.advance(P); }
+        for (int it = group; it < total; it += 2) {
+            if (!warp_wait(bar_full_p + 8 * ring_p.slot, ring_p.phase, abort_flag, lane)) break;
+            const uint8_t* pk = smem_gen + p.off_p + ring_p.slot * p.packed_slot_bytes;
+            const uint32_t* pw = reinterpret_cast<const uint32_t*>(pk);
+            const __half* ps = reinterpret_cast<const __half*>(pk + p.words_bytes);
+            const __half* pz = reinterpret_cast<const __half*>(pk + p.words_bytes + p.scale_bytes);
+            uint32_t w[2][BITS];
+            __half sc[2], zp[2];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const int chunk = (chunk0 + c) ^ (row & 7);
-                    *reinterpret_cast<uint4*>(ws + chunk * 16) = make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
-                }
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_full_w + 8 * slot);
+            for (int b = 0; b < 2; ++b) {
+                const uint32_t kb = (uint32_t)(kb0 + b * kb_stride);
+#pragma unroll
+                for (int i = 0; i < BITS; ++i) w[b][i] = pw[(kb * BITS + i) * pcols + col];
+                sc[b] = ps[srow[b] * pcols + col];
+                zp[b] = pz[srow[b] * pcols + col];
             }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty_p + 8 * ring_p.slot);
+
+            uint32_t out[2][16];
+#pragma unroll
+            for (int b = 0; b < 2; ++b) dequant32<BITS>(w[b], group_params(sc[b], zp[b]), out[b]);
+
+            if (!warp_wait(bar_empty + 8 * ring_w.slot, ring_w.phase ^ 1u, abort_flag, lane)) break;
+            uint8_t* ws = smem_gen + p.off_w + ring_w.slot * kWStageBytes;
+#pragma unroll
+            for (int b = 0; b < 2; ++b)
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    *reinterpret_cast<uint4*>(ws + w_off[b] + (((chunk0[b] + c) ^ sw) << 4)) =
+                        make_uint4(out[b][4 * c], out[b][4 * c + 1], out[b][4 * c + 2], out[b][4 * c + 3]);
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_full_w + 8 * ring_w.slot);
+            ring_w.advance(S); ring_w.advance(S);
+            ring_p.advance(P); ring_p.advance(P);
         }
     }
 
+done:
     // ---------------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
