@@ -44,8 +44,7 @@ Workspace carve(const qlora_desc& d, int M) {
     w.p0_off = 0;
     w.p1_off = p;
     w.grad_off = 2 * p;
-    const size_t ga = lora_grad_scratch_bytes(M, d.K, d.r), gb = lora_grad_scratch_bytes(M, d.N, d.r);
-    w.total = w.grad_off + align_up(ga > gb ? ga : gb, 256);
+    w.total = w.grad_off + align_up(lora_grad_scratch_bytes(M, d.K, d.N, d.r), 256);
     if (w.total == 0) w.total = 256;
     return w;
 }
@@ -192,9 +191,7 @@ int qlora_bwd_lora(const qlora_desc* desc, int M, const void* X, const void* dY,
         if (rc != QLORA_OK) return rc;
         G = Gs;
     }
-    rc = launch_lora_grad(M, d.N, d.r, s, true, dY, H, dB, accumulate, ws + w.grad_off, st);
-    if (rc != QLORA_OK) return rc;
-    return launch_lora_grad(M, d.K, d.r, s, false, X, G, dA, accumulate, ws + w.grad_off, st);
+    return launch_lora_grads(M, d.K, d.N, d.r, s, X, dY, H, G, dA, dB, accumulate, ws + w.grad_off, st);
 }
 
 }  // extern "C"

@@ -22,10 +22,11 @@ int launch_simt_gemm(const qlora_desc& d, int M, bool transposed, const void* In
                      cudaStream_t st);
 // P[m, j] = sum_t In[m, t] * L(j, t);  l_is_A: L = A [r, K] (t = k) else L = B [N, r] (t = n).
 int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const void* L, float* P, cudaStream_t st);
-// Out = s * sum_m In[m, c] * P[m, j]; out_is_dB: Out[c * r + j] (dB [N, r]) else Out[j * C + c] (dA [r, K]).
-size_t lora_grad_scratch_bytes(int M, int C, int r);
-int launch_lora_grad(int M, int C, int r, float s, bool out_is_dB, const void* In, const float* P, float* Out,
-                     int accumulate, void* scratch, cudaStream_t st);
+// dB = s dY^T H [N, r] and dA = s G^T X [r, K] in one pair of launches (partial sums per row slice, then a fixed-order
+// reduction); scratch needs lora_grad_scratch_bytes().
+size_t lora_grad_scratch_bytes(int M, int K, int N, int r);
+int launch_lora_grads(int M, int K, int N, int r, float s, const void* X, const void* dY, const float* H, const float* G,
+                      float* dA, float* dB, int accumulate, void* scratch, cudaStream_t st);
 
 // umma_kernel.cu -- tcgen05 tensor-core kernel (both directions); same contract as launch_simt_gemm
 bool umma_supported(const qlora_desc& d, int M);

@@ -109,76 +109,111 @@ int launch_simt_gemm(const qlora_desc& d, int M, bool transposed, const void* In
 }
 
 // ------------------------------------------------------------------------------------------------------------
-// LoRA down-projections: H = X A^T (contraction over K) and G = dY B (contraction over N).  One warp per token row;
-// lanes stride over the contraction in 8-element (16-byte) vectors; 8 ranks at a time; warp-shuffle reduction.
+// LoRA down-projections: H = X A^T (contraction over K) and G = dY B (contraction over N), fp32 [M, r].
+// Skinny products bound by reading the activations once, so they use the warp-level mma.sync (m16n8k16, bf16 in,
+// fp32 accumulate): a block owns 16 token rows, its 8 warps stride over the contraction in steps of 32, and every lane
+// feeds the tensor core straight from two 16-byte row loads.  The 32 contraction indices of a step are assigned to the
+// fragments in a permuted order (lane q of a quad owns indices 8q..8q+7); activation and adapter fragments use the same
+// permutation, so the sum is unchanged.  The 8 per-warp partial tiles are added in warp order through shared memory
+// (fixed order: deterministic).
 // ------------------------------------------------------------------------------------------------------------
-template <bool L_IS_A>
-__global__ void __launch_bounds__(128)
+constexpr int LD_WARPS = 8;
+constexpr int LD_MAX_NT = 8;   // rank tiles of 8 (r <= 64)
+
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <bool L_IS_A, int NT>
+__global__ void __launch_bounds__(LD_WARPS * 32)
 lora_down_kernel(int M, int T, int r, const __nv_bfloat16* __restrict__ In, const __nv_bfloat16* __restrict__ L,
                  float* __restrict__ P) {
-    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    const int m = blockIdx.x * 4 + warp;
-    if (m >= M) return;
-    const __nv_bfloat16* row = In + (size_t)m * T;
-    for (int j0 = 0; j0 < r; j0 += 8) {
-        float acc[8] = {};
-        for (int t = lane * 8; t < T; t += 256) {
-            const uint4 xv = *reinterpret_cast<const uint4*>(row + t);
-            const float x[8] = {bf16_lo(xv.x), bf16_hi(xv.x), bf16_lo(xv.y), bf16_hi(xv.y),
-                                bf16_lo(xv.z), bf16_hi(xv.z), bf16_lo(xv.w), bf16_hi(xv.w)};
-            if (L_IS_A) {
+    __shared__ float red[LD_WARPS][NT][4][32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, q = lane & 3;
+    const int m_base = blockIdx.x * 16;
+    const int r0 = m_base + g, r1 = r0 + 8;
+    const __nv_bfloat16* row0 = In + (size_t)r0 * T;
+    const __nv_bfloat16* row1 = In + (size_t)r1 * T;
+    const bool v0 = r0 < M, v1 = r1 < M;
+    float acc[NT][4];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {   // A[j0 + j, t .. t+7]
-                    const uint4 lv = __ldg(reinterpret_cast<const uint4*>(L + (size_t)(j0 + j) * T + t));
-                    acc[j] += x[0] * bf16_lo(lv.x) + x[1] * bf16_hi(lv.x) + x[2] * bf16_lo(lv.y) + x[3] * bf16_hi(lv.y) +
-                              x[4] * bf16_lo(lv.z) + x[5] * bf16_hi(lv.z) + x[6] * bf16_lo(lv.w) + x[7] * bf16_hi(lv.w);
-                }
-            } else {
+    for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+#pragma unroll 2
+    for (int k0 = warp * 32; k0 < T; k0 += LD_WARPS * 32) {
+        const int k = k0 + q * 8;
+        const bool kin = k < T;                     // T is a multiple of 8
+        const uint4 xlo = (v0 && kin) ? *reinterpret_cast<const uint4*>(row0 + k) : zero4;
+        const uint4 xhi = (v1 && kin) ? *reinterpret_cast<const uint4*>(row1 + k) : zero4;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {   // B[t + i, j0 .. j0+7]
-                    const uint4 lv = __ldg(reinterpret_cast<const uint4*>(L + (size_t)(t + i) * r + j0));
-                    acc[0] = fmaf(x[i], bf16_lo(lv.x), acc[0]); acc[1] = fmaf(x[i], bf16_hi(lv.x), acc[1]);
-                    acc[2] = fmaf(x[i], bf16_lo(lv.y), acc[2]); acc[3] = fmaf(x[i], bf16_hi(lv.y), acc[3]);
-                    acc[4] = fmaf(x[i], bf16_lo(lv.z), acc[4]); acc[5] = fmaf(x[i], bf16_hi(lv.z), acc[5]);
-                    acc[6] = fmaf(x[i], bf16_lo(lv.w), acc[6]); acc[7] = fmaf(x[i], bf16_hi(lv.w), acc[7]);
+        for (int nt = 0; nt < NT; ++nt) {
+            const int j = nt * 8 + g;               // rank index of this lane's adapter fragment
+            uint4 lv = zero4;
+            if (kin && j < r) {
+                if (L_IS_A) {
+                    lv = __ldg(reinterpret_cast<const uint4*>(L + (size_t)j * T + k));            // A[j, k..k+7]
+                } else {
+                    uint32_t e[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) e[i] = __bfloat16_as_ushort(__ldg(L + (size_t)(k + i) * r + j));   // B[k+i, j]
+                    lv = make_uint4(e[0] | (e[1] << 16), e[2] | (e[3] << 16), e[4] | (e[5] << 16), e[6] | (e[7] << 16));
                 }
             }
+            mma_bf16_16816(acc[nt], xlo.x, xhi.x, xlo.y, xhi.y, lv.x, lv.y);
+            mma_bf16_16816(acc[nt], xlo.z, xhi.z, xlo.w, xhi.w, lv.z, lv.w);
         }
+    }
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            float v = acc[j];
+    for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
-            acc[j] = v;
-        }
-        if (lane < 8) {
-            float v = acc[0];
+        for (int c = 0; c < 4; ++c) red[warp][nt][c][lane] = acc[nt][c];
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < NT * 128; idx += LD_WARPS * 32) {
+        const int nt = idx >> 7, c = (idx >> 5) & 3, ln = idx & 31;
+        float v = 0.f;
 #pragma unroll
-            for (int j = 1; j < 8; ++j) v = (lane == j) ? acc[j] : v;
-            P[(size_t)m * r + j0 + lane] = v;
-        }
+        for (int w = 0; w < LD_WARPS; ++w) v += red[w][nt][c][ln];
+        const int row = m_base + (ln >> 2) + ((c & 2) ? 8 : 0);
+        const int col = nt * 8 + (ln & 3) * 2 + (c & 1);
+        if (row < M && col < r) P[(size_t)row * r + col] = v;
     }
 }
 
 int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const void* L, float* P, cudaStream_t st) {
     if (M == 0 || r == 0) return QLORA_OK;
-    const unsigned grid = (unsigned)((M + 3) / 4);
-    if (l_is_A) lora_down_kernel<true><<<grid, 128, 0, st>>>(M, T, r, (const __nv_bfloat16*)In, (const __nv_bfloat16*)L, P);
-    else        lora_down_kernel<false><<<grid, 128, 0, st>>>(M, T, r, (const __nv_bfloat16*)In, (const __nv_bfloat16*)L, P);
+    const unsigned grid = (unsigned)((M + 15) / 16);
+    const __nv_bfloat16* in = (const __nv_bfloat16*)In;
+    const __nv_bfloat16* l = (const __nv_bfloat16*)L;
+    const int nt = (r + 7) / 8;
+#define QLORA_LD(NTV)                                                                                  \
+    do {                                                                                               \
+        if (l_is_A) lora_down_kernel<true, NTV><<<grid, LD_WARPS * 32, 0, st>>>(M, T, r, in, l, P);   \
+        else        lora_down_kernel<false, NTV><<<grid, LD_WARPS * 32, 0, st>>>(M, T, r, in, l, P);  \
+    } while (0)
+    if (nt <= 1) QLORA_LD(1);
+    else if (nt <= 2) QLORA_LD(2);
+    else if (nt <= 4) QLORA_LD(4);
+    else QLORA_LD(8);
+#undef QLORA_LD
     return cudaGetLastError() == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
 }
 
 // ------------------------------------------------------------------------------------------------------------
-// LoRA gradients: Out(c, j) = s * sum_m In[m, c] * P[m, j]   (dB: In = dY, P = H;  dA: In = X, P = G).
-// Pass 1: each block owns 256 columns (2 per thread) and one slice of the token rows, keeps 2 x 8 fp32 sums per
-// thread per rank chunk and writes them to scratch[slice].  Pass 2 adds the slices in index order, so the result
-// does not depend on scheduling.
+// LoRA gradients: Out(c, j) = s * sum_m In[m, c] * P[m, j]   (dB: In = dY, P = H, C = N;  dA: In = X, P = G, C = K).
+// Bound by reading X and dY once.  Pass 1 (one launch for both gradients): a block owns 256 columns and one slice of
+// the token rows; each lane keeps an 8-column x 8-rank tile of fp32 sums, the block's four warps take interleaved rows
+// and are added in warp order through shared memory; the block writes its tile to scratch[slice].  Pass 2 adds the
+// slices in index order, scales by s and writes (or adds to) dA / dB.  Nothing depends on scheduling.
 // ------------------------------------------------------------------------------------------------------------
-constexpr int LG_COLS = 256;          // columns per block
+constexpr int LG_COLS = 256;          // columns per block (8 per lane)
 constexpr int LG_MAX_SLICES = 64;
 
-static int lora_grad_slices(int M, int C) {
-    const int col_blocks = (C + LG_COLS - 1) / LG_COLS;
+static int lora_grad_slices(int M, int K, int N) {
+    const int col_blocks = (K + LG_COLS - 1) / LG_COLS + (N + LG_COLS - 1) / LG_COLS;
     int slices = (4 * 148 + col_blocks - 1) / col_blocks;        // aim for ~4 blocks per SM
     const int max_by_rows = (M + 31) / 32;                       // at least 32 rows per slice
     if (slices > max_by_rows) slices = max_by_rows;
@@ -187,64 +222,106 @@ static int lora_grad_slices(int M, int C) {
     return slices;
 }
 
-size_t lora_grad_scratch_bytes(int M, int C, int r) {
-    return (size_t)lora_grad_slices(M, C) * (size_t)C * (size_t)r * sizeof(float);
+size_t lora_grad_scratch_bytes(int M, int K, int N, int r) {
+    return (size_t)lora_grad_slices(M, K, N) * (size_t)(K + N) * (size_t)r * sizeof(float);
 }
 
+struct GradSide {
+    const __nv_bfloat16* In;   // [M, C]
+    const float* P;            // [M, r]
+    float* partial;            // [slices][C][r]
+    float* Out;
+    int C;
+};
+
 __global__ void __launch_bounds__(128)
-lora_grad_partial_kernel(int M, int C, int r, int rows_per_slice, const __nv_bfloat16* __restrict__ In,
-                         const float* __restrict__ P, float* __restrict__ partial) {
-    const int c = blockIdx.x * LG_COLS + threadIdx.x * 2;
+lora_grad_partial_kernel(int M, int r, int rows_per_slice, GradSide side0, GradSide side1) {
+    __shared__ float red[4][64][32];
+    const GradSide& sd = blockIdx.z == 0 ? side0 : side1;
+    const int C = sd.C;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int cb = blockIdx.x * LG_COLS;
+    if (cb >= C) return;
+    const int c0 = cb + lane * 8;
+    const bool live = c0 < C;                                       // C is a multiple of 8
     const int slice = blockIdx.y;
     const int m_begin = slice * rows_per_slice;
     const int m_end = min(M, m_begin + rows_per_slice);
-    const bool live = c < C;                                       // C is even
-    float* out = partial + ((size_t)slice * C + c) * r;            // [slice][c][j]
     for (int j0 = 0; j0 < r; j0 += 8) {
-        float a0[8] = {}, a1[8] = {};
+        float acc[8][8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
         if (live) {
-            for (int m = m_begin; m < m_end; ++m) {
-                const uint32_t xv = *reinterpret_cast<const uint32_t*>(In + (size_t)m * C + c);
-                const float x0 = bf16_lo(xv), x1 = bf16_hi(xv);
-                const float4 p0 = __ldg(reinterpret_cast<const float4*>(P + (size_t)m * r + j0));
-                const float4 p1 = __ldg(reinterpret_cast<const float4*>(P + (size_t)m * r + j0 + 4));
-                const float p[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
+#pragma unroll 2
+            for (int m = m_begin + warp; m < m_end; m += 4) {
+                const uint4 xv = *reinterpret_cast<const uint4*>(sd.In + (size_t)m * C + c0);
+                const float4 p0 = __ldg(reinterpret_cast<const float4*>(sd.P + (size_t)m * r + j0));
+                const float4 p1 = __ldg(reinterpret_cast<const float4*>(sd.P + (size_t)m * r + j0 + 4));
+                const float x[8] = {bf16_lo(xv.x), bf16_hi(xv.x), bf16_lo(xv.y), bf16_hi(xv.y),
+                                    bf16_lo(xv.z), bf16_hi(xv.z), bf16_lo(xv.w), bf16_hi(xv.w)};
+                const float pj[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
 #pragma unroll
-                for (int j = 0; j < 8; ++j) { a0[j] = fmaf(x0, p[j], a0[j]); a1[j] = fmaf(x1, p[j], a1[j]); }
+                for (int i = 0; i < 8; ++i)
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(x[i], pj[j], acc[i][j]);
             }
-#pragma unroll
-            for (int j = 0; j < 8; ++j) { out[j0 + j] = a0[j]; out[r + j0 + j] = a1[j]; }
         }
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) red[warp][i * 8 + j][lane] = acc[i][j];
+        __syncthreads();
+        // 64 x 32 sums; thread t adds the four warps' values for 16 of them and writes partial[slice][c][j0 + j]
+        for (int e = threadIdx.x; e < 64 * 32; e += 128) {
+            const int ij = e >> 5, ln = e & 31;
+            const float v = ((red[0][ij][ln] + red[1][ij][ln]) + red[2][ij][ln]) + red[3][ij][ln];
+            const int c = cb + ln * 8 + (ij >> 3);
+            if (c < C) sd.partial[((size_t)slice * C + c) * r + j0 + (ij & 7)] = v;
+        }
+        __syncthreads();
     }
 }
 
-__global__ void lora_grad_reduce_kernel(int C, int r, int slices, float s, int out_is_dB, int accumulate,
-                                        const float* __restrict__ partial, float* __restrict__ Out) {
-    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;   // index into [C][r]
-    if (idx >= (size_t)C * r) return;
+__global__ void lora_grad_reduce_kernel(int r, int slices, float s, int accumulate, GradSide dB_side, GradSide dA_side) {
+    // elements [0, N*r): dB[n, j]; elements [N*r, N*r + K*r): dA (stored [r, K])
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t nb = (size_t)dB_side.C * r, na = (size_t)dA_side.C * r;
+    if (idx >= nb + na) return;
+    const bool is_dB = idx < nb;
+    const GradSide& sd = is_dB ? dB_side : dA_side;
+    const size_t e = is_dB ? idx : idx - nb;          // index into [C][r]
     float v = 0.f;
-    for (int sl = 0; sl < slices; ++sl) v += partial[(size_t)sl * C * r + idx];
+    for (int sl = 0; sl < slices; ++sl) v += sd.partial[(size_t)sl * sd.C * r + e];
     v *= s;
-    const int c = (int)(idx / r), j = (int)(idx % r);
-    float* dst = out_is_dB ? Out + idx : Out + (size_t)j * C + c;
+    const int c = (int)(e / r), j = (int)(e % r);
+    float* dst = is_dB ? sd.Out + e : sd.Out + (size_t)j * sd.C + c;
     *dst = accumulate ? (*dst + v) : v;
 }
 
-int launch_lora_grad(int M, int C, int r, float s, bool out_is_dB, const void* In, const float* P, float* Out,
-                     int accumulate, void* scratch, cudaStream_t st) {
-    if (r == 0 || C == 0) return QLORA_OK;
-    const size_t total = (size_t)C * r;
-    if (M == 0) {   // empty sum: dA = dB = 0 unless accumulating
-        if (!accumulate && cudaMemsetAsync(Out, 0, total * sizeof(float), st) != cudaSuccess) return QLORA_ERR_CUDA;
+int launch_lora_grads(int M, int K, int N, int r, float s, const void* X, const void* dY, const float* H, const float* G,
+                      float* dA, float* dB, int accumulate, void* scratch, cudaStream_t st) {
+    if (r == 0) return QLORA_OK;
+    if (M == 0) {   // empty sums: dA = dB = 0 unless accumulating
+        if (!accumulate) {
+            if (cudaMemsetAsync(dA, 0, (size_t)r * K * sizeof(float), st) != cudaSuccess) return QLORA_ERR_CUDA;
+            if (cudaMemsetAsync(dB, 0, (size_t)N * r * sizeof(float), st) != cudaSuccess) return QLORA_ERR_CUDA;
+        }
         return QLORA_OK;
     }
-    const int slices = lora_grad_slices(M, C);
+    const int slices = lora_grad_slices(M, K, N);
     const int rows_per_slice = (M + slices - 1) / slices;
-    dim3 grid((C + LG_COLS - 1) / LG_COLS, slices);
-    lora_grad_partial_kernel<<<grid, 128, 0, st>>>(M, C, r, rows_per_slice, (const __nv_bfloat16*)In, P, (float*)scratch);
+    float* part_dB = (float*)scratch;
+    float* part_dA = part_dB + (size_t)slices * N * r;
+    GradSide sB{(const __nv_bfloat16*)dY, H, part_dB, dB, N};
+    GradSide sA{(const __nv_bfloat16*)X, G, part_dA, dA, K};
+    const int cols = (N > K ? N : K);
+    dim3 grid((cols + LG_COLS - 1) / LG_COLS, slices, 2);
+    lora_grad_partial_kernel<<<grid, 128, 0, st>>>(M, r, rows_per_slice, sB, sA);
     if (cudaGetLastError() != cudaSuccess) return QLORA_ERR_CUDA;
-    lora_grad_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(C, r, slices, s, out_is_dB ? 1 : 0,
-                                                                              accumulate, (const float*)scratch, Out);
+    const size_t total = (size_t)(N + K) * r;
+    lora_grad_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(r, slices, s, accumulate, sB, sA);
     return cudaGetLastError() == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
 }
 
