@@ -51,7 +51,8 @@ enum {
     QLORA_ERR_ALIGNMENT = -3,   /* a tensor pointer is not 16-byte aligned */
     QLORA_ERR_WORKSPACE = -4,   /* workspace missing or smaller than qlora_workspace_bytes() */
     QLORA_ERR_CUDA = -5,        /* a CUDA runtime / driver call failed (launch, tensor-map encoding, ...) */
-    QLORA_ERR_TIMEOUT = -6      /* a bounded device-side wait gave up (reported by qlora_device_status) */
+    QLORA_ERR_TIMEOUT = -6,     /* a bounded device-side wait gave up (reported by qlora_device_status) */
+    QLORA_ERR_STATIC_LIMIT = -7 /* qlora_bwd_lora_static: the call needs more scratch than the built-in array holds */
 };
 
 /* Layer descriptor (host memory). */
@@ -90,6 +91,25 @@ int qlora_bwd_input(const qlora_desc* desc, int M, const void* dY, const int32_t
 int qlora_bwd_lora(const qlora_desc* desc, int M, const void* X, const void* dY, const void* A, const void* B,
                    const float* H, const float* G, float* dA, float* dB, int accumulate, void* workspace,
                    size_t workspace_bytes, void* cuda_stream);
+
+/* Size of the scratch array built into the library for qlora_bwd_lora_static (16 MiB, held by every GPU that loads
+ * the library until the process exits). */
+#define QLORA_STATIC_SCRATCH_BYTES (16u << 20)
+
+/* qlora_bwd_lora without a workspace argument, for callers that cannot allocate device memory when they call the
+ * library: a host that has handed the whole device to its own memory pool, or a step loop that forbids allocation calls
+ * because cudaMalloc / cudaFree synchronise the device.  The paper has no counterpart; this is a packaging variant of
+ * qlora_bwd_lora: same arguments otherwise, same kernels, same results bit for bit.  Its scratch is a fixed array of
+ * QLORA_STATIC_SCRATCH_BYTES inside the library; the call itself allocates and frees nothing.
+ *   - Limit: returns QLORA_ERR_STATIC_LIMIT, with nothing enqueued, when qlora_workspace_bytes(desc, M) exceeds
+ *     QLORA_STATIC_SCRATCH_BYTES (LLaMA-7B projections at M = 2048 with r <= 16 need 5 - 11 MiB).
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device
+ *     current) and remembers it; make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, which still holds what the previous call left there.  A call
+ *     overwrites every element it later reads, so nothing has to be cleared; but two calls whose kernels overlap on
+ *     the GPU (different streams, no ordering between them) race on it.  Keep the calls of one device in stream order. */
+int qlora_bwd_lora_static(const qlora_desc* desc, int M, const void* X, const void* dY, const void* A, const void* B,
+                          const float* H, const float* G, float* dA, float* dB, int accumulate, void* cuda_stream);
 
 /* Format utilities (Section 3.1: bit-packed INT32 storage).  codes: uint8 [K, N], one code per byte.
  * qlora_pack rejects nothing about code values: only the low `bits` bits of each byte are used. */

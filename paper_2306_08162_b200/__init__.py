@@ -4,8 +4,10 @@ The work is done by hand-written CUDA kernels behind the C ABI of include/qlora.
 Python binding (argument marshalling only).  There is no CPU or PyTorch fallback: every call raises if the CUDA
 library is missing.
 """
-from .binding import (QloraError, desc, library, library_path, qlora_bwd_input, qlora_bwd_lora, qlora_dequant, qlora_device_status,
+from .binding import (STATIC_SCRATCH_BYTES, QloraError, desc, library, library_path, qlora_bwd_input, qlora_bwd_lora,
+                      qlora_bwd_lora_static, qlora_dequant, qlora_device_status,
                       qlora_fwd, qlora_pack, qlora_status_string, qlora_unpack, qlora_workspace_bytes)
 
-__all__ = ["QloraError", "desc", "library", "library_path", "qlora_bwd_input", "qlora_bwd_lora", "qlora_dequant", "qlora_device_status",
+__all__ = ["STATIC_SCRATCH_BYTES", "QloraError", "desc", "library", "library_path", "qlora_bwd_input", "qlora_bwd_lora",
+           "qlora_bwd_lora_static", "qlora_dequant", "qlora_device_status",
            "qlora_fwd", "qlora_pack", "qlora_status_string", "qlora_unpack", "qlora_workspace_bytes"]

@@ -47,11 +47,12 @@ def library() -> ctypes.CDLL:
     lib.qlora_fwd.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.qlora_bwd_input.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.qlora_bwd_lora.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
+    lib.qlora_bwd_lora_static.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp]
     lib.qlora_pack.argtypes = [i32, i32, i32, vp, vp, vp]
     lib.qlora_unpack.argtypes = [i32, i32, i32, vp, vp, vp]
     lib.qlora_dequant.argtypes = [dp, vp, vp, vp, vp, vp]
     lib.qlora_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint), i32]
-    for name in ("qlora_workspace_bytes", "qlora_fwd", "qlora_bwd_input", "qlora_bwd_lora", "qlora_pack",
+    for name in ("qlora_workspace_bytes", "qlora_fwd", "qlora_bwd_input", "qlora_bwd_lora", "qlora_bwd_lora_static", "qlora_pack",
                  "qlora_unpack", "qlora_dequant", "qlora_device_status"):
         getattr(lib, name).restype = i32
     _lib = lib
@@ -115,6 +116,17 @@ def qlora_bwd_lora(d, M, X, dY, A, B, H, G, dA, dB, accumulate, workspace, strea
     _check(library().qlora_bwd_lora(ctypes.byref(d), int(M), _ptr(X), _ptr(dY), _ptr(A), _ptr(B), _ptr(H), _ptr(G),
                                     _ptr(dA), _ptr(dB), int(accumulate), _ptr(workspace), wb, _stream(stream)),
            "qlora_bwd_lora")
+
+
+STATIC_SCRATCH_BYTES = 16 << 20   # QLORA_STATIC_SCRATCH_BYTES
+
+
+def qlora_bwd_lora_static(d, M, X, dY, A, B, H, G, dA, dB, accumulate, stream=None):
+    """qlora_bwd_lora for callers that may not allocate device memory: no workspace argument, the scratch is an array
+    inside the library (STATIC_SCRATCH_BYTES).  Raises QloraError(-7) when the shape needs more than that."""
+    _check(library().qlora_bwd_lora_static(ctypes.byref(d), int(M), _ptr(X), _ptr(dY), _ptr(A), _ptr(B), _ptr(H), _ptr(G),
+                                           _ptr(dA), _ptr(dB), int(accumulate), _stream(stream)),
+           "qlora_bwd_lora_static")
 
 
 def qlora_pack(bits, K, N, codes, Q, stream=None):

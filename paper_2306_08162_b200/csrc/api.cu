@@ -62,6 +62,7 @@ const char* qlora_status_string(int status) {
         case QLORA_ERR_WORKSPACE: return "workspace missing or too small";
         case QLORA_ERR_CUDA: return "CUDA call failed";
         case QLORA_ERR_TIMEOUT: return "bounded device-side wait gave up";
+        case QLORA_ERR_STATIC_LIMIT: return "scratch need exceeds the library's built-in array";
         default: return "unknown status";
     }
 }
