@@ -36,7 +36,8 @@ constexpr int kWRows = 128;          // weight rows (MMA M) per tile: n in forwa
 constexpr int kStepC = 64;           // contraction elements per pipeline stage
 constexpr int kWStageBytes = kWRows * kStepC * 2;   // 16 KiB of bf16 per stage
 constexpr int kAccStride = 256;      // tensor-memory columns per accumulator buffer
-constexpr uint32_t kSpinLimit = 1u << 23;
+constexpr uint32_t kSpinLimit = 1u << 26;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any healthy wait, short enough not to look like a hang
 
 struct Params {
     int M, N, K, bits, g, r, r_pad;
@@ -76,11 +77,23 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok;
 }
-// Bounded wait.  Returns false when the kernel is aborting (this wait or another one ran out of polls).
+__device__ __forceinline__ uint64_t global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: gives up after kWaitLimitNs of wall time (or kSpinLimit polls).  Returns false when the kernel is
+// aborting (this wait or another one ran out).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    uint64_t t0 = 0;
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 63u) == 63u && *abort_flag) return false;
+        if ((i & 63u) == 63u) {
+            if (*abort_flag) return false;
+            const uint64_t now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) break;
+        }
     }
     *abort_flag = 1;
     atomicOr(&g_device_status, 1u);
@@ -486,6 +499,8 @@ int launch_impl(const CUtensorMap& ta, const CUtensorMap& tq, const CUtensorMap&
     return cudaGetLastError() == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
 }
 
+#include "umma_pair.cuh"
+
 }  // namespace
 
 bool umma_supported(const qlora_desc& d, int M) {
@@ -496,8 +511,68 @@ bool umma_supported(const qlora_desc& d, int M) {
     return true;
 }
 
+// CTA-pair kernel: 512 tokens x 256 weight rows per pair of SMs.  Used when there are more than 256 tokens.
+static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
+                            const void* zeros, const void* L, const float* Pmat, void* Out, cudaStream_t st) {
+    PairParams p{};
+    p.M = M; p.N = d.N; p.K = d.K; p.bits = d.bits; p.g = d.group_size; p.r = d.r; p.r_pad = (d.r + 15) / 16 * 16;
+    p.C = transposed ? d.K : d.N;
+    const int T = transposed ? d.N : d.K;
+    p.n_tok_tiles = (M + 4 * kPairTok - 1) / (4 * kPairTok);
+    const int n_w_tiles = (p.C + 2 * kPairW - 1) / (2 * kPairW);
+    p.n_tiles = p.n_tok_tiles * n_w_tiles;
+    p.steps = T / kStepC;
+    p.packed_cols = transposed ? 64 : 128;
+    p.packed_rows = (transposed ? 128 : 64) * d.bits / 32;
+    p.scale_rows = transposed ? (d.group_size >= 128 ? 1 : 128 / d.group_size) : 1;
+    p.words_bytes = (uint32_t)(p.packed_rows * p.packed_cols * 4);
+    p.scale_bytes = (uint32_t)(p.scale_rows * p.packed_cols * 2);
+    p.packed_slot_bytes = (p.words_bytes + 2 * p.scale_bytes + 127u) / 128u * 128u;
+    p.s = d.r > 0 ? d.alpha / (float)d.r : 0.f;
+    p.Pmat = Pmat; p.L = (const __nv_bfloat16*)L; p.Out = (__nv_bfloat16*)Out;
+
+    const uint32_t lora_l = (uint32_t)(kPairW * p.r_pad * 2), lora_p = (uint32_t)(2 * kPairTok * p.r_pad * 2);
+    const uint32_t budget = 232448 - 1024 /*alignment slack*/ - 2048 /*static, barriers, padding*/;
+    p.P = 4;
+    const uint32_t fixed = lora_l + lora_p + p.P * p.packed_slot_bytes + 512;
+    const uint32_t per_stage = kPairXStage + kWStageBytes;
+    int S = (int)((budget - fixed) / per_stage);
+    if (S > 8) S = 8;
+    if (S < 2) return QLORA_ERR_UNSUPPORTED;
+    p.S = S;
+    p.off_x = 0;
+    p.off_w = p.off_x + S * kPairXStage;
+    p.off_p = p.off_w + S * kWStageBytes;
+    p.off_lora_l = p.off_p + p.P * p.packed_slot_bytes;
+    p.off_lora_p = p.off_lora_l + lora_l;
+    p.off_bar = (p.off_lora_p + lora_p + 127u) / 128u * 128u;
+    const size_t smem_bytes = (size_t)p.off_bar + 512 + 1024;
+
+    CUtensorMap ta, tq, ts, tz;
+    if (!make_map_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, In, (uint64_t)T, (uint64_t)M, 64, (uint32_t)kPairTok, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_2d(&tq, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, Q, (uint64_t)d.N, (uint64_t)(d.K * d.bits / 32), (uint32_t)p.packed_cols, (uint32_t)p.packed_rows, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_map_2d(&ts, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, scales, (uint64_t)d.N, (uint64_t)(d.K / d.group_size), (uint32_t)p.packed_cols, (uint32_t)p.scale_rows, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_map_2d(&tz, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, zeros, (uint64_t)d.N, (uint64_t)(d.K / d.group_size), (uint32_t)p.packed_cols, (uint32_t)p.scale_rows, CU_TENSOR_MAP_SWIZZLE_NONE))
+        return QLORA_ERR_CUDA;
+
+    const int pairs = sm_count() / 2;
+    const int grid = 2 * (p.n_tiles < pairs ? p.n_tiles : pairs);
+#define QLORA_LAUNCH_PAIR(B)                                                                              \
+    return transposed ? launch_pair_impl<B, true>(ta, tq, ts, tz, p, smem_bytes, grid, st)                \
+                      : launch_pair_impl<B, false>(ta, tq, ts, tz, p, smem_bytes, grid, st)
+    switch (d.bits) {
+        case 2: QLORA_LAUNCH_PAIR(2);
+        case 3: QLORA_LAUNCH_PAIR(3);
+        case 4: QLORA_LAUNCH_PAIR(4);
+        case 8: QLORA_LAUNCH_PAIR(8);
+    }
+#undef QLORA_LAUNCH_PAIR
+    return QLORA_ERR_UNSUPPORTED;
+}
+
 int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
                      const void* zeros, const void* L, const float* Pmat, void* Out, cudaStream_t st) {
+    if (M > 256) return launch_umma_pair(d, M, transposed, In, Q, scales, zeros, L, Pmat, Out, st);
     Params p{};
     p.M = M; p.N = d.N; p.K = d.K; p.bits = d.bits; p.g = d.group_size; p.r = d.r; p.r_pad = (d.r + 15) / 16 * 16;
     p.C = transposed ? d.K : d.N;

@@ -1,0 +1,437 @@
+// CTA-pair variant of the tensor-core kernel (included by umma_kernel.cu, inside its anonymous namespace).
+//
+// Two CTAs on the two SMs of one TPC (a cluster of 2) work on one output tile of 512 tokens x 256 weight rows with
+// tcgen05.mma.cta_group::2 (M = 256 across the pair, N = 256):
+//   - tokens are the MMA's M side (A operand): each CTA stages 2 x 128 token rows per pipeline stage by TMA and owns the
+//     accumulator rows of those tokens in its own tensor memory (two accumulators of 256 columns = all 512 columns);
+//   - the dequantised weights are the N side (B operand): each CTA unpacks 128 weight rows per stage into its own shared
+//     memory; the tensor cores of the pair exchange the halves, so a dequantised weight is reused by 512 tokens and each
+//     SM reads only half of the weight operand and half of the activations a single-CTA tile would need.
+// Per stage and per SM this is 1024 tensor-core cycles against 32 KB of TMA fill, 16 KB of dequant stores and 64 KB of
+// operand reads, i.e. about half the shared-memory and L2 traffic per flop of the single-CTA kernel.
+//
+// The MMA is issued by one thread of the pair's first CTA (the leader).  Barriers the leader waits on (activation
+// tile landed, weight tile written, accumulators drained, LoRA operands staged) live in the leader's shared memory
+// and collect arrivals from both CTAs (remote mbarrier arrive / TMA complete_tx); barriers that both CTAs wait on
+// (stage free, accumulators complete) exist in both and are signalled by one multicast tcgen05.commit.
+// Every wait is bounded, as in the single-CTA kernel; the CTAs leave together through a cluster barrier.
+
+constexpr int kPairTok = 128;                          // token rows per CTA per accumulator
+constexpr int kPairW = 128;                            // weight rows per CTA (256 per pair tile)
+constexpr int kPairXSub = kPairTok * kStepC * 2;       // 16 KiB: one 128-token sub-tile of a stage
+constexpr int kPairXStage = 2 * kPairXSub;             // two accumulators' sub-tiles
+
+struct PairParams {
+    int M, N, K, bits, g, r, r_pad;
+    int C;                       // output columns (N forward, K backward)
+    int n_tok_tiles, n_tiles, steps;
+    int S, P;
+    int packed_cols, packed_rows, scale_rows;
+    uint32_t words_bytes, scale_bytes, packed_slot_bytes;
+    uint32_t off_x, off_w, off_p, off_lora_l, off_lora_p, off_bar;
+    float s;
+    const float* Pmat;           // H (forward) or G (backward), fp32 [M, r]
+    const __nv_bfloat16* L;      // B [N, r] (forward) or A [r, K] (backward)
+    __nv_bfloat16* Out;
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+// Bounded wait on a barrier that receives arrivals from the peer CTA.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    uint64_t t0 = 0;
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if ((i & 63u) == 63u) {
+            if (*abort_flag) return false;
+            const uint64_t now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) break;
+        }
+    }
+    *abort_flag = 1;
+    atomicOr(&g_device_status, 1u);
+    return false;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA tile load of a CTA pair: the transfer lands in this CTA's shared memory, its bytes are counted on `bar`, which may
+// be the leader's barrier (a shared::cluster address).  No multicast.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrive on the barrier at the same shared-memory offset in both CTAs of the pair once all MMAs issued so far complete.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+// Instruction descriptor for the pair: bf16 x bf16 -> fp32, M = 256 across the two CTAs.
+__device__ __forceinline__ uint32_t instr_desc_pair(uint32_t n_mma, uint32_t a_mn_major, uint32_t b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn_major << 15) | (b_mn_major << 16) | ((n_mma >> 3) << 17) |
+           ((256u >> 4) << 24);
+}
+
+template <int BITS, bool TRANSPOSED>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_q,
+                 const __grid_constant__ CUtensorMap tm_scales, const __grid_constant__ CUtensorMap tm_zeros,
+                 const PairParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag_s;
+    volatile int* abort_flag = &abort_flag_s;
+
+    const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem0 - smem_u32(smem_raw));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t S = (uint32_t)p.S, P = (uint32_t)p.P;
+    const uint32_t cta = cluster_ctarank();            // 0 = leader (issues the MMAs), 1 = follower
+    const int first_tile = (int)(blockIdx.x >> 1), tile_stride = (int)(gridDim.x >> 1);
+
+    // barriers (same offsets in both CTAs)
+    const uint32_t bar_full_x = smem0 + p.off_bar;          // [S] leader's: activation sub-tiles of both CTAs landed (TMA)
+    const uint32_t bar_full_w = bar_full_x + 8 * S;         // [S] leader's: weight tiles of both CTAs written
+    const uint32_t bar_empty = bar_full_w + 8 * S;          // [S] both: MMAs reading the stage have completed (multicast commit)
+    const uint32_t bar_full_p = bar_empty + 8 * S;          // [P] local: packed words + group parameters landed (TMA)
+    const uint32_t bar_empty_p = bar_full_p + 8 * P;        // [P] local: the dequant group has read them into registers
+    const uint32_t bar_acc_full = bar_empty_p + 8 * P;      // [1] both: accumulators complete (multicast commit)
+    const uint32_t bar_acc_empty = bar_acc_full + 8;        // [1] leader's: both CTAs' epilogues have drained the accumulators
+    const uint32_t bar_lora_full = bar_acc_empty + 8;       // [1] leader's: both CTAs' LoRA operand tiles staged
+
+    if (threadIdx.x == 0) {
+        abort_flag_s = 0;
+        for (uint32_t i = 0; i < S; ++i) {
+            mbar_init(bar_full_x + 8 * i, 1);
+            mbar_init(bar_full_w + 8 * i, 2 * kGroupWarps);
+            mbar_init(bar_empty + 8 * i, 1);
+        }
+        for (uint32_t i = 0; i < P; ++i) {
+            mbar_init(bar_full_p + 8 * i, 1);
+            mbar_init(bar_empty_p + 8 * i, kGroupWarps);
+        }
+        mbar_init(bar_acc_full, 1);
+        mbar_init(bar_acc_empty, 2 * kEpiWarps);
+        mbar_init(bar_lora_full, 2 * kEpiWarps);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {   // whole warp, in both CTAs: all 512 tensor-memory columns of each SM of the pair
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();        // the peer's barriers are initialised before anything arrives on them
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer: activation sub-tiles
+        if (lane == 0) {
+            Ring ring;
+            const uint32_t leader_full_x = map_to_cta(bar_full_x, 0);
+            for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride) {
+                const int m0 = (tile % p.n_tok_tiles) * (4 * kPairTok) + (int)cta * kPairTok;
+                for (int step = 0; step < p.steps; ++step) {
+                    if (!mbar_wait(bar_empty + 8 * ring.slot, ring.phase ^ 1u, abort_flag)) goto done;
+                    if (cta == 0) mbar_expect_tx(bar_full_x + 8 * ring.slot, 2 * kPairXStage);   // both CTAs' bytes
+                    const uint32_t dst = smem0 + p.off_x + ring.slot * kPairXStage;
+                    const uint32_t bar = leader_full_x + 8 * ring.slot;
+                    tma_load_2d_pair(dst, &tm_act, bar, step * kStepC, m0);
+                    tma_load_2d_pair(dst + kPairXSub, &tm_act, bar, step * kStepC, m0 + 2 * kPairTok);
+                    ring.advance(S);
+                }
+            }
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ TMA producer: packed codes, scales, zeros (local)
+        if (lane == 0) {
+            Ring ring;
+            const uint32_t tx_bytes = p.words_bytes + 2 * p.scale_bytes;
+            for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride) {
+                const int w0 = (tile / p.n_tok_tiles) * (2 * kPairW) + (int)cta * kPairW;
+                const int g_row = TRANSPOSED ? w0 / p.g : 0;
+                for (int step = 0; step < p.steps; ++step) {
+                    if (!mbar_wait(bar_empty_p + 8 * ring.slot, ring.phase ^ 1u, abort_flag)) goto done;
+                    const uint32_t dst = smem0 + p.off_p + ring.slot * p.packed_slot_bytes;
+                    const uint32_t bar = bar_full_p + 8 * ring.slot;
+                    mbar_expect_tx(bar, tx_bytes);
+                    const int c0 = step * kStepC;
+                    if (!TRANSPOSED) {
+                        const int gr = c0 / p.g;
+                        tma_load_2d(dst, &tm_q, bar, w0, c0 * BITS / 32);
+                        tma_load_2d(dst + p.words_bytes, &tm_scales, bar, w0, gr);
+                        tma_load_2d(dst + p.words_bytes + p.scale_bytes, &tm_zeros, bar, w0, gr);
+                    } else {
+                        tma_load_2d(dst, &tm_q, bar, c0, w0 * BITS / 32);
+                        tma_load_2d(dst + p.words_bytes, &tm_scales, bar, c0, g_row);
+                        tma_load_2d(dst + p.words_bytes + p.scale_bytes, &tm_zeros, bar, c0, g_row);
+                    }
+                    ring.advance(P);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (one thread of the leader CTA)
+        if (lane == 0 && cta == 0) {
+            const uint32_t idesc = instr_desc_pair(2 * kPairW, 0u, TRANSPOSED ? 1u : 0u);
+            const uint32_t idesc_lora = instr_desc_pair(2 * kPairW, 0u, 0u);
+            // activation sub-tile (A operand): contraction-contiguous rows of 128 B, 128-byte swizzle, 8-row groups 1024 B apart.
+            // weight tile (B operand): forward = the same layout (rows n); backward = rows are the contraction (n) with 64 k
+            //   contiguous: MN-major, 64-element atoms 8192 B apart (LBO), 8-row contraction groups 1024 B apart (SBO).
+            const uint64_t a_desc0 = smem_desc(smem0 + p.off_x, 16, 1024, 2);
+            const uint64_t b_desc0 = TRANSPOSED ? smem_desc(smem0 + p.off_w, 8192, 1024, 2) : smem_desc(smem0 + p.off_w, 16, 1024, 2);
+            constexpr uint32_t b_k16 = TRANSPOSED ? (2048u >> 4) : (32u >> 4);
+            Ring ring;
+            uint32_t tile_it = 0;
+            for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride, ++tile_it) {
+                if (!mbar_wait_cluster(bar_acc_empty, (tile_it & 1u) ^ 1u, abort_flag)) goto done;
+                tc_fence_after();
+                uint32_t acc = 0;
+                for (int step = 0; step < p.steps; ++step) {
+                    if (!mbar_wait(bar_full_x + 8 * ring.slot, ring.phase, abort_flag)) goto done;
+                    if (!mbar_wait_cluster(bar_full_w + 8 * ring.slot, ring.phase, abort_flag)) goto done;
+                    tc_fence_after();
+                    const uint64_t a_desc = a_desc0 + ring.slot * (uint32_t)(kPairXStage >> 4);
+                    const uint64_t b_desc = b_desc0 + ring.slot * (uint32_t)(kWStageBytes >> 4);
+#pragma unroll
+                    for (int a = 0; a < 2; ++a)
+#pragma unroll
+                        for (int k16 = 0; k16 < kStepC / 16; ++k16)
+                            tc_mma_pair(tmem_base + a * kAccStride, a_desc + a * (kPairXSub >> 4) + k16 * 2, b_desc + k16 * b_k16,
+                                        idesc, acc | (uint32_t)(k16 > 0));
+                    acc = 1;
+                    tc_commit_pair(bar_empty + 8 * ring.slot);
+                    ring.advance(S);
+                }
+                if (p.r > 0) {
+                    if (!mbar_wait_cluster(bar_lora_full, tile_it & 1u, abort_flag)) goto done;
+                    tc_fence_after();
+                    for (int a = 0; a < 2; ++a)
+                        for (int jb = 0; jb < p.r_pad / 16; ++jb) {
+                            // un-swizzled operands: 8-row x 16-byte core matrices 128 B apart (SBO), contraction halves LBO apart
+                            const uint64_t a_desc = smem_desc(smem0 + p.off_lora_p + a * (kPairTok * p.r_pad * 2) + jb * 2 * (kPairTok * 16),
+                                                              kPairTok * 16, 128, 0);
+                            const uint64_t b_desc = smem_desc(smem0 + p.off_lora_l + jb * 2 * (kPairW * 16), kPairW * 16, 128, 0);
+                            tc_mma_pair(tmem_base + a * kAccStride, a_desc, b_desc, idesc_lora, 1u);
+                        }
+                }
+                tc_commit_pair(bar_acc_full);
+            }
+        }
+    } else if (warp >= kEpiWarp0 && warp < kDequantWarp0) {
+        // ------------------------------------------------------------------ epilogue (+ LoRA operand staging), both CTAs
+        const int q = warp & 3;                      // tensor-memory lane quarter this warp may read
+        const int et = threadIdx.x - kEpiWarp0 * 32; // 0..127
+        const uint32_t leader_acc_empty = map_to_cta(bar_acc_empty, 0);
+        const uint32_t leader_lora_full = map_to_cta(bar_lora_full, 0);
+        uint32_t tile_it = 0;
+        for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride, ++tile_it) {
+            const int wt = tile / p.n_tok_tiles, tt = tile % p.n_tok_tiles;
+            const int w0 = wt * (2 * kPairW);                          // first weight row (output column) of the pair tile
+            const int m0 = tt * (4 * kPairTok) + (int)cta * kPairTok;  // this CTA's first token row of accumulator 0
+            if (p.r > 0) {
+                // (the previous tile's LoRA MMA has completed: its accumulator-full barrier was observed below)
+                uint8_t* ll = smem_gen + p.off_lora_l;
+                uint8_t* lp = smem_gen + p.off_lora_p;
+                {   // this CTA's 128 weight rows of B (forward) / columns of A (backward)
+                    const int row = et, wrow = w0 + (int)cta * kPairW + row;
+                    for (int jc = 0; jc < p.r_pad / 8; ++jc) {
+                        uint4 v = make_uint4(0, 0, 0, 0);
+                        if (jc * 8 < p.r && wrow < p.C) {
+                            if (!TRANSPOSED) {
+                                v = __ldg(reinterpret_cast<const uint4*>(p.L + (size_t)wrow * p.r + jc * 8));      // B[n, j..j+7]
+                            } else {
+                                uint32_t e[8];
+#pragma unroll
+                                for (int j = 0; j < 8; ++j)
+                                    e[j] = __bfloat16_as_ushort(__ldg(p.L + (size_t)(jc * 8 + j) * p.K + wrow));     // A[j, k]
+                                v = make_uint4(e[0] | (e[1] << 16), e[2] | (e[3] << 16), e[4] | (e[5] << 16), e[6] | (e[7] << 16));
+                            }
+                        }
+                        *reinterpret_cast<uint4*>(ll + jc * (kPairW * 16) + (row >> 3) * 128 + (row & 7) * 16) = v;
+                    }
+                }
+#pragma unroll
+                for (int a = 0; a < 2; ++a) {   // this CTA's token rows of s * H (or s * G) for both accumulators
+                    const int m = m0 + a * (2 * kPairTok) + et;
+                    for (int jc = 0; jc < p.r_pad / 8; ++jc) {
+                        uint4 v = make_uint4(0, 0, 0, 0);
+                        if (jc * 8 < p.r && m < p.M) {
+                            const float4 x = __ldg(reinterpret_cast<const float4*>(p.Pmat + (size_t)m * p.r + jc * 8));
+                            const float4 y = __ldg(reinterpret_cast<const float4*>(p.Pmat + (size_t)m * p.r + jc * 8 + 4));
+                            __nv_bfloat162 h0 = __floats2bfloat162_rn(p.s * x.x, p.s * x.y), h1 = __floats2bfloat162_rn(p.s * x.z, p.s * x.w);
+                            __nv_bfloat162 h2 = __floats2bfloat162_rn(p.s * y.x, p.s * y.y), h3 = __floats2bfloat162_rn(p.s * y.z, p.s * y.w);
+                            v = make_uint4(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1),
+                                           *reinterpret_cast<uint32_t*>(&h2), *reinterpret_cast<uint32_t*>(&h3));
+                        }
+                        *reinterpret_cast<uint4*>(lp + a * (kPairTok * p.r_pad * 2) + jc * (kPairTok * 16) + (et >> 3) * 128 + (et & 7) * 16) = v;
+                    }
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(leader_lora_full);
+            }
+            if (!warp_wait(bar_acc_full, tile_it & 1u, abort_flag, lane)) break;
+            tc_fence_after();
+            // thread = one token row; 32 consecutive output columns per tensor-memory load -> 64 contiguous bytes
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+            for (int a = 0; a < 2; ++a) {
+                const int m = m0 + a * (2 * kPairTok) + q * 32 + lane;
+                __nv_bfloat16* orow = p.Out + (size_t)m * p.C + w0;
+#pragma unroll 1
+                for (int cb = 0; cb < 2 * kPairW; cb += 32) {
+                    uint32_t v[32];
+                    tc_ld32(taddr + a * kAccStride + cb, v);
+                    tc_wait_ld();
+                    if (m < p.M) {
+#pragma unroll
+                        for (int c8 = 0; c8 < 4; ++c8) {
+                            if (w0 + cb + c8 * 8 < p.C) {   // C is a multiple of 8: a chunk of 8 columns is all-in or all-out
+                                uint32_t o[4];
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    const __nv_bfloat162 pr = __floats2bfloat162_rn(__uint_as_float(v[c8 * 8 + 2 * j]),
+                                                                                    __uint_as_float(v[c8 * 8 + 2 * j + 1]));
+                                    o[j] = *reinterpret_cast<const uint32_t*>(&pr);
+                                }
+                                *reinterpret_cast<uint4*>(orow + cb + c8 * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(leader_acc_empty);
+        }
+    } else if (warp >= kDequantWarp0) {
+        // ------------------------------------------------------------------ unpack + dequant of this CTA's 128 weight rows
+        const int group = (warp - kDequantWarp0) / kGroupWarps;    // 0 or 1: the groups take alternate stages
+        const int gt = threadIdx.x - (kDequantWarp0 + group * kGroupWarps) * 32;   // 0..127 inside the group
+        const int col = gt % p.packed_cols;                       // column of the packed tile (n in both directions)
+        const int kb0 = gt / p.packed_cols;                       // forward: 0; backward: 0..1
+        const int kb_stride = TRANSPOSED ? 2 : 1;                 // the thread's two code blocks are kb0 and kb0 + kb_stride
+        const uint32_t row_base = (uint32_t)(col >> 3) * 1024u + (uint32_t)(col & 7) * 128u;   // row `col` of a swizzled tile
+        const uint32_t sw = (uint32_t)(col & 7);
+        uint32_t w_off[2], chunk0[2], srow[2];
+#pragma unroll
+        for (int b = 0; b < 2; ++b) {
+            const int kb = kb0 + b * kb_stride;                   // 32-code block along k: 0..1 forward, 0..3 backward
+            w_off[b] = row_base + (TRANSPOSED ? (uint32_t)(kb >> 1) * 8192u : 0u);
+            chunk0[b] = (uint32_t)((TRANSPOSED ? (kb & 1) : kb) * 4);
+            srow[b] = TRANSPOSED ? (uint32_t)(((kb * 32) / p.g) % p.scale_rows) : 0u;
+        }
+        const uint32_t pcols = (uint32_t)p.packed_cols;
+        const uint32_t leader_full_w = map_to_cta(bar_full_w, 0);
+        const int my_tiles = first_tile < p.n_tiles ? (p.n_tiles - first_tile + tile_stride - 1) / tile_stride : 0;
+        const int total = my_tiles * p.steps;
+        Ring ring_w, ring_p;
+        if (group == 1) { ring_w.advance(S); ring_p.advance(P); }
+        for (int it = group; it < total; it += 2) {
+            if (!warp_wait(bar_full_p + 8 * ring_p.slot, ring_p.phase, abort_flag, lane)) break;
+            const uint8_t* pk = smem_gen + p.off_p + ring_p.slot * p.packed_slot_bytes;
+            const uint32_t* pw = reinterpret_cast<const uint32_t*>(pk);
+            const __half* ps = reinterpret_cast<const __half*>(pk + p.words_bytes);
+            const __half* pz = reinterpret_cast<const __half*>(pk + p.words_bytes + p.scale_bytes);
+            uint32_t w[2][BITS];
+            __half sc[2], zp[2];
+#pragma unroll
+            for (int b = 0; b < 2; ++b) {
+                const uint32_t kb = (uint32_t)(kb0 + b * kb_stride);
+#pragma unroll
+                for (int i = 0; i < BITS; ++i) w[b][i] = pw[(kb * BITS + i) * pcols + col];
+                sc[b] = ps[srow[b] * pcols + col];
+                zp[b] = pz[srow[b] * pcols + col];
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty_p + 8 * ring_p.slot);
+
+            uint32_t out[2][16];
+#pragma unroll
+            for (int b = 0; b < 2; ++b) dequant32<BITS>(w[b], group_params(sc[b], zp[b]), out[b]);
+
+            if (!warp_wait(bar_empty + 8 * ring_w.slot, ring_w.phase ^ 1u, abort_flag, lane)) break;
+            uint8_t* ws = smem_gen + p.off_w + ring_w.slot * kWStageBytes;
+#pragma unroll
+            for (int b = 0; b < 2; ++b)
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    *reinterpret_cast<uint4*>(ws + w_off[b] + (((chunk0[b] + c) ^ sw) << 4)) =
+                        make_uint4(out[b][4 * c], out[b][4 * c + 1], out[b][4 * c + 2], out[b][4 * c + 3]);
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(leader_full_w + 8 * ring_w.slot);
+            ring_w.advance(S); ring_w.advance(S);
+            ring_p.advance(P); ring_p.advance(P);
+        }
+    }
+
+done:
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {   // give copies that may still be in flight time to land before the CTA's memory is released
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    cluster_sync_all();   // neither CTA leaves (or frees tensor memory) while its peer may still signal it or read its operands
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+template <int BITS, bool TRANSPOSED>
+int launch_pair_impl(const CUtensorMap& ta, const CUtensorMap& tq, const CUtensorMap& ts, const CUtensorMap& tz, const PairParams& p,
+                     size_t smem_bytes, int grid, cudaStream_t st) {
+    static bool configured = false;
+    auto kern = umma_pair_kernel<BITS, TRANSPOSED>;
+    if (!configured) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024) != cudaSuccess) return QLORA_ERR_CUDA;
+        configured = true;
+    }
+    kern<<<grid, kThreads, smem_bytes, st>>>(ta, tq, ts, tz, p);
+    return cudaGetLastError() == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
+}

@@ -74,6 +74,19 @@ def test_edge_feature_counts(K, N):
     check_layer(qi.random_codes_layer(K=K, N=N, bits=2, group_size=g, r=16, alpha=32.0, M=40, seed=K + N))
 
 
+@pytest.mark.parametrize("M", [257, 300, 513, 1000])
+@pytest.mark.parametrize("bits,g,K,N", [(4, 128, 256, 320), (2, 64, 320, 256), (3, 64, 512, 192), (8, 128, 384, 576)])
+def test_token_counts_above_256_with_ragged_weight_tiles(M, bits, g, K, N):
+    """More than 256 tokens selects the CTA-pair kernel (512 tokens x 256 weight rows per tile); K and N here are
+    not multiples of 256, so the last weight tile is ragged in both directions, and M leaves a ragged token tile."""
+    check_layer(qi.random_codes_layer(K=K, N=N, bits=bits, group_size=g, r=8, alpha=16.0, M=M, seed=M + bits))
+
+
+@pytest.mark.parametrize("r", [0, 16, 64])
+def test_ranks_above_256_tokens(r):
+    check_layer(qi.random_codes_layer(K=256, N=512, bits=4, group_size=128, r=r, alpha=2.0 * max(r, 1), M=600, seed=r))
+
+
 @pytest.mark.parametrize("r", [0, 8, 16, 24, 32, 64])
 def test_ranks(r):
     check_layer(qi.random_codes_layer(K=256, N=384, bits=4, group_size=128, r=r, alpha=2.0 * max(r, 1), M=70, seed=r))
