@@ -111,14 +111,14 @@ int launch_simt_gemm(const qlora_desc& d, int M, bool transposed, const void* In
 // ------------------------------------------------------------------------------------------------------------
 // LoRA down-projections: H = X A^T (contraction over K) and G = dY B (contraction over N), fp32 [M, r].
 // Skinny products bound by reading the activations once, so they use the warp-level mma.sync (m16n8k16, bf16 in,
-// fp32 accumulate): a block owns 16 token rows, its 8 warps stride over the contraction in steps of 32, and every lane
-// feeds the tensor core straight from two 16-byte row loads.  The 32 contraction indices of a step are assigned to the
-// fragments in a permuted order (lane q of a quad owns indices 8q..8q+7); activation and adapter fragments use the same
-// permutation, so the sum is unchanged.  The 8 per-warp partial tiles are added in warp order through shared memory
-// (fixed order: deterministic).
+// fp32 accumulate) fed straight from 16-byte row loads: a block owns 16 token rows, its warps stride over the
+// contraction in steps of 32 and keep four steps of loads in flight.  The 32 contraction indices of a step are assigned
+// to the fragments in a permuted order (lane q of a quad owns indices 8q..8q+7); activation and adapter fragments use the
+// same permutation, so the sum is unchanged.  A [r, K] is contraction-contiguous and loads directly; B [N, r] is
+// rank-contiguous, so its 8 x 8 fragment tiles are loaded row-wise and transposed across the warp with movmatrix.
+// The per-warp partial tiles are added in warp order through shared memory (fixed order: deterministic).
 // ------------------------------------------------------------------------------------------------------------
-constexpr int LD_WARPS = 8;
-constexpr int LD_MAX_NT = 8;   // rank tiles of 8 (r <= 64)
+constexpr int LD_UNROLL = 4;
 
 __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
@@ -126,12 +126,18 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// Transpose an 8 x 8 matrix of 16-bit elements held across the warp (lane l: row l / 4, elements 2 (l % 4), +1).
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
 
-template <bool L_IS_A, int NT>
-__global__ void __launch_bounds__(LD_WARPS * 32)
+template <bool L_IS_A, int NT, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32)
 lora_down_kernel(int M, int T, int r, const __nv_bfloat16* __restrict__ In, const __nv_bfloat16* __restrict__ L,
                  float* __restrict__ P) {
-    __shared__ float red[LD_WARPS][NT][4][32];
+    __shared__ float red[WARPS][NT][4][32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, q = lane & 3;
     const int m_base = blockIdx.x * 16;
@@ -143,28 +149,41 @@ lora_down_kernel(int M, int T, int r, const __nv_bfloat16* __restrict__ In, cons
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
-#pragma unroll 2
-    for (int k0 = warp * 32; k0 < T; k0 += LD_WARPS * 32) {
-        const int k = k0 + q * 8;
-        const bool kin = k < T;                     // T is a multiple of 8
-        const uint4 xlo = (v0 && kin) ? *reinterpret_cast<const uint4*>(row0 + k) : zero4;
-        const uint4 xhi = (v1 && kin) ? *reinterpret_cast<const uint4*>(row1 + k) : zero4;
+    for (int kk = warp * 32; kk < T; kk += WARPS * 32 * LD_UNROLL) {
+        uint4 xlo[LD_UNROLL], xhi[LD_UNROLL];
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            const int j = nt * 8 + g;               // rank index of this lane's adapter fragment
-            uint4 lv = zero4;
-            if (kin && j < r) {
+        for (int u = 0; u < LD_UNROLL; ++u) {                 // all activation loads of the unrolled steps first
+            const int k = kk + u * WARPS * 32 + q * 8;         // T is a multiple of 8: 8 elements are all-in or all-out
+            xlo[u] = (v0 && k < T) ? *reinterpret_cast<const uint4*>(row0 + k) : zero4;
+            xhi[u] = (v1 && k < T) ? *reinterpret_cast<const uint4*>(row1 + k) : zero4;
+        }
+#pragma unroll
+        for (int u = 0; u < LD_UNROLL; ++u) {
+            const int k0 = kk + u * WARPS * 32;                // warp-uniform
+            if (k0 >= T) break;
+            const int k = k0 + q * 8;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                uint4 lv = zero4;
                 if (L_IS_A) {
-                    lv = __ldg(reinterpret_cast<const uint4*>(L + (size_t)j * T + k));            // A[j, k..k+7]
+                    const int j = nt * 8 + g;                  // rank index of this lane's adapter fragment
+                    if (k < T && j < r) lv = __ldg(reinterpret_cast<const uint4*>(L + (size_t)j * T + k));   // A[j, k..k+7]
                 } else {
-                    uint32_t e[8];
+                    // tile t: row rho (0..7) <-> n = k0 + 8 (rho / 2) + (rho % 2) + 2 t, columns = ranks 8 nt .. 8 nt + 7;
+                    // after the transpose lane (g, q) holds B[k0 + 8q + 2t, 8nt + g], B[k0 + 8q + 2t + 1, 8nt + g]
+                    uint32_t w[4];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) e[i] = __bfloat16_as_ushort(__ldg(L + (size_t)(k + i) * r + j));   // B[k+i, j]
-                    lv = make_uint4(e[0] | (e[1] << 16), e[2] | (e[3] << 16), e[4] | (e[5] << 16), e[6] | (e[7] << 16));
+                    for (int t = 0; t < 4; ++t) {
+                        const int n = k0 + 8 * (g >> 1) + (g & 1) + 2 * t;
+                        uint32_t v = 0;
+                        if (n < T && nt * 8 < r) v = __ldg(reinterpret_cast<const uint32_t*>(L + (size_t)n * r + nt * 8 + 2 * q));
+                        w[t] = movmatrix_trans(v);
+                    }
+                    lv = make_uint4(w[0], w[1], w[2], w[3]);
                 }
+                mma_bf16_16816(acc[nt], xlo[u].x, xhi[u].x, xlo[u].y, xhi[u].y, lv.x, lv.y);
+                mma_bf16_16816(acc[nt], xlo[u].z, xhi[u].z, xlo[u].w, xhi[u].w, lv.z, lv.w);
             }
-            mma_bf16_16816(acc[nt], xlo.x, xhi.x, xlo.y, xhi.y, lv.x, lv.y);
-            mma_bf16_16816(acc[nt], xlo.z, xhi.z, xlo.w, xhi.w, lv.z, lv.w);
         }
     }
 #pragma unroll
@@ -172,11 +191,11 @@ lora_down_kernel(int M, int T, int r, const __nv_bfloat16* __restrict__ In, cons
 #pragma unroll
         for (int c = 0; c < 4; ++c) red[warp][nt][c][lane] = acc[nt][c];
     __syncthreads();
-    for (int idx = threadIdx.x; idx < NT * 128; idx += LD_WARPS * 32) {
+    for (int idx = threadIdx.x; idx < NT * 128; idx += WARPS * 32) {
         const int nt = idx >> 7, c = (idx >> 5) & 3, ln = idx & 31;
         float v = 0.f;
 #pragma unroll
-        for (int w = 0; w < LD_WARPS; ++w) v += red[w][nt][c][ln];
+        for (int w = 0; w < WARPS; ++w) v += red[w][nt][c][ln];
         const int row = m_base + (ln >> 2) + ((c & 2) ? 8 : 0);
         const int col = nt * 8 + (ln & 3) * 2 + (c & 1);
         if (row < M && col < r) P[(size_t)row * r + col] = v;
@@ -189,15 +208,15 @@ int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const voi
     const __nv_bfloat16* in = (const __nv_bfloat16*)In;
     const __nv_bfloat16* l = (const __nv_bfloat16*)L;
     const int nt = (r + 7) / 8;
-#define QLORA_LD(NTV)                                                                                  \
-    do {                                                                                               \
-        if (l_is_A) lora_down_kernel<true, NTV><<<grid, LD_WARPS * 32, 0, st>>>(M, T, r, in, l, P);   \
-        else        lora_down_kernel<false, NTV><<<grid, LD_WARPS * 32, 0, st>>>(M, T, r, in, l, P);  \
+#define QLORA_LD(NTV, W)                                                                              \
+    do {                                                                                              \
+        if (l_is_A) lora_down_kernel<true, NTV, W><<<grid, W * 32, 0, st>>>(M, T, r, in, l, P);       \
+        else        lora_down_kernel<false, NTV, W><<<grid, W * 32, 0, st>>>(M, T, r, in, l, P);      \
     } while (0)
-    if (nt <= 1) QLORA_LD(1);
-    else if (nt <= 2) QLORA_LD(2);
-    else if (nt <= 4) QLORA_LD(4);
-    else QLORA_LD(8);
+    if (nt <= 1) QLORA_LD(1, 16);
+    else if (nt <= 2) QLORA_LD(2, 16);
+    else if (nt <= 4) QLORA_LD(4, 8);
+    else QLORA_LD(8, 8);
 #undef QLORA_LD
     return cudaGetLastError() == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
 }
@@ -205,25 +224,39 @@ int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const voi
 // ------------------------------------------------------------------------------------------------------------
 // LoRA gradients: Out(c, j) = s * sum_m In[m, c] * P[m, j]   (dB: In = dY, P = H, C = N;  dA: In = X, P = G, C = K).
 // Bound by reading X and dY once.  Pass 1 (one launch for both gradients): a block owns 256 columns and one slice of
-// the token rows; each lane keeps an 8-column x 8-rank tile of fp32 sums, the block's four warps take interleaved rows
-// and are added in warp order through shared memory; the block writes its tile to scratch[slice].  Pass 2 adds the
-// slices in index order, scales by s and writes (or adds to) dA / dB.  Nothing depends on scheduling.
+// the token rows; a warp owns 32 of the columns and runs mma.sync m16n8k16 with the ranks as the MMA's M side:
+//   D[j, c] += sum_m P^T[j, m] In[m, c]
+// The P^T fragments come from a bf16 copy of the slice's P rows staged (transposed) in shared memory; the In fragments
+// need pairs of consecutive m for a fixed column, so the 16-byte row loads (8 columns per lane) are transposed across
+// the warp with movmatrix.  This permutes which column each accumulator element belongs to (lane (g, q), tile c,
+// element e  <->  column 8q + 2c + e of the warp's 32), which the write-out undoes.  The block writes its tile to
+// scratch[slice]; pass 2 adds the slices in index order, scales by s and writes (or adds to) dA / dB.
+// Nothing depends on scheduling: the result is bitwise reproducible.
 // ------------------------------------------------------------------------------------------------------------
-constexpr int LG_COLS = 256;          // columns per block (8 per lane)
+constexpr int LG_COLS = 256;          // columns per block (32 per warp)
+constexpr int LG_WARPS = 8;
+constexpr int LG_UNROLL = 4;          // 16-row steps whose loads are issued together
 constexpr int LG_MAX_SLICES = 64;
 
-static int lora_grad_slices(int M, int K, int N) {
+struct GradPlan { int slices, rows_per_slice; };
+
+static GradPlan lora_grad_plan(int M, int K, int N) {
     const int col_blocks = (K + LG_COLS - 1) / LG_COLS + (N + LG_COLS - 1) / LG_COLS;
-    int slices = (4 * 148 + col_blocks - 1) / col_blocks;        // aim for ~4 blocks per SM
-    const int max_by_rows = (M + 31) / 32;                       // at least 32 rows per slice
-    if (slices > max_by_rows) slices = max_by_rows;
+    int slices = (3 * 148 + col_blocks - 1) / col_blocks;        // aim for ~3 blocks per SM
     if (slices > LG_MAX_SLICES) slices = LG_MAX_SLICES;
     if (slices < 1) slices = 1;
-    return slices;
+    int rows = (M + slices - 1) / slices;
+    rows = (rows + 63) / 64 * 64;                                // whole 16-row MMA steps; keeps the staged P^T conflict-free
+    if (rows < 64) rows = 64;
+    if (rows > 1024) rows = 1024;                                // bounds the staged P^T (64 ranks x 1032 x 2 B = 129 KiB at most)
+    GradPlan g;
+    g.rows_per_slice = rows;
+    g.slices = M > 0 ? (M + rows - 1) / rows : 1;
+    return g;
 }
 
 size_t lora_grad_scratch_bytes(int M, int K, int N, int r) {
-    return (size_t)lora_grad_slices(M, K, N) * (size_t)(K + N) * (size_t)r * sizeof(float);
+    return (size_t)lora_grad_plan(M, K, N).slices * (size_t)(K + N) * (size_t)r * sizeof(float);
 }
 
 struct GradSide {
@@ -234,54 +267,81 @@ struct GradSide {
     int C;
 };
 
-__global__ void __launch_bounds__(128)
+template <int RT>   // rank tiles of 16
+__global__ void __launch_bounds__(LG_WARPS * 32)
 lora_grad_partial_kernel(int M, int r, int rows_per_slice, GradSide side0, GradSide side1) {
-    __shared__ float red[4][64][32];
+    extern __shared__ __align__(16) uint8_t lg_smem[];
+    __nv_bfloat16* Pt = reinterpret_cast<__nv_bfloat16*>(lg_smem);   // [RT * 16][rows_per_slice + 8]
     const GradSide& sd = blockIdx.z == 0 ? side0 : side1;
     const int C = sd.C;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int cb = blockIdx.x * LG_COLS;
     if (cb >= C) return;
-    const int c0 = cb + lane * 8;
-    const bool live = c0 < C;                                       // C is a multiple of 8
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, q = lane & 3;
     const int slice = blockIdx.y;
     const int m_begin = slice * rows_per_slice;
-    const int m_end = min(M, m_begin + rows_per_slice);
-    for (int j0 = 0; j0 < r; j0 += 8) {
-        float acc[8][8];
+    const int stride = rows_per_slice + 8;                     // in bf16: (stride / 2) % 32 == 4 -> conflict-free fragment loads
+    constexpr int RP = RT * 16;
+    // stage P^T (bf16) of this slice: rows beyond M and ranks beyond r are zero
+    for (int e = threadIdx.x; e < rows_per_slice * RP; e += LG_WARPS * 32) {
+        const int ml = e / RP, j = e % RP;
+        const int m = m_begin + ml;
+        const float v = (m < M && j < r) ? __ldg(sd.P + (size_t)m * r + j) : 0.f;
+        Pt[j * stride + ml] = __float2bfloat16_rn(v);
+    }
+    __syncthreads();
+
+    const int c0 = cb + warp * 32 + q * 8;                     // this lane loads columns c0 .. c0 + 7
+    const bool live = c0 < C;                                  // C is a multiple of 8
+    const __nv_bfloat16* src = sd.In + c0;
+    float acc[RT][4][4];
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
+    for (int rt = 0; rt < RT; ++rt)
 #pragma unroll
-            for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
-        if (live) {
-#pragma unroll 2
-            for (int m = m_begin + warp; m < m_end; m += 4) {
-                const uint4 xv = *reinterpret_cast<const uint4*>(sd.In + (size_t)m * C + c0);
-                const float4 p0 = __ldg(reinterpret_cast<const float4*>(sd.P + (size_t)m * r + j0));
-                const float4 p1 = __ldg(reinterpret_cast<const float4*>(sd.P + (size_t)m * r + j0 + 4));
-                const float x[8] = {bf16_lo(xv.x), bf16_hi(xv.x), bf16_lo(xv.y), bf16_hi(xv.y),
-                                    bf16_lo(xv.z), bf16_hi(xv.z), bf16_lo(xv.w), bf16_hi(xv.w)};
-                const float pj[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
+        for (int c = 0; c < 4; ++c) acc[rt][c][0] = acc[rt][c][1] = acc[rt][c][2] = acc[rt][c][3] = 0.f;
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+    const int m_stop = min(M, m_begin + rows_per_slice);
+    for (int mm = m_begin; mm < m_stop; mm += 16 * LG_UNROLL) {
+        uint4 x0[LG_UNROLL], x1[LG_UNROLL];
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
+        for (int u = 0; u < LG_UNROLL; ++u) {
+            const int ma = mm + 16 * u + g, mb = ma + 8;
+            x0[u] = (live && ma < m_stop) ? *reinterpret_cast<const uint4*>(src + (size_t)ma * C) : zero4;
+            x1[u] = (live && mb < m_stop) ? *reinterpret_cast<const uint4*>(src + (size_t)mb * C) : zero4;
+        }
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(x[i], pj[j], acc[i][j]);
+        for (int u = 0; u < LG_UNROLL; ++u) {
+            const int ml = mm + 16 * u - m_begin;              // warp-uniform
+            if (ml >= rows_per_slice || mm + 16 * u >= m_stop) break;
+            uint32_t b0[4], b1[4];
+            b0[0] = movmatrix_trans(x0[u].x); b0[1] = movmatrix_trans(x0[u].y);
+            b0[2] = movmatrix_trans(x0[u].z); b0[3] = movmatrix_trans(x0[u].w);
+            b1[0] = movmatrix_trans(x1[u].x); b1[1] = movmatrix_trans(x1[u].y);
+            b1[2] = movmatrix_trans(x1[u].z); b1[3] = movmatrix_trans(x1[u].w);
+#pragma unroll
+            for (int rt = 0; rt < RT; ++rt) {
+                const __nv_bfloat16* pa = Pt + (rt * 16 + g) * stride + ml + 2 * q;
+                const uint32_t a0 = *reinterpret_cast<const uint32_t*>(pa);
+                const uint32_t a1 = *reinterpret_cast<const uint32_t*>(pa + 8 * stride);
+                const uint32_t a2 = *reinterpret_cast<const uint32_t*>(pa + 8);
+                const uint32_t a3 = *reinterpret_cast<const uint32_t*>(pa + 8 * stride + 8);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) mma_bf16_16816(acc[rt][c], a0, a1, a2, a3, b0[c], b1[c]);
             }
         }
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-#pragma unroll
-            for (int j = 0; j < 8; ++j) red[warp][i * 8 + j][lane] = acc[i][j];
-        __syncthreads();
-        // 64 x 32 sums; thread t adds the four warps' values for 16 of them and writes partial[slice][c][j0 + j]
-        for (int e = threadIdx.x; e < 64 * 32; e += 128) {
-            const int ij = e >> 5, ln = e & 31;
-            const float v = ((red[0][ij][ln] + red[1][ij][ln]) + red[2][ij][ln]) + red[3][ij][ln];
-            const int c = cb + ln * 8 + (ij >> 3);
-            if (c < C) sd.partial[((size_t)slice * C + c) * r + j0 + (ij & 7)] = v;
-        }
-        __syncthreads();
     }
+    // accumulator element (rt, c, i): rank rt*16 + g (+8 for i >= 2), column 8q + 2c + (i & 1) of the warp's 32
+    float* part = sd.partial + (size_t)slice * C * r;
+#pragma unroll
+    for (int rt = 0; rt < RT; ++rt)
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int j = rt * 16 + g + ((i & 2) ? 8 : 0);
+                const int col = cb + warp * 32 + q * 8 + 2 * c + (i & 1);
+                if (col < C && j < r) part[(size_t)col * r + j] = acc[rt][c][i];
+            }
 }
 
 __global__ void lora_grad_reduce_kernel(int r, int slices, float s, int accumulate, GradSide dB_side, GradSide dA_side) {
@@ -292,8 +352,15 @@ __global__ void lora_grad_reduce_kernel(int r, int slices, float s, int accumula
     const bool is_dB = idx < nb;
     const GradSide& sd = is_dB ? dB_side : dA_side;
     const size_t e = is_dB ? idx : idx - nb;          // index into [C][r]
+    const size_t step = (size_t)sd.C * r;
     float v = 0.f;
-    for (int sl = 0; sl < slices; ++sl) v += sd.partial[(size_t)sl * sd.C * r + e];
+    int sl = 0;
+    for (; sl + 4 <= slices; sl += 4) {               // four independent loads in flight, added in slice order
+        const float p0 = sd.partial[(size_t)sl * step + e], p1 = sd.partial[(size_t)(sl + 1) * step + e];
+        const float p2 = sd.partial[(size_t)(sl + 2) * step + e], p3 = sd.partial[(size_t)(sl + 3) * step + e];
+        v = (((v + p0) + p1) + p2) + p3;
+    }
+    for (; sl < slices; ++sl) v += sd.partial[(size_t)sl * step + e];
     v *= s;
     const int c = (int)(e / r), j = (int)(e % r);
     float* dst = is_dB ? sd.Out + e : sd.Out + (size_t)j * sd.C + c;
@@ -310,18 +377,35 @@ int launch_lora_grads(int M, int K, int N, int r, float s, const void* X, const 
         }
         return QLORA_OK;
     }
-    const int slices = lora_grad_slices(M, K, N);
-    const int rows_per_slice = (M + slices - 1) / slices;
+    const GradPlan plan = lora_grad_plan(M, K, N);
     float* part_dB = (float*)scratch;
-    float* part_dA = part_dB + (size_t)slices * N * r;
+    float* part_dA = part_dB + (size_t)plan.slices * N * r;
     GradSide sB{(const __nv_bfloat16*)dY, H, part_dB, dB, N};
     GradSide sA{(const __nv_bfloat16*)X, G, part_dA, dA, K};
     const int cols = (N > K ? N : K);
-    dim3 grid((cols + LG_COLS - 1) / LG_COLS, slices, 2);
-    lora_grad_partial_kernel<<<grid, 128, 0, st>>>(M, r, rows_per_slice, sB, sA);
+    dim3 grid((cols + LG_COLS - 1) / LG_COLS, plan.slices, 2);
+    const int rt = (r + 15) / 16;
+    const size_t smem = (size_t)rt * 16 * (plan.rows_per_slice + 8) * sizeof(__nv_bfloat16);
+#define QLORA_LG(RTV)                                                                                          \
+    do {                                                                                                       \
+        static bool configured = false;                                                                        \
+        if (!configured) {                                                                                     \
+            if (cudaFuncSetAttribute(lora_grad_partial_kernel<RTV>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                     RTV * 16 * (1024 + 8) * 2) != cudaSuccess) return QLORA_ERR_CUDA;          \
+            configured = true;                                                                                 \
+        }                                                                                                      \
+        lora_grad_partial_kernel<RTV><<<grid, LG_WARPS * 32, smem, st>>>(M, r, plan.rows_per_slice, sB, sA);   \
+    } while (0)
+    switch (rt) {
+        case 1: QLORA_LG(1); break;
+        case 2: QLORA_LG(2); break;
+        case 3: QLORA_LG(3); break;
+        default: QLORA_LG(4); break;
+    }
+#undef QLORA_LG
     if (cudaGetLastError() != cudaSuccess) return QLORA_ERR_CUDA;
     const size_t total = (size_t)(N + K) * r;
-    lora_grad_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(r, slices, s, accumulate, sB, sA);
+    lora_grad_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(r, plan.slices, s, accumulate, sB, sA);
     return cudaGetLastError() == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
 }
 
