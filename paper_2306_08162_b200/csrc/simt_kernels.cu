@@ -213,8 +213,8 @@ int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const voi
         if (l_is_A) lora_down_kernel<true, NTV, W><<<grid, W * 32, 0, st>>>(M, T, r, in, l, P);       \
         else        lora_down_kernel<false, NTV, W><<<grid, W * 32, 0, st>>>(M, T, r, in, l, P);      \
     } while (0)
-    if (nt <= 1) QLORA_LD(1, 16);
-    else if (nt <= 2) QLORA_LD(2, 16);
+    if (nt <= 1) QLORA_LD(1, 32);
+    else if (nt <= 2) QLORA_LD(2, 32);
     else if (nt <= 4) QLORA_LD(4, 8);
     else QLORA_LD(8, 8);
 #undef QLORA_LD

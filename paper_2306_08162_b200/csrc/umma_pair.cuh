@@ -314,32 +314,41 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             }
             if (!warp_wait(bar_acc_full, tile_it & 1u, abort_flag, lane)) break;
             tc_fence_after();
-            // thread = one token row; 32 consecutive output columns per tensor-memory load -> 64 contiguous bytes
+            // thread = one token row; 32 consecutive output columns per tensor-memory load -> 64 contiguous bytes.
+            // Two register buffers: the load of the next 32 columns is in flight while the current ones are stored.
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-#pragma unroll 1
-            for (int a = 0; a < 2; ++a) {
-                const int m = m0 + a * (2 * kPairTok) + q * 32 + lane;
-                __nv_bfloat16* orow = p.Out + (size_t)m * p.C + w0;
-#pragma unroll 1
-                for (int cb = 0; cb < 2 * kPairW; cb += 32) {
-                    uint32_t v[32];
-                    tc_ld32(taddr + a * kAccStride + cb, v);
-                    tc_wait_ld();
-                    if (m < p.M) {
+            const int m_a0 = m0 + q * 32 + lane;                       // this thread's token row in accumulator 0
+            auto store_chunk = [&](const uint32_t (&v)[32], int idx) {  // chunk idx: accumulator idx / 8, columns (idx % 8) * 32 ..
+                const int m = m_a0 + (idx >> 3) * (2 * kPairTok);
+                const int cb = (idx & 7) * 32;
+                if (m < p.M) {
+                    __nv_bfloat16* orow = p.Out + (size_t)m * p.C + w0 + cb;
 #pragma unroll
-                        for (int c8 = 0; c8 < 4; ++c8) {
-                            if (w0 + cb + c8 * 8 < p.C) {   // C is a multiple of 8: a chunk of 8 columns is all-in or all-out
-                                uint32_t o[4];
+                    for (int c8 = 0; c8 < 4; ++c8) {
+                        if (w0 + cb + c8 * 8 < p.C) {   // C is a multiple of 8: a chunk of 8 columns is all-in or all-out
+                            uint32_t o[4];
 #pragma unroll
-                                for (int j = 0; j < 4; ++j) {
-                                    const __nv_bfloat162 pr = __floats2bfloat162_rn(__uint_as_float(v[c8 * 8 + 2 * j]),
-                                                                                    __uint_as_float(v[c8 * 8 + 2 * j + 1]));
-                                    o[j] = *reinterpret_cast<const uint32_t*>(&pr);
-                                }
-                                *reinterpret_cast<uint4*>(orow + cb + c8 * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                            for (int j = 0; j < 4; ++j) {
+                                const __nv_bfloat162 pr = __floats2bfloat162_rn(__uint_as_float(v[c8 * 8 + 2 * j]),
+                                                                                __uint_as_float(v[c8 * 8 + 2 * j + 1]));
+                                o[j] = *reinterpret_cast<const uint32_t*>(&pr);
                             }
+                            *reinterpret_cast<uint4*>(orow + c8 * 8) = make_uint4(o[0], o[1], o[2], o[3]);
                         }
                     }
+                }
+            };
+            {
+                uint32_t va[32], vb[32];
+                tc_ld32(taddr, va);
+#pragma unroll 1
+                for (int idx = 0; idx < 16; idx += 2) {
+                    tc_wait_ld();
+                    tc_ld32(taddr + ((idx + 1) >> 3) * kAccStride + ((idx + 1) & 7) * 32, vb);
+                    store_chunk(va, idx);
+                    tc_wait_ld();
+                    if (idx + 2 < 16) tc_ld32(taddr + ((idx + 2) >> 3) * kAccStride + ((idx + 2) & 7) * 32, va);
+                    store_chunk(vb, idx + 1);
                 }
             }
             tc_fence_before();
