@@ -128,6 +128,14 @@ int qlora_fwd(const qlora_desc* desc, int M, const void* X, const int32_t* Q, co
     if (workspace == nullptr || workspace_bytes < w.total) return QLORA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     float* H = H_out ? H_out : reinterpret_cast<float*>(static_cast<char*>(workspace) + w.p0_off);
+    if (skinny_supported(d, M)) {
+        const bool fused = d.r > 0 && d.r <= 16;      // the down-projection rides along inside the kernel
+        if (d.r > 0 && !fused) {
+            rc = launch_lora_down(M, d.K, d.r, true, X, A, H, st);
+            if (rc != QLORA_OK) return rc;
+        }
+        return launch_skinny_gemm(d, M, false, X, Q, scales, zeros, A, B, H, !fused, Y, st);
+    }
     if (d.r > 0) {
         rc = launch_lora_down(M, d.K, d.r, true, X, A, H, st);
         if (rc != QLORA_OK) return rc;
@@ -153,6 +161,14 @@ int qlora_bwd_input(const qlora_desc* desc, int M, const void* dY, const int32_t
     if (workspace == nullptr || workspace_bytes < w.total) return QLORA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     float* G = G_out ? G_out : reinterpret_cast<float*>(static_cast<char*>(workspace) + w.p0_off);
+    if (skinny_supported(d, M)) {
+        const bool fused = d.r > 0 && d.r <= 16;
+        if (d.r > 0 && !fused) {
+            rc = launch_lora_down(M, d.N, d.r, false, dY, B, G, st);
+            if (rc != QLORA_OK) return rc;
+        }
+        return launch_skinny_gemm(d, M, true, dY, Q, scales, zeros, B, A, G, !fused, dX, st);
+    }
     if (d.r > 0) {
         rc = launch_lora_down(M, d.N, d.r, false, dY, B, G, st);
         if (rc != QLORA_OK) return rc;

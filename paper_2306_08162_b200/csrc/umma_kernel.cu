@@ -500,8 +500,67 @@ int launch_impl(const CUtensorMap& ta, const CUtensorMap& tq, const CUtensorMap&
 }
 
 #include "umma_pair.cuh"
+#include "skinny_kernel.cuh"
 
 }  // namespace
+
+bool skinny_supported(const qlora_desc& d, int M) {
+    if (M < 1 || M > 64) return false;
+    if (d.K < 32 || d.N < 8) return false;
+    return SK_STAGE % d.group_size == 0 || d.group_size % SK_STAGE == 0;   // a forward stage of 256 k holds whole groups
+}
+
+int launch_skinny_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
+                       const void* zeros, const void* Ldown, const void* Lup, float* P, bool p_is_input, void* Out,
+                       cudaStream_t st) {
+    SkinnyParams p{};
+    p.M = M; p.N = d.N; p.K = d.K; p.bits = d.bits; p.g = d.group_size; p.r = d.r;
+    p.T = transposed ? d.N : d.K;
+    p.C = transposed ? d.K : d.N;
+    p.stages_total = (p.T + SK_STAGE - 1) / SK_STAGE;
+    p.scale_rows = transposed ? 1 : (d.group_size < SK_STAGE ? SK_STAGE / d.group_size : 1);
+    p.words_bytes = (uint32_t)(d.bits * 1024);                       // 8 bits rows x 32 columns, or bits rows x 256 columns
+    p.scale_bytes = transposed ? (uint32_t)(SK_STAGE * 2) : (uint32_t)(p.scale_rows * SK_COLS * 2);
+    p.scale_stride = (p.scale_bytes + 127u) / 128u * 128u;
+    p.stage_bytes = p.words_bytes + 2 * p.scale_stride;
+    int S = (int)((160u * 1024u) / p.stage_bytes);
+    if (S > SK_MAX_STAGES) S = SK_MAX_STAGES;
+    if (S > p.stages_total) S = p.stages_total;
+    if (S < 1) S = 1;
+    p.S = S;
+    p.off_red = (uint32_t)S * p.stage_bytes;
+    p.off_p = p.off_red + SK_WARPS * 16 * 48 * 4;
+    p.off_bar = p.off_p + 16 * 16 * 4;
+    const size_t smem_bytes = (size_t)p.off_bar + 2 * 8 * SK_MAX_STAGES + 128;
+    p.s = d.r > 0 ? d.alpha / (float)d.r : 0.f;
+    p.In = (const __nv_bfloat16*)In; p.Ldown = (const __nv_bfloat16*)Ldown; p.Lup = (const __nv_bfloat16*)Lup;
+    p.P = P; p.p_is_input = p_is_input ? 1 : 0; p.Out = (__nv_bfloat16*)Out;
+    const int ntl = (d.r > 0 && !p_is_input) ? d.r / 8 : 0;          // fused down-projection tiles (r = 8 or 16)
+    if (ntl > 2) return QLORA_ERR_INVALID_ARG;
+
+    CUtensorMap tq, ts, tz;
+    const uint32_t bx = transposed ? SK_STAGE : SK_COLS;
+    const uint32_t by_q = transposed ? (uint32_t)d.bits : (uint32_t)(8 * d.bits);
+    if (!make_map_2d(&tq, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, Q, (uint64_t)d.N, (uint64_t)(d.K * d.bits / 32), bx, by_q, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_map_2d(&ts, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, scales, (uint64_t)d.N, (uint64_t)(d.K / d.group_size), bx, (uint32_t)p.scale_rows, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_map_2d(&tz, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, zeros, (uint64_t)d.N, (uint64_t)(d.K / d.group_size), bx, (uint32_t)p.scale_rows, CU_TENSOR_MAP_SWIZZLE_NONE))
+        return QLORA_ERR_CUDA;
+    dim3 grid((unsigned)((p.C + SK_COLS - 1) / SK_COLS), (unsigned)((M + 15) / 16));
+#define QLORA_SK(B, NT)                                                                                      \
+    return transposed ? launch_skinny_impl<B, NT, true>(tq, ts, tz, p, smem_bytes, grid, st)                \
+                      : launch_skinny_impl<B, NT, false>(tq, ts, tz, p, smem_bytes, grid, st)
+#define QLORA_SK_BITS(NT)                  \
+    switch (d.bits) {                      \
+        case 2: QLORA_SK(2, NT);           \
+        case 3: QLORA_SK(3, NT);           \
+        case 4: QLORA_SK(4, NT);           \
+        case 8: QLORA_SK(8, NT);           \
+    }
+    if (ntl == 0) { QLORA_SK_BITS(0) } else if (ntl == 1) { QLORA_SK_BITS(1) } else { QLORA_SK_BITS(2) }
+#undef QLORA_SK_BITS
+#undef QLORA_SK
+    return QLORA_ERR_UNSUPPORTED;
+}
 
 bool umma_supported(const qlora_desc& d, int M) {
     if (M < 1) return false;
