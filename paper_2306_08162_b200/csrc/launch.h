@@ -33,7 +33,7 @@ bool umma_supported(const qlora_desc& d, int M);
 int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q,
                      const void* scales, const void* zeros, const void* L, const float* P, void* Out,
                      cudaStream_t st);
-// Small token counts (M <= 64): TMA-fed mma.sync streaming kernels.  Ldown / Lup: the adapter applied first / second
+// Small token counts (M <= 32): TMA-fed mma.sync streaming kernels.  Ldown / Lup: the adapter applied first / second
 // (forward A, B; backward B, A).  P = H or G, fp32 [M, r]: read when p_is_input, otherwise computed inside the kernel
 // (ranks 8 and 16 only) and written out.
 bool skinny_supported(const qlora_desc& d, int M);

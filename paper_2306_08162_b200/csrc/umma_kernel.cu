@@ -505,9 +505,10 @@ int launch_impl(const CUtensorMap& ta, const CUtensorMap& tq, const CUtensorMap&
 }  // namespace
 
 bool skinny_supported(const qlora_desc& d, int M) {
-    if (M < 1 || M > 64) return false;
+    if (M < 1 || M > 32) return false;
     if (d.K < 32 || d.N < 8) return false;
-    return SK_STAGE % d.group_size == 0 || d.group_size % SK_STAGE == 0;   // a forward stage of 256 k holds whole groups
+    // a forward stage of 256 k and a backward tile of 128 k must hold whole groups (or lie inside one)
+    return (SK_STAGE % d.group_size == 0 || d.group_size % SK_STAGE == 0) && (SK_TILE % d.group_size == 0 || d.group_size % SK_TILE == 0);
 }
 
 int launch_skinny_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
@@ -518,37 +519,56 @@ int launch_skinny_gemm(const qlora_desc& d, int M, bool transposed, const void* 
     p.T = transposed ? d.N : d.K;
     p.C = transposed ? d.K : d.N;
     p.stages_total = (p.T + SK_STAGE - 1) / SK_STAGE;
-    p.scale_rows = transposed ? 1 : (d.group_size < SK_STAGE ? SK_STAGE / d.group_size : 1);
-    p.words_bytes = (uint32_t)(d.bits * 1024);                       // 8 bits rows x 32 columns, or bits rows x 256 columns
-    p.scale_bytes = transposed ? (uint32_t)(SK_STAGE * 2) : (uint32_t)(p.scale_rows * SK_COLS * 2);
-    p.scale_stride = (p.scale_bytes + 127u) / 128u * 128u;
-    p.stage_bytes = p.words_bytes + 2 * p.scale_stride;
-    int S = (int)((160u * 1024u) / p.stage_bytes);
-    if (S > SK_MAX_STAGES) S = SK_MAX_STAGES;
-    if (S > p.stages_total) S = p.stages_total;
-    if (S < 1) S = 1;
-    p.S = S;
-    p.off_red = (uint32_t)S * p.stage_bytes;
-    p.off_p = p.off_red + SK_WARPS * 16 * 48 * 4;
-    p.off_bar = p.off_p + 16 * 16 * 4;
-    const size_t smem_bytes = (size_t)p.off_bar + 2 * 8 * SK_MAX_STAGES + 128;
-    p.s = d.r > 0 ? d.alpha / (float)d.r : 0.f;
-    p.In = (const __nv_bfloat16*)In; p.Ldown = (const __nv_bfloat16*)Ldown; p.Lup = (const __nv_bfloat16*)Lup;
-    p.P = P; p.p_is_input = p_is_input ? 1 : 0; p.Out = (__nv_bfloat16*)Out;
+    // forward: packed tile 256 k x 128 n, group rows of the stage's 256 k; backward: 128 k x 256 n, group rows of the 128 k
+    const int span_k = transposed ? SK_TILE : SK_STAGE;
+    p.scale_rows = d.group_size < span_k ? span_k / d.group_size : 1;
+    p.words_bytes = (uint32_t)(d.bits * 4096);                       // 256 x 128 codes (either orientation)
+    p.scale_bytes = (uint32_t)(p.scale_rows * (transposed ? SK_STAGE : SK_TILE) * 2);
     const int ntl = (d.r > 0 && !p_is_input) ? d.r / 8 : 0;          // fused down-projection tiles (r = 8 or 16)
     if (ntl > 2) return QLORA_ERR_INVALID_ARG;
+    p.act_bytes = 16 * SK_STAGE * 2;                                 // 16 token rows x 256 contraction elements, bf16
+    p.l_bytes = ntl > 0 ? (uint32_t)(transposed ? SK_STAGE * d.r * 2 : 8 * ntl * SK_STAGE * 2) : 0u;
+    p.off_scale = p.words_bytes;
+    p.off_zero = p.off_scale + p.scale_bytes;                        // multiples of 512 bytes
+    p.off_act = (p.off_zero + p.scale_bytes + 1023u) / 1024u * 1024u;
+    p.off_l = p.off_act + p.act_bytes;
+    p.stage_bytes = (p.off_l + p.l_bytes + 1023u) / 1024u * 1024u;
+    const int my_stages = (p.stages_total + SK_SPLIT - 1) / SK_SPLIT;   // stages of the busiest CTA of a cluster
+    int S = (int)((200u * 1024u) / p.stage_bytes);
+    if (S > SK_MAX_STAGES) S = SK_MAX_STAGES;
+    if (S >= my_stages) S = my_stages;
+    else S = S / 2 * 2;   // even and odd stages have their own consumer warps: a slot must keep its parity lap after lap
+    if (S < 1) return QLORA_ERR_UNSUPPORTED;
+    p.S = S;
+    const uint32_t part_bytes = SK_PLANES * 16 * SK_PW * 4;                  // partial tiles; they reuse the ring after the main loop
+    const uint32_t ring_bytes = (uint32_t)S * p.stage_bytes;
+    p.off_p = (ring_bytes > part_bytes ? ring_bytes : part_bytes);
+    p.off_bar = p.off_p + 16 * 16 * 4;
+    const size_t smem_bytes = (size_t)p.off_bar + 2 * 8 * SK_MAX_STAGES + 1024;
+    p.s = d.r > 0 ? d.alpha / (float)d.r : 0.f;
+    p.Lup = (const __nv_bfloat16*)Lup;
+    p.P = P; p.p_is_input = p_is_input ? 1 : 0; p.Out = (__nv_bfloat16*)Out;
 
-    CUtensorMap tq, ts, tz;
-    const uint32_t bx = transposed ? SK_STAGE : SK_COLS;
-    const uint32_t by_q = transposed ? (uint32_t)d.bits : (uint32_t)(8 * d.bits);
-    if (!make_map_2d(&tq, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, Q, (uint64_t)d.N, (uint64_t)(d.K * d.bits / 32), bx, by_q, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+    CUtensorMap tq, ts, tz, ta, tl;
+    const uint32_t bx = transposed ? SK_STAGE : SK_TILE;             // packed columns (n) per box
+    const uint32_t by = (uint32_t)((transposed ? SK_TILE : SK_STAGE) / 32 * d.bits);   // packed rows per box
+    if (!make_map_2d(&tq, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, Q, (uint64_t)d.N, (uint64_t)(d.K * d.bits / 32), bx, by, CU_TENSOR_MAP_SWIZZLE_NONE) ||
         !make_map_2d(&ts, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, scales, (uint64_t)d.N, (uint64_t)(d.K / d.group_size), bx, (uint32_t)p.scale_rows, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-        !make_map_2d(&tz, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, zeros, (uint64_t)d.N, (uint64_t)(d.K / d.group_size), bx, (uint32_t)p.scale_rows, CU_TENSOR_MAP_SWIZZLE_NONE))
+        !make_map_2d(&tz, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, zeros, (uint64_t)d.N, (uint64_t)(d.K / d.group_size), bx, (uint32_t)p.scale_rows, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_map_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, In, (uint64_t)p.T, (uint64_t)M, 64, 16, CU_TENSOR_MAP_SWIZZLE_128B))
         return QLORA_ERR_CUDA;
-    dim3 grid((unsigned)((p.C + SK_COLS - 1) / SK_COLS), (unsigned)((M + 15) / 16));
+    if (ntl > 0) {
+        const bool ok = transposed
+            ? make_map_2d(&tl, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Ldown, (uint64_t)d.r, (uint64_t)d.N, (uint32_t)d.r, SK_STAGE, CU_TENSOR_MAP_SWIZZLE_NONE)
+            : make_map_2d(&tl, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Ldown, (uint64_t)d.K, (uint64_t)d.r, 64, (uint32_t)(8 * ntl), CU_TENSOR_MAP_SWIZZLE_128B);
+        if (!ok) return QLORA_ERR_CUDA;
+    } else {
+        tl = ta;   // unused by the kernel
+    }
+    dim3 grid(SK_SPLIT, (unsigned)((p.C + SK_TILE - 1) / SK_TILE), (unsigned)((M + 15) / 16));
 #define QLORA_SK(B, NT)                                                                                      \
-    return transposed ? launch_skinny_impl<B, NT, true>(tq, ts, tz, p, smem_bytes, grid, st)                \
-                      : launch_skinny_impl<B, NT, false>(tq, ts, tz, p, smem_bytes, grid, st)
+    return transposed ? launch_skinny_impl<B, NT, true>(tq, ts, tz, ta, tl, p, smem_bytes, grid, st)        \
+                      : launch_skinny_impl<B, NT, false>(tq, ts, tz, ta, tl, p, smem_bytes, grid, st)
 #define QLORA_SK_BITS(NT)                  \
     switch (d.bits) {                      \
         case 2: QLORA_SK(2, NT);           \
@@ -654,7 +674,9 @@ int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In
     // shared-memory plan (offsets from a 1024-byte aligned base)
     const uint32_t lora_a = (uint32_t)(kWRows * p.r_pad * 2), lora_p = (uint32_t)(p.BT * p.r_pad * 2);
     const uint32_t budget = 232448 - 1024 /*alignment slack*/ - 2048 /*static, barriers, padding*/;
-    p.P = 4;
+    // With few tokens the kernel is bound by the latency of streaming cold packed weights through a handful of CTAs,
+    // so the packed ring is deep (bytes in flight), at the cost of one or two operand stages.
+    p.P = p.BT <= 128 ? 16 : 8;
     const uint32_t fixed = lora_a + lora_p + p.P * p.packed_slot_bytes + 512;
     const uint32_t per_stage = p.x_stage_bytes + kWStageBytes;
     int S = (int)((budget - fixed) / per_stage);
