@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the quantized-linear + LoRA layer, forward + backward, at the LLaMA-7B q_proj shape.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME] [--no-graph]
 
 One "step" = qlora_fwd + qlora_bwd_input + qlora_bwd_lora on one projection (K = N = 4096, INT4, group 128,
 LoRA r = 8, alpha = 16, M = 2048 bf16 tokens; synthetic seeded inputs).  Consecutive steps rotate through several
@@ -31,13 +31,40 @@ if ROOT not in sys.path:
 
 METRIC = "fwd+bwd TFLOP/s & % roofline, INTn dequant-GEMM+LoRA at LLaMA-7B shapes"
 UNIT = "TFLOP/s"
-WORKLOAD = dict(K=4096, N=4096, bits=4, group_size=128, r=8, alpha=16.0, M=2048)
-WORKLOAD_NAME = "configs[1]: LLaMA-7B q_proj K=N=4096, INT4 group 128, LoRA r=8 alpha=16, M=2048 (4x512) bf16 tokens, fwd+bwd"
-ROTATION = 4                      # independent layer copies cycled through (4 x ~73 MiB > 126 MB of L2)
+# The default (and the headline) workload is configs[1]; the others are there to time and profile the other regimes.
+WORKLOADS = {
+    "config2": (dict(K=4096, N=4096, bits=4, group_size=128, r=8, alpha=16.0, M=2048),
+                "configs[1]: LLaMA-7B q_proj K=N=4096, INT4 group 128, LoRA r=8 alpha=16, M=2048 (4x512) bf16 tokens, fwd+bwd"),
+    "config3_gate": (dict(K=4096, N=11008, bits=2, group_size=64, r=16, alpha=32.0, M=2048),
+                     "configs[2]: LLaMA-7B gate_proj 4096->11008, INT2 group 64, LoRA r=16 alpha=32, M=2048, fwd+bwd"),
+    "config3_down": (dict(K=11008, N=4096, bits=2, group_size=64, r=16, alpha=32.0, M=2048),
+                     "configs[2]: LLaMA-7B down_proj 11008->4096, INT2 group 64, LoRA r=16 alpha=32, M=2048, fwd+bwd"),
+    "config4_int3_m8192": (dict(K=4096, N=4096, bits=3, group_size=128, r=8, alpha=16.0, M=8192),
+                           "configs[3]: K=N=4096, INT3 group 128, LoRA r=8, M=8192, fwd+bwd"),
+    "config4_int8_m128": (dict(K=4096, N=4096, bits=8, group_size=128, r=8, alpha=16.0, M=128),
+                          "configs[3]: K=N=4096, INT8 group 128, LoRA r=8, M=128, fwd+bwd"),
+    "config4_int3_m16": (dict(K=4096, N=4096, bits=3, group_size=128, r=8, alpha=16.0, M=16),
+                         "configs[3]: K=N=4096, INT3 group 128, LoRA r=8, M=16 (memory-bound), fwd+bwd"),
+    "config4_int8_m1": (dict(K=4096, N=4096, bits=8, group_size=128, r=8, alpha=16.0, M=1),
+                        "configs[3]: K=N=4096, INT8 group 128, LoRA r=8, M=1 (memory-bound), fwd+bwd"),
+}
+WORKLOAD, WORKLOAD_NAME = WORKLOADS["config2"]
+ROTATION = 4                      # independent layer copies cycled through; set in main() so that they exceed the L2
+
+
+def layer_bytes(w):
+    """Device footprint of one layer copy: packed weights, group parameters, activations, outputs."""
+    M, K, N, r = w["M"], w["K"], w["N"], w["r"]
+    return N * K * w["bits"] // 8 + 4 * N * K // w["group_size"] + 4 * M * (K + N) + 8 * r * (K + N) + 8 * M * r
+
+
+def weight_bytes(w):
+    return w["N"] * w["K"] * w["bits"] / 8 + 4 * w["N"] * w["K"] / w["group_size"]
 KERNELS_PER_STEP = None           # filled from the library's dispatch (see launches_per_step)
 
-# DRAM traffic per launch of the dominant kernel, from an ncu capture (profiles/); None until one is recorded.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# DRAM traffic (read + write) per launch of the dominant kernel of the default workload, from the ncu capture
+# summarised in profiles/umma_pair_config2_int4_m2048.md.  Set back to None whenever that kernel changes.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 25.89e6
 
 
 def layer_flops(M, K, N, r):
@@ -67,7 +94,7 @@ class ClockSampler:
                0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
                0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
 
-    def __init__(self, index: int, period_s: float = 0.05):
+    def __init__(self, index: int, period_s: float = 0.005):
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
@@ -211,9 +238,11 @@ def run_ours(args):
     def bf16(bits16):
         return torch.from_numpy(np.ascontiguousarray(bits16).view(np.int16)).to(dev).view(torch.bfloat16)
 
-    layers, host = [], []
+    layers, host, gen = [], [], []
     for i in range(ROTATION):
-        L = qi.config2(seed=10 * rank + i)
+        if i < 4:                                   # four distinct seeded layers; further copies reuse their values
+            gen.append(qi.make_layer(seed=1000 + 10 * rank + i, **w))   # (what matters for the rotation is distinct memory)
+        L = gen[i % 4]
         codes = torch.from_numpy(L["codes"]).to(dev)
         Q = torch.empty((K * w["bits"] // 32, N), dtype=torch.int32, device=dev)
         ql.qlora_pack(w["bits"], K, N, codes, Q)
@@ -263,6 +292,29 @@ def run_ours(args):
     total_ms = ev[0][0].elapsed_time(ev[-1][3])
     call_ms = [float(np.mean([ev[i][c].elapsed_time(ev[i][c + 1]) for i in range(args.steps)])) for c in range(3)]
 
+    eager_ms_per_step = total_ms / args.steps
+    if args.graph:
+        # The same K steps (same C-ABI calls, same rotation) captured once in a CUDA graph and replayed, so that the
+        # Python interpreter's per-call cost (tens of microseconds, more than some of the kernels) is not what is timed.
+        def graph_ms(body):
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr):
+                for i in range(args.steps):
+                    body(layers[i % ROTATION])
+            gr.replay()
+            barrier()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            g0.record(); gr.replay(); g1.record()
+            barrier()
+            return g0.elapsed_time(g1)
+        sampler = ClockSampler(local)
+        sampler.start()
+        total_ms = graph_ms(step)
+        clocks = sampler.stop()
+        call_ms = [graph_ms(lambda L: ql.qlora_fwd(d, M, L["X"], L["Q"], L["scales"], L["zeros"], L["A"], L["B"], L["Y"], L["H"], ws)) / args.steps,
+                   graph_ms(lambda L: ql.qlora_bwd_input(d, M, L["dY"], L["Q"], L["scales"], L["zeros"], L["A"], L["B"], L["dX"], L["G"], ws)) / args.steps,
+                   graph_ms(lambda L: ql.qlora_bwd_lora(d, M, L["X"], L["dY"], L["A"], L["B"], L["H"], L["G"], L["dA"], L["dB"], 0, ws)) / args.steps]
+
     # ---- end to end: pinned host inputs copied in, results copied out, every step --------------------------
     e2e_steps = max(3, min(args.steps, 50))
     s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -302,9 +354,18 @@ def run_ours(args):
         # dominant kernel: the dequant-GEMM of the forward or backward-input call, whichever takes longer
         dom = 0 if call_ms[0] >= call_ms[1] else 1
         dom_name = ("qlora_fwd", "qlora_bwd_input")[dom]
-        achieved = fwd_flops(M, K, N, r) / (call_ms[dom] * 1e-3) / 1e12
         long_run = total_ms > 1000.0
-        peak = peaks["bf16_sustained"] if long_run else peaks["bf16_burst"]
+        if M > 64:    # a dense contraction: tensor roofline
+            bound, r_unit = "tensor", "TFLOP/s"
+            achieved = fwd_flops(M, K, N, r) / (call_ms[dom] * 1e-3) / 1e12
+            peak = peaks["bf16_sustained"] if long_run else peaks["bf16_burst"]
+            peak_kind = f"{peaks['source']} cuBLAS bf16 {'sustained' if long_run else 'burst'}"
+        else:         # a few tokens: streaming the packed weights once is the bound
+            bound, r_unit = "hbm", "GB/s"
+            alg_bytes = weight_bytes(w) + 2 * M * (K + N) + 2 * r * (K + N)
+            achieved = alg_bytes / (call_ms[dom] * 1e-3) / 1e9
+            peak = peaks["hbm"]
+            peak_kind = f"{peaks['source']} HBM copy bandwidth"
         cpu = (time_oracle(target_seconds=20.0, steps=3, warmup=1) if not args.skip_cpu_baseline
                else dict(value=None, sample="skipped (--skip-cpu-baseline)"))
         line = {
@@ -312,16 +373,20 @@ def run_ours(args):
             "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD_NAME, "parallelism": "replicas only" if world > 1 else "single GPU",
-                       "l2": f"inputs larger than L2: steps rotate through {ROTATION} independent layer copies (~{ROTATION * 73} MiB)",
+                       "launch": ("the K steps' C-ABI calls captured in one CUDA graph, replayed once inside the timed region"
+                                  if args.graph else "one C-ABI call at a time from Python"),
+                       "eager_ms_per_step": eager_ms_per_step,
+                       "l2": f"inputs larger than L2: steps rotate through {ROTATION} independent layer copies "
+                             f"(~{ROTATION * layer_bytes(w) // 2**20} MiB)",
                        "calls_ms": {"qlora_fwd": call_ms[0], "qlora_bwd_input": call_ms[1], "qlora_bwd_lora": call_ms[2]}},
-            "roofline": {"bound": "tensor", "kernel": dom_name, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                         "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
-                         "peak_kind": f"{peaks['source']} cuBLAS bf16 {'sustained' if long_run else 'burst'}",
-                         "step_frac_of_peak": value / world / peak},
+            "roofline": {"bound": bound, "kernel": dom_name, "achieved": achieved, "peak": peak, "unit": r_unit,
+                         "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if args.workload == "config2" else None,
+                         "peak_kind": peak_kind,
+                         "step_frac_of_peak": (value / world / peak) if bound == "tensor" else None},
             "cpu_baseline": {"value": cpu["value"], "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": cpu["sample"]},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
-            "gpu_launches": launches_per_step(r) * args.steps,
+            "gpu_launches": launches_per_step(M, r) * args.steps,
             "clocks": clocks,
         }
         print(json.dumps(line))
@@ -330,10 +395,14 @@ def run_ours(args):
     return 0
 
 
-def launches_per_step(r: int) -> int:
-    """Kernels the library launches for one fwd + bwd_input + bwd_lora at the benchmark shape: the LoRA
-    down-projection and the dequant-GEMM for each of fwd and bwd_input, and two (partial, reduce) for each of dA, dB."""
-    return (2 + 2 + 4) if r > 0 else 2
+def launches_per_step(M: int, r: int) -> int:
+    """Kernels the library launches for one fwd + bwd_input + bwd_lora (H, G saved).  Up to 32 tokens the LoRA
+    down-projection is fused into the streaming kernel for r <= 16 (one launch per call); otherwise each of fwd and
+    bwd_input is a down-projection launch plus the dequant-GEMM.  The gradients are a partial-sum and a reduction launch."""
+    if r == 0:
+        return 2
+    per_call = 1 if (M <= 32 and r <= 16) else 2
+    return 2 * per_call + 2
 
 
 def main():
@@ -342,11 +411,19 @@ def main():
     ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="config2",
+                    help="layer shape to run (default: configs[1], the headline workload)")
+    ap.add_argument("--no-graph", dest="graph", action="store_false",
+                    help="time the K steps as issued call by call from Python instead of as one CUDA-graph replay "
+                         "(the default; the interpreter's per-call cost is otherwise part of every step)")
     ap.add_argument("--skip-cpu-baseline", action="store_true",
                     help="leave out the CPU-oracle timing leg (for profiler runs, where only the GPU launches matter)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    global WORKLOAD, WORKLOAD_NAME, ROTATION
+    WORKLOAD, WORKLOAD_NAME = WORKLOADS[args.workload]
+    ROTATION = max(4, -(-300 * 2**20 // layer_bytes(WORKLOAD)))     # > 126 MB of L2 with margin
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)
