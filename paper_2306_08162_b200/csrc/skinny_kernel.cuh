@@ -93,12 +93,6 @@ __device__ __forceinline__ uint32_t sk_movmatrix(uint32_t a) {
     return d;
 }
 __device__ __forceinline__ uint32_t sk_comp(const uint4& v, int i) { return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w)); }
-__device__ __forceinline__ float ld_cluster_f32(uint32_t cluster_addr) {
-    float v;
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr) : "memory");
-    return v;
-}
-
 // Producer warp.  Issuing a TMA load costs its thread some tens of nanoseconds, so the loads of a stage are spread over
 // four lanes and the ring slots over the lane quads: lanes 4 s .. 4 s + 3 own slot s and issue its stages in order (one
 // owner per slot keeps the parity waits on the slot's barriers one phase apart).

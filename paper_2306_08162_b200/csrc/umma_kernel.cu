@@ -44,6 +44,7 @@ struct Params {
     int C;               // output columns (N forward, K backward)
     int BT;              // token rows per tile (MMA N): 32, 64, 128 or 256
     int n_tok_tiles, n_tiles, steps;
+    int split;           // CTAs per cluster sharing one tile, each taking `steps` consecutive steps of the contraction (1 = no cluster)
     int S, P;            // stages of the activation/weight ring and of the packed ring
     int packed_cols;     // 128 forward, 64 backward
     int packed_rows;     // int32 rows per stage
@@ -135,6 +136,28 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ---------------------------------------------------------------- thread-block cluster helpers
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t cluster_addr) {
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr) : "memory");
+    return v;
+}
+
+
 // Shared-memory matrix descriptor (version 1).  Offsets in bytes; layout 0 = no swizzle, 2 = 128-byte swizzle.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo, uint32_t layout) {
     return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) |
@@ -204,7 +227,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
 
-    const int first_tile = blockIdx.x, tile_stride = gridDim.x;
+    // Few tokens give few tiles: the contraction of a tile is then split over a cluster of p.split CTAs (rank i takes steps
+    // i * p.steps ...), each accumulates its part in tensor memory, and the parts are added through distributed shared
+    // memory at the end.  One tile per cluster in that mode.
+    const int rank = p.split > 1 ? (int)cluster_ctarank() : 0;
+    const int first_tile = blockIdx.x / p.split, tile_stride = gridDim.x / p.split;
+    const int step0 = rank * p.steps;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer: activation tiles
@@ -216,7 +244,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                     if (!mbar_wait(bar_empty + 8 * ring.slot, ring.phase ^ 1u, abort_flag)) goto done;
                     const uint32_t bar = bar_full_x + 8 * ring.slot;
                     mbar_expect_tx(bar, p.x_stage_bytes);
-                    tma_load_2d(smem0 + p.off_x + ring.slot * p.x_stage_bytes, &tm_act, bar, step * kStepC, m0);
+                    tma_load_2d(smem0 + p.off_x + ring.slot * p.x_stage_bytes, &tm_act, bar, (step0 + step) * kStepC, m0);
                     ring.advance(S);
                 }
             }
@@ -235,7 +263,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                     const uint32_t dst = smem0 + p.off_p + ring.slot * p.packed_slot_bytes;
                     const uint32_t bar = bar_full_p + 8 * ring.slot;
                     mbar_expect_tx(bar, tx_bytes);
-                    const int c0 = step * kStepC;
+                    const int c0 = (step0 + step) * kStepC;
                     if (!TRANSPOSED) {
                         const int gr = c0 / p.g;
                         tma_load_2d(dst, &tm_q, bar, w0, c0 * BITS / 32);
@@ -285,7 +313,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                     tc_commit(bar_empty + 8 * ring.slot);
                     ring.advance(S);
                 }
-                if (p.r > 0) {
+                if (p.r > 0 && rank == 0) {   // the LoRA update goes into one rank's part only
                     if (!mbar_wait(bar_lora_full, tile_it & 1u, abort_flag)) goto done;
                     tc_fence_after();
                     for (int jb = 0; jb < p.r_pad / 16; ++jb) {
@@ -350,6 +378,20 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             tc_fence_after();
             const int c = w0 + q * 32 + lane;                 // output column owned by this thread
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccStride;
+            if (p.split > 1) {
+                // this rank's part of the tile, fp32 [token][128 weight rows], over the (now idle) operand ring
+                float* part = reinterpret_cast<float*>(smem_gen);
+#pragma unroll 1
+                for (int cb = 0; cb < p.BT; cb += 16) {
+                    uint32_t v[16];
+                    tc_ld16(taddr + cb, v);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) part[(cb + j) * kWRows + q * 32 + lane] = __uint_as_float(v[j]);
+                }
+                tc_fence_before();
+                break;
+            }
 #pragma unroll 1
             for (int cb = 0; cb < p.BT; cb += 16) {
                 uint32_t v[16];
@@ -441,6 +483,26 @@ done:
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
         __syncthreads();
     }
+    if (p.split > 1) {
+        // Add the ranks' parts in rank order (fixed order: deterministic); rank i finishes tokens i * BT / split ...
+        __syncwarp();
+        cluster_sync_all();
+        if (!*abort_flag && first_tile < p.n_tiles) {
+            const int wt = first_tile / p.n_tok_tiles, tt = first_tile % p.n_tok_tiles;
+            const int w0 = wt * kWRows, m0 = tt * p.BT;
+            const int tok_per_rank = p.BT / p.split;
+            const uint32_t part_addr = smem0;
+            for (int e = threadIdx.x; e < tok_per_rank * kWRows; e += kThreads) {
+                const int t = rank * tok_per_rank + e / kWRows, cw = e % kWRows;
+                float v = 0.f;
+                for (int rk = 0; rk < p.split; ++rk)
+                    v += ld_cluster_f32(map_to_cta(part_addr, (uint32_t)rk) + (uint32_t)((t * kWRows + cw) * 4));
+                if (m0 + t < p.M && w0 + cw < p.C) p.Out[(size_t)(m0 + t) * p.C + w0 + cw] = __float2bfloat16_rn(v);
+            }
+        }
+        __syncwarp();
+        cluster_sync_all();   // nobody leaves while a peer may still read its part
+    }
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
@@ -494,6 +556,19 @@ int launch_impl(const CUtensorMap& ta, const CUtensorMap& tq, const CUtensorMap&
     if (!configured) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024) != cudaSuccess) return QLORA_ERR_CUDA;
         configured = true;
+    }
+    if (p.split > 1) {   // one cluster of p.split CTAs per tile
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)grid);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = smem_bytes;
+        cfg.stream = st;
+        cudaLaunchAttribute attr{};
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = (unsigned)p.split; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, kern, ta, tq, ts, tz, p) == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
     }
     kern<<<grid, kThreads, smem_bytes, st>>>(ta, tq, ts, tz, p);
     return cudaGetLastError() == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
@@ -676,10 +751,14 @@ int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In
     const uint32_t budget = 232448 - 1024 /*alignment slack*/ - 2048 /*static, barriers, padding*/;
     // With few tokens the kernel is bound by the latency of streaming cold packed weights through a handful of CTAs,
     // so the packed ring is deep (bytes in flight), at the cost of one or two operand stages.
-    p.P = p.BT <= 128 ? 16 : 8;
-    const uint32_t fixed = lora_a + lora_p + p.P * p.packed_slot_bytes + 512;
     const uint32_t per_stage = p.x_stage_bytes + kWStageBytes;
-    int S = (int)((budget - fixed) / per_stage);
+    int S = 0;
+    uint32_t fixed = 0;
+    for (p.P = p.BT <= 128 ? 16 : 8; p.P >= 4; p.P -= 4) {   // the packed ring gives way until three operand stages fit
+        fixed = lora_a + lora_p + p.P * p.packed_slot_bytes + 512;
+        S = budget > fixed ? (int)((budget - fixed) / per_stage) : 0;
+        if (S >= 3 || p.P == 4) break;
+    }
     if (S > 8) S = 8;
     if (S < 2) return QLORA_ERR_UNSUPPORTED;
     p.S = S;
@@ -698,7 +777,15 @@ int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In
         !make_map_2d(&tz, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, zeros, (uint64_t)d.N, (uint64_t)(d.K / d.group_size), (uint32_t)p.packed_cols, (uint32_t)p.scale_rows, CU_TENSOR_MAP_SWIZZLE_NONE))
         return QLORA_ERR_CUDA;
 
-    const int grid = p.n_tiles < sm_count() ? p.n_tiles : sm_count();
+    // Few tiles (few tokens): split each tile's contraction over a cluster of 2 or 4 CTAs so that the whole GPU streams
+    // the weights.  Needs one tile per cluster, an even split of the steps, and room for the fp32 part in the operand ring.
+    p.split = 1;
+    for (int sp = 4; sp >= 2; sp /= 2) {
+        if (p.n_tiles * sp <= sm_count() && p.steps % sp == 0 && p.steps / sp >= 4 && p.BT % sp == 0 &&
+            (uint32_t)(kWRows * p.BT * 4) <= p.off_p) { p.split = sp; break; }
+    }
+    p.steps /= p.split;
+    const int grid = p.split > 1 ? p.n_tiles * p.split : (p.n_tiles < sm_count() ? p.n_tiles : sm_count());
 #define QLORA_LAUNCH(B)                                                                              \
     return transposed ? launch_impl<B, true>(ta, tq, ts, tz, p, smem_bytes, grid, st)                \
                       : launch_impl<B, false>(ta, tq, ts, tz, p, smem_bytes, grid, st)

@@ -97,6 +97,14 @@ def test_ranks_small_token_counts(r):
     check_layer(qi.random_codes_layer(K=384, N=256, bits=4, group_size=128, r=r, alpha=2.0 * max(r, 1), M=20, seed=40 + r))
 
 
+@pytest.mark.parametrize("M", [33, 100, 129, 256])
+@pytest.mark.parametrize("bits,g,K,N,r", [(4, 128, 1024, 256, 8), (2, 64, 2048, 192, 16), (3, 128, 512, 320, 0), (8, 64, 1536, 128, 64)])
+def test_mid_token_counts_split_contraction(M, bits, g, K, N, r):
+    """33 .. 256 tokens give few tiles of the single-CTA tensor-core kernel; the contraction is then split over a cluster
+    of 2 or 4 CTAs and the parts are added through distributed shared memory (K / 64 steps: 16, 32, 8, 24)."""
+    check_layer(qi.random_codes_layer(K=K, N=N, bits=bits, group_size=g, r=r, alpha=2.0 * max(r, 1), M=M, seed=M + bits + r))
+
+
 @pytest.mark.parametrize("r", [0, 16, 64])
 def test_ranks_above_256_tokens(r):
     check_layer(qi.random_codes_layer(K=256, N=512, bits=4, group_size=128, r=r, alpha=2.0 * max(r, 1), M=600, seed=r))
