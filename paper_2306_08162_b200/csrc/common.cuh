@@ -25,6 +25,14 @@ __device__ __forceinline__ __nv_bfloat16 dequant_one(uint32_t q, __half scale, _
     return __float2bfloat16_rn(__half2float(scale) * d);
 }
 
+// Programmatic dependent launch.  Every layer kernel is launched with the programmatic-stream-serialization attribute:
+// it may be scheduled while its predecessor in the stream is still running, does its own set-up (barriers, tensor memory,
+// descriptor fetches), and then blocks in pdl_wait() until the predecessor has completed and its writes are visible.
+// Nothing may read or write global memory before pdl_wait().  pdl_launch_dependents() at the top lets the successor be
+// scheduled as soon as every CTA of this grid has started.  This hides the launch latency between the six kernels of a step.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ float bf16_lo(uint32_t packed) { return __uint_as_float(packed << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t packed) { return __uint_as_float(packed & 0xFFFF0000u); }
 
@@ -112,6 +120,30 @@ __device__ __forceinline__ void dequant32(const uint32_t (&w)[BITS], const Group
             out[j / 2] = *reinterpret_cast<const uint32_t*>(&pr);
         }
     }
+}
+
+// Host side: launch with the programmatic-stream-serialization attribute (and an optional cluster width).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, unsigned cluster_x,
+                              Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attrs[2];
+    unsigned n = 0;
+    attrs[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attrs[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+    if (cluster_x > 1) {
+        attrs[n].id = cudaLaunchAttributeClusterDimension;
+        attrs[n].val.clusterDim.x = cluster_x; attrs[n].val.clusterDim.y = 1; attrs[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    cfg.attrs = attrs;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 
 }  // namespace qlora

@@ -19,6 +19,8 @@ __global__ void __launch_bounds__(256)
 simt_gemm_kernel(int bits, int g, int K, int N, int r, float s, int M, const __nv_bfloat16* __restrict__ In,
                  const uint32_t* __restrict__ Q, const __half* __restrict__ scales, const __half* __restrict__ zeros,
                  const __nv_bfloat16* __restrict__ L, const float* __restrict__ P, __nv_bfloat16* __restrict__ Out) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int T = TRANSPOSED ? N : K;   // contraction length
     const int C = TRANSPOSED ? K : N;   // output columns
     __shared__ float sIn[SG_BT][SG_BM + 4];
@@ -97,15 +99,16 @@ int launch_simt_gemm(const qlora_desc& d, int M, bool transposed, const void* In
     if (M == 0 || C == 0) return QLORA_OK;
     const float s = d.r > 0 ? d.alpha / (float)d.r : 0.f;
     dim3 grid((C + SG_BC - 1) / SG_BC, (M + SG_BM - 1) / SG_BM);
+    cudaError_t err;
     if (transposed)
-        simt_gemm_kernel<true><<<grid, 256, 0, st>>>(d.bits, d.group_size, d.K, d.N, d.r, s, M,
+        err = launch_pdl(simt_gemm_kernel<true>, grid, dim3(256), 0, st, 1, d.bits, d.group_size, d.K, d.N, d.r, s, M,
             (const __nv_bfloat16*)In, (const uint32_t*)Q, (const __half*)scales, (const __half*)zeros,
             (const __nv_bfloat16*)L, P, (__nv_bfloat16*)Out);
     else
-        simt_gemm_kernel<false><<<grid, 256, 0, st>>>(d.bits, d.group_size, d.K, d.N, d.r, s, M,
+        err = launch_pdl(simt_gemm_kernel<false>, grid, dim3(256), 0, st, 1, d.bits, d.group_size, d.K, d.N, d.r, s, M,
             (const __nv_bfloat16*)In, (const uint32_t*)Q, (const __half*)scales, (const __half*)zeros,
             (const __nv_bfloat16*)L, P, (__nv_bfloat16*)Out);
-    return cudaGetLastError() == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
+    return err == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
 }
 
 // ------------------------------------------------------------------------------------------------------------
@@ -138,6 +141,8 @@ __global__ void __launch_bounds__(WARPS * 32)
 lora_down_kernel(int M, int T, int r, const __nv_bfloat16* __restrict__ In, const __nv_bfloat16* __restrict__ L,
                  float* __restrict__ P) {
     __shared__ float red[WARPS][NT][4][32];
+    pdl_launch_dependents();
+    pdl_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, q = lane & 3;
     const int m_base = blockIdx.x * 16;
@@ -208,17 +213,18 @@ int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const voi
     const __nv_bfloat16* in = (const __nv_bfloat16*)In;
     const __nv_bfloat16* l = (const __nv_bfloat16*)L;
     const int nt = (r + 7) / 8;
+    cudaError_t err = cudaSuccess;
 #define QLORA_LD(NTV, W)                                                                              \
     do {                                                                                              \
-        if (l_is_A) lora_down_kernel<true, NTV, W><<<grid, W * 32, 0, st>>>(M, T, r, in, l, P);       \
-        else        lora_down_kernel<false, NTV, W><<<grid, W * 32, 0, st>>>(M, T, r, in, l, P);      \
+        if (l_is_A) err = launch_pdl(lora_down_kernel<true, NTV, W>, dim3(grid), dim3(W * 32), 0, st, 1, M, T, r, in, l, P);   \
+        else        err = launch_pdl(lora_down_kernel<false, NTV, W>, dim3(grid), dim3(W * 32), 0, st, 1, M, T, r, in, l, P);  \
     } while (0)
     if (nt <= 1) QLORA_LD(1, 32);
     else if (nt <= 2) QLORA_LD(2, 32);
     else if (nt <= 4) QLORA_LD(4, 8);
     else QLORA_LD(8, 8);
 #undef QLORA_LD
-    return cudaGetLastError() == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
+    return err == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
 }
 
 // ------------------------------------------------------------------------------------------------------------
@@ -271,6 +277,8 @@ template <int RT>   // rank tiles of 16
 __global__ void __launch_bounds__(LG_WARPS * 32)
 lora_grad_partial_kernel(int M, int r, int rows_per_slice, GradSide side0, GradSide side1) {
     extern __shared__ __align__(16) uint8_t lg_smem[];
+    pdl_launch_dependents();
+    pdl_wait();
     __nv_bfloat16* Pt = reinterpret_cast<__nv_bfloat16*>(lg_smem);   // [RT * 16][rows_per_slice + 8]
     const GradSide& sd = blockIdx.z == 0 ? side0 : side1;
     const int C = sd.C;
@@ -346,6 +354,8 @@ lora_grad_partial_kernel(int M, int r, int rows_per_slice, GradSide side0, GradS
 
 __global__ void lora_grad_reduce_kernel(int r, int slices, float s, int accumulate, GradSide dB_side, GradSide dA_side) {
     // elements [0, N*r): dB[n, j]; elements [N*r, N*r + K*r): dA (stored [r, K])
+    pdl_launch_dependents();
+    pdl_wait();
     const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     const size_t nb = (size_t)dB_side.C * r, na = (size_t)dA_side.C * r;
     if (idx >= nb + na) return;
@@ -386,6 +396,7 @@ int launch_lora_grads(int M, int K, int N, int r, float s, const void* X, const 
     dim3 grid((cols + LG_COLS - 1) / LG_COLS, plan.slices, 2);
     const int rt = (r + 15) / 16;
     const size_t smem = (size_t)rt * 16 * (plan.rows_per_slice + 8) * sizeof(__nv_bfloat16);
+    cudaError_t err = cudaSuccess;
 #define QLORA_LG(RTV)                                                                                          \
     do {                                                                                                       \
         static bool configured = false;                                                                        \
@@ -394,7 +405,7 @@ int launch_lora_grads(int M, int K, int N, int r, float s, const void* X, const 
                                      RTV * 16 * (1024 + 8) * 2) != cudaSuccess) return QLORA_ERR_CUDA;          \
             configured = true;                                                                                 \
         }                                                                                                      \
-        lora_grad_partial_kernel<RTV><<<grid, LG_WARPS * 32, smem, st>>>(M, r, plan.rows_per_slice, sB, sA);   \
+        err = launch_pdl(lora_grad_partial_kernel<RTV>, grid, dim3(LG_WARPS * 32), smem, st, 1, M, r, plan.rows_per_slice, sB, sA); \
     } while (0)
     switch (rt) {
         case 1: QLORA_LG(1); break;
@@ -403,10 +414,10 @@ int launch_lora_grads(int M, int K, int N, int r, float s, const void* X, const 
         default: QLORA_LG(4); break;
     }
 #undef QLORA_LG
-    if (cudaGetLastError() != cudaSuccess) return QLORA_ERR_CUDA;
+    if (err != cudaSuccess) return QLORA_ERR_CUDA;
     const size_t total = (size_t)(N + K) * r;
-    lora_grad_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(r, plan.slices, s, accumulate, sB, sA);
-    return cudaGetLastError() == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
+    err = launch_pdl(lora_grad_reduce_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st, 1, r, plan.slices, s, accumulate, sB, sA);
+    return err == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
 }
 
 }  // namespace qlora

@@ -182,6 +182,7 @@ __device__ __forceinline__ void sk_cluster_epilogue(const SkinnyParams& p, uint3
 }
 
 #define SK_COMMON_PROLOGUE()                                                                                         \
+    pdl_launch_dependents();                                                                                        \
     extern __shared__ uint8_t smem_raw[];                                                                           \
     __shared__ int abort_flag_s;                                                                                    \
     volatile int* abort_flag = &abort_flag_s;                                                                       \
@@ -200,7 +201,8 @@ __device__ __forceinline__ void sk_cluster_epilogue(const SkinnyParams& p, uint3
         for (int i = 0; i < p.S; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, SK_WARPS / 2); } \
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");                                          \
     }                                                                                                               \
-    __syncthreads();
+    __syncthreads();                                                                                                \
+    pdl_wait();   /* set-up done; from here on global memory is touched */
 
 // After the main loop: every consumer warp has read every stage this CTA loaded, so no TMA write is still to come and
 // the ring's memory can hold the partial tiles; then the cluster reduces them.  On an abort nothing is stored.
@@ -394,20 +396,21 @@ template <int BITS, int NTL, bool TRANSPOSED>
 int launch_skinny_impl(const CUtensorMap& tq, const CUtensorMap& ts, const CUtensorMap& tz, const CUtensorMap& ta, const CUtensorMap& tl,
                        const SkinnyParams& p, size_t smem_bytes, dim3 grid, cudaStream_t st) {
     static bool configured = false;
+    cudaError_t err;
     if (TRANSPOSED) {
         auto kern = skinny_bwd_kernel<BITS, NTL>;
         if (!configured) {
             if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024) != cudaSuccess) return QLORA_ERR_CUDA;
             configured = true;
         }
-        kern<<<grid, SK_THREADS, smem_bytes, st>>>(tq, ts, tz, ta, tl, p);
+        err = launch_pdl(kern, grid, dim3(SK_THREADS), smem_bytes, st, 1, tq, ts, tz, ta, tl, p);
     } else {
         auto kern = skinny_fwd_kernel<BITS, NTL>;
         if (!configured) {
             if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024) != cudaSuccess) return QLORA_ERR_CUDA;
             configured = true;
         }
-        kern<<<grid, SK_THREADS, smem_bytes, st>>>(tq, ts, tz, ta, tl, p);
+        err = launch_pdl(kern, grid, dim3(SK_THREADS), smem_bytes, st, 1, tq, ts, tz, ta, tl, p);
     }
-    return cudaGetLastError() == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
+    return err == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
 }

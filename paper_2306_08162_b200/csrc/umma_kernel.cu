@@ -184,6 +184,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag_s;
     volatile int* abort_flag = &abort_flag_s;
+    pdl_launch_dependents();
 
     const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem0 - smem_u32(smem_raw));
@@ -226,6 +227,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
+    pdl_wait();   // set-up done; from here on global memory is touched
 
     // Few tokens give few tiles: the contraction of a tile is then split over a cluster of p.split CTAs (rank i takes steps
     // i * p.steps ...), each accumulates its part in tensor memory, and the parts are added through distributed shared
@@ -557,21 +559,9 @@ int launch_impl(const CUtensorMap& ta, const CUtensorMap& tq, const CUtensorMap&
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024) != cudaSuccess) return QLORA_ERR_CUDA;
         configured = true;
     }
-    if (p.split > 1) {   // one cluster of p.split CTAs per tile
-        cudaLaunchConfig_t cfg{};
-        cfg.gridDim = dim3((unsigned)grid);
-        cfg.blockDim = dim3(kThreads);
-        cfg.dynamicSmemBytes = smem_bytes;
-        cfg.stream = st;
-        cudaLaunchAttribute attr{};
-        attr.id = cudaLaunchAttributeClusterDimension;
-        attr.val.clusterDim.x = (unsigned)p.split; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-        cfg.attrs = &attr;
-        cfg.numAttrs = 1;
-        return cudaLaunchKernelEx(&cfg, kern, ta, tq, ts, tz, p) == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
-    }
-    kern<<<grid, kThreads, smem_bytes, st>>>(ta, tq, ts, tz, p);
-    return cudaGetLastError() == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
+    // one cluster of p.split CTAs per tile when the contraction is split
+    return launch_pdl(kern, dim3((unsigned)grid), dim3(kThreads), smem_bytes, st, (unsigned)p.split, ta, tq, ts, tz, p) == cudaSuccess
+               ? QLORA_OK : QLORA_ERR_CUDA;
 }
 
 #include "umma_pair.cuh"

@@ -107,6 +107,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag_s;
     volatile int* abort_flag = &abort_flag_s;
+    pdl_launch_dependents();
 
     const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem0 - smem_u32(smem_raw));
@@ -150,6 +151,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     cluster_sync_all();        // the peer's barriers are initialised before anything arrives on them
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
+    pdl_wait();                // set-up done; from here on global memory is touched
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer: activation sub-tiles
@@ -427,6 +429,6 @@ int launch_pair_impl(const CUtensorMap& ta, const CUtensorMap& tq, const CUtenso
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024) != cudaSuccess) return QLORA_ERR_CUDA;
         configured = true;
     }
-    kern<<<grid, kThreads, smem_bytes, st>>>(ta, tq, ts, tz, p);
-    return cudaGetLastError() == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
+    return launch_pdl(kern, dim3((unsigned)grid), dim3(kThreads), smem_bytes, st, 1, ta, tq, ts, tz, p) == cudaSuccess
+               ? QLORA_OK : QLORA_ERR_CUDA;   // (the cluster width of 2 is a compile-time attribute of the kernel)
 }
