@@ -675,7 +675,8 @@ static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const v
     p.s = d.r > 0 ? d.alpha / (float)d.r : 0.f;
     p.Pmat = Pmat; p.L = (const __nv_bfloat16*)L; p.Out = (__nv_bfloat16*)Out;
 
-    const uint32_t lora_l = (uint32_t)(kPairW * p.r_pad * 2), lora_p = (uint32_t)(2 * kPairTok * p.r_pad * 2);
+    uint32_t lora_l = (uint32_t)(kPairW * p.r_pad * 2), lora_p = (uint32_t)(2 * kPairTok * p.r_pad * 2);
+    if (lora_l + lora_p < 8192) lora_p = 8192 - lora_l;   // the area doubles as the epilogue's staging slices (4 warps x 2 KiB)
     const uint32_t budget = 232448 - 1024 /*alignment slack*/ - 2048 /*static, barriers, padding*/;
     p.P = 4;
     const uint32_t fixed = lora_l + lora_p + p.P * p.packed_slot_bytes + 512;

@@ -302,28 +302,37 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             }
             if (!warp_wait(bar_acc_full, tile_it & 1u, abort_flag, lane)) break;
             tc_fence_after();
-            // thread = one token row; 32 consecutive output columns per tensor-memory load -> 64 contiguous bytes.
-            // Two register buffers: the load of the next 32 columns is in flight while the current ones are stored.
+            // Tensor memory hands each thread one token row: 32 consecutive output columns per load = 64 bytes of bf16.  Stored
+            // straight from there, one warp instruction would touch 32 different rows (32 cache lines, 16 bytes each), so the
+            // chunk takes a turn through a 2 KiB per-warp staging slice (in the LoRA operand area, idle by now): written by
+            // row, read back so that four lanes cover the 64 bytes of one row and an instruction covers 8 rows.  The 16-byte
+            // pieces are XOR-swizzled by row so that both passes are free of bank conflicts.  Two register buffers: the
+            // tensor-memory load of the next 32 columns is in flight while the current ones are converted and stored.
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-            const int m_a0 = m0 + q * 32 + lane;                       // this thread's token row in accumulator 0
+            uint8_t* slice = smem_gen + p.off_lora_l + (et >> 5) * 2048;
+            const int m_w0 = m0 + q * 32;                               // this warp's first token row in accumulator 0
             auto store_chunk = [&](const uint32_t (&v)[32], int idx) {  // chunk idx: accumulator idx / 8, columns (idx % 8) * 32 ..
-                const int m = m_a0 + (idx >> 3) * (2 * kPairTok);
-                const int cb = (idx & 7) * 32;
-                if (m < p.M) {
-                    __nv_bfloat16* orow = p.Out + (size_t)m * p.C + w0 + cb;
+                __syncwarp();                                           // the previous chunk has been read back
 #pragma unroll
-                    for (int c8 = 0; c8 < 4; ++c8) {
-                        if (w0 + cb + c8 * 8 < p.C) {   // C is a multiple of 8: a chunk of 8 columns is all-in or all-out
-                            uint32_t o[4];
+                for (int c8 = 0; c8 < 4; ++c8) {
+                    uint32_t o[4];
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const __nv_bfloat162 pr = __floats2bfloat162_rn(__uint_as_float(v[c8 * 8 + 2 * j]),
-                                                                                __uint_as_float(v[c8 * 8 + 2 * j + 1]));
-                                o[j] = *reinterpret_cast<const uint32_t*>(&pr);
-                            }
-                            *reinterpret_cast<uint4*>(orow + c8 * 8) = make_uint4(o[0], o[1], o[2], o[3]);
-                        }
+                    for (int j = 0; j < 4; ++j) {
+                        const __nv_bfloat162 pr = __floats2bfloat162_rn(__uint_as_float(v[c8 * 8 + 2 * j]),
+                                                                        __uint_as_float(v[c8 * 8 + 2 * j + 1]));
+                        o[j] = *reinterpret_cast<const uint32_t*>(&pr);
                     }
+                    *reinterpret_cast<uint4*>(slice + lane * 64 + ((c8 ^ ((lane >> 1) & 3)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                }
+                __syncwarp();
+                const int cb = (idx & 7) * 32 + (lane & 3) * 8;         // this lane's 8 columns of the chunk
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int R = 8 * i + (lane >> 2);
+                    const uint4 val = *reinterpret_cast<const uint4*>(slice + R * 64 + (((lane & 3) ^ ((R >> 1) & 3)) << 4));
+                    const int m = m_w0 + (idx >> 3) * (2 * kPairTok) + R;
+                    if (m < p.M && w0 + cb < p.C)                       // C is a multiple of 8: 8 columns are all-in or all-out
+                        *reinterpret_cast<uint4*>(p.Out + (size_t)m * p.C + w0 + cb) = val;
                 }
             };
             {
