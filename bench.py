@@ -212,6 +212,22 @@ def run_reference(args):
 # --------------------------------------------------------------------------------------------------------------
 # the GPU arm
 # --------------------------------------------------------------------------------------------------------------
+def max_over_ranks(times_ms, world, device):
+    """The job's time is the slowest rank's: element-wise MAX of the per-rank device times over the process group
+    (the only collective in this benchmark: the layer itself has no exchange step).  Identity for a single rank."""
+    import torch
+    t = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def aggregate_value(flops_per_step, steps, world, total_ms):
+    """Whole-job throughput in TFLOP/s: every rank runs the same work (weak scaling), timed by the slowest rank."""
+    return flops_per_step * steps * world / (total_ms * 1e-3) / 1e12
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -341,15 +357,12 @@ def run_ours(args):
     h2d = 2 * M * (K + N)
     d2h = 2 * M * (K + N) + 4 * r * (K + N)
 
-    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = float(times[0]), float(times[1])
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], world, dev)
 
     if rank == 0:
         flops_step = layer_flops(M, K, N, r)
-        value = flops_step * args.steps * world / (total_ms * 1e-3) / 1e12
-        e2e_value = flops_step * e2e_steps * world / (e2e_ms * 1e-3) / 1e12
+        value = aggregate_value(flops_step, args.steps, world, total_ms)
+        e2e_value = aggregate_value(flops_step, e2e_steps, world, e2e_ms)
         peaks = measured_peaks()
         # dominant kernel: the dequant-GEMM of the forward or backward-input call, whichever takes longer
         dom = 0 if call_ms[0] >= call_ms[1] else 1
