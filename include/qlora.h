@@ -20,6 +20,11 @@
  * Words are to be read as unsigned.  Zero-points are fp16 values holding integers in [0, 2^bits - 1].
  * Groups are contiguous along K: group(k) = k / group_size.
  *
+ * Stacked adapters (Appendix D: a frozen error-correcting pair A2 [r2, K], B2 [N, r2] with scale s2 that stays with the
+ * quantized weight, plus a newly injected trainable pair): pass ONE adapter of rank r + r2 whose A is the two A stacked
+ * row-wise and whose B is [B | (s2 / s) B2] column-wise, with alpha = s (r + r2).  Y and dX are then those of the stacked
+ * layer, and rows 0 .. r-1 of dA / columns 0 .. r-1 of dB are the trainable pair's gradients (the rest is ignored).
+ *
  * General rules for every entry point below.
  *   - All tensor pointers are DEVICE pointers owned by the caller, dense row-major, 16-byte aligned.  The
  *     descriptor is a HOST pointer.  The library allocates no device memory, keeps no per-call state and never

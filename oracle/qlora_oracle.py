@@ -178,6 +178,32 @@ def backward(X, dY, W, A, B, alpha: float):
     return dX, dA, dB, G
 
 
+# ----------------------------------------------------------------------------------------------
+# Stacked adapters (Appendix D, "LREC Augmented EMEF"): a frozen error-correcting pair (A2, B2) that
+# stays with the quantized weight, plus a newly injected trainable pair (A, B).  Only the new pair
+# receives gradients.
+# ----------------------------------------------------------------------------------------------
+def forward_stacked(X, W, A, B, alpha, A2, B2, alpha2):
+    """Y = X W^T + s (X A^T) B^T + s2 (X A2^T) B2^T,  s = alpha / r,  s2 = alpha2 / r2.  float64."""
+    X = np.asarray(X, dtype=np.float64)
+    A2 = np.asarray(A2, dtype=np.float64)
+    B2 = np.asarray(B2, dtype=np.float64)
+    Y, H = forward(X, W, A, B, alpha)
+    s2 = lora_scale(alpha2, A2.shape[0])
+    return Y + s2 * ((X @ A2.T) @ B2.T), H
+
+
+def backward_stacked(X, dY, W, A, B, alpha, A2, B2, alpha2):
+    """dX = dY W + s (dY B) A + s2 (dY B2) A2;  dA, dB of the trainable pair as in `backward`
+    (the frozen pair appears in neither of them: Y is linear in each pair separately)."""
+    dY = np.asarray(dY, dtype=np.float64)
+    A2 = np.asarray(A2, dtype=np.float64)
+    B2 = np.asarray(B2, dtype=np.float64)
+    dX, dA, dB, G = backward(X, dY, W, A, B, alpha)
+    s2 = lora_scale(alpha2, A2.shape[0])
+    return dX + s2 * ((dY @ B2) @ A2), dA, dB, G
+
+
 def layer_reference(inputs: dict, rows=None) -> dict:
     """Convenience wrapper for the tests: takes the dict produced by the synthetic-input module
     (bf16 bit patterns for X, dY, A, B; uint8 codes; fp16 scales / zeros) and returns the oracle's

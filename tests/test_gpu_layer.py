@@ -120,6 +120,28 @@ def test_group_equals_k_and_small_group():
     check_layer(qi.random_codes_layer(K=512, N=128, bits=8, group_size=32, r=8, alpha=16.0, M=33, seed=2))
 
 
+def test_stacked_adapters_through_rank_concatenation():
+    """A frozen error-correcting pair (r2 = 32) plus a trainable pair (r = 8) on one quantized layer: run as ONE adapter of
+    rank 40 (A rows stacked, the frozen up-projection rescaled by s2 / s, a power of two here, so exact in bf16) and
+    checked against the oracle's stacked definition; the trainable pair's gradients are the first 8 rows / columns."""
+    K, N, M, r, r2, alpha, alpha2 = 512, 384, 300, 8, 32, 16.0, 16.0
+    base = qi.random_codes_layer(K=K, N=N, bits=4, group_size=128, r=r, alpha=alpha, M=M, seed=77)
+    A2 = qi.uniform_bf16(78, 1, (r2, K), 1.0 / np.sqrt(K))
+    B2 = qi.normal_bf16(78, 2, (N, r2), 0.01)
+    s, s2 = alpha / r, alpha2 / r2                                       # 2 and 0.5
+    B2_scaled = qi.f32_to_bf16_bits(qi.bf16_bits_to_f32(B2) * np.float32(s2 / s))
+    assert np.array_equal(qi.bf16_bits_to_f32(B2_scaled), qi.bf16_bits_to_f32(B2) * np.float32(0.25))   # exact
+    cat = dict(base, r=r + r2, alpha=s * (r + r2), A=np.vstack([base["A"], A2]), B=np.hstack([base["B"], B2_scaled]))
+    out = GpuLayer(cat).run()
+    f64 = orc.bf16_bits_to_f64
+    W = orc.dequant(orc.pack(base["codes"], 4), base["scales"], base["zeros"], 4, 128)
+    X, dY = f64(base["X"]), f64(base["dY"])
+    Y, _ = orc.forward_stacked(X, W, f64(base["A"]), f64(base["B"]), alpha, f64(A2), f64(B2), alpha2)
+    dX, dA, dB, _ = orc.backward_stacked(X, dY, W, f64(base["A"]), f64(base["B"]), alpha, f64(A2), f64(B2), alpha2)
+    assert rel_err(to_f64(out["Y"]), Y) <= REL_TOL and rel_err(to_f64(out["dX"]), dX) <= REL_TOL
+    assert rel_err(to_f64(out["dA"])[:r], dA) <= REL_TOL and rel_err(to_f64(out["dB"])[:, :r], dB) <= REL_TOL
+
+
 def test_recompute_h_g_matches_saved():
     layer = qi.random_codes_layer(K=512, N=256, bits=4, group_size=128, r=8, alpha=16.0, M=200, seed=3)
     _, saved, gl = check_layer(layer, save_hg=True)

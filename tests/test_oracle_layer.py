@@ -208,3 +208,49 @@ def test_layer_reference_row_sampling_matches_full():
     assert np.allclose(part["dX"], full["dX"][rows], atol=1e-12)
     assert np.allclose(part["dA"], full["dA"], atol=1e-12) and np.allclose(part["dB"], full["dB"], atol=1e-12)
     assert rel_err(full["Y"], full["Y"]) == 0.0
+
+
+def test_stacked_adapters_gradients_and_reductions():
+    """Frozen pair + trainable pair (Appendix D): central differences for dX, dA, dB of the trainable pair; B2 = 0 gives
+    the single-pair layer; and the identity the CUDA library relies on -- one adapter of rank r + r2 made of the
+    concatenated pairs (the frozen up-projection rescaled by s2 / s) is the same function, with the trainable pair's
+    gradients in its first r rows / columns."""
+    codes, scales, zeros, X, dY, A, B = tiny(41, M=4, K=32, N=8, r=4)
+    rng = np.random.default_rng(42)
+    A2 = rng.standard_normal((8, 32)) * 0.3
+    B2 = rng.standard_normal((8, 8)) * 0.3
+    alpha, alpha2 = 6.0, 4.0
+    W = orc.dequant(orc.pack(codes, 4), scales, zeros, 4, 32)
+    Y, _ = orc.forward_stacked(X, W, A, B, alpha, A2, B2, alpha2)
+    dX, dA, dB, _ = orc.backward_stacked(X, dY, W, A, B, alpha, A2, B2, alpha2)
+
+    def loss(X_, A_, B_):
+        return float(np.sum(dY * orc.forward_stacked(X_, W, A_, B_, alpha, A2, B2, alpha2)[0]))
+
+    eps = 1e-4
+    for arr, grad in ((X, dX), (A, dA), (B, dB)):
+        num = np.zeros_like(arr)
+        for idx in np.ndindex(*arr.shape):
+            up, dn = arr.copy(), arr.copy()
+            up[idx] += eps
+            dn[idx] -= eps
+            args = [X, A, B]
+            pos = [i for i, a in enumerate(args) if a is arr][0]
+            au, ad = list(args), list(args)
+            au[pos], ad[pos] = up, dn
+            num[idx] = (loss(*au) - loss(*ad)) / (2 * eps)
+        assert rel_err(grad, num) < 1e-6
+    # B2 = 0: the plain layer
+    Y0, _ = orc.forward_stacked(X, W, A, B, alpha, A2, np.zeros_like(B2), alpha2)
+    assert np.allclose(Y0, orc.forward(X, W, A, B, alpha)[0], rtol=0, atol=1e-12)
+    # the frozen pair's term, written out
+    s2 = alpha2 / 8
+    assert np.allclose(Y - orc.forward(X, W, A, B, alpha)[0], s2 * (X @ A2.T) @ B2.T, rtol=1e-12, atol=1e-12)
+    # concatenation identity
+    s = alpha / 4
+    A_cat, B_cat = np.vstack([A, A2]), np.hstack([B, B2 * (s2 / s)])
+    alpha_cat = s * 12
+    Yc, _ = orc.forward(X, W, A_cat, B_cat, alpha_cat)
+    dXc, dAc, dBc, _ = orc.backward(X, dY, W, A_cat, B_cat, alpha_cat)
+    assert np.allclose(Yc, Y, rtol=1e-12, atol=1e-12) and np.allclose(dXc, dX, rtol=1e-12, atol=1e-12)
+    assert np.allclose(dAc[:4], dA, rtol=1e-12, atol=1e-12) and np.allclose(dBc[:, :4], dB, rtol=1e-12, atol=1e-12)
