@@ -97,6 +97,26 @@ int qlora_bwd_lora(const qlora_desc* desc, int M, const void* X, const void* dY,
                    const float* H, const float* G, float* dA, float* dB, int accumulate, void* workspace,
                    size_t workspace_bytes, void* cuda_stream);
 
+/* LoRA dropout (Appendix B: dropout 0.05 on the LoRA branch).  The branch sees D(X) = keep_scale * mask (.) X instead of X,
+ * the frozen weight still sees X:
+ *   Y  = X W^T + s (D(X) A^T) B^T                     H_out = D(X) A^T
+ *   dX = dY W + keep_scale * mask (.) (s (dY B) A)    G_out = dY B
+ *   dA = s (dY B)^T D(X)                              dB = s dY^T (D(X) A^T)
+ * mask: uint8 [M, K] device pointer, non-zero = keep (the random draw is the caller's: it is an input, so that a test can
+ * hand the same mask to an independent implementation); keep_scale = 1 / (1 - p) >= 1.  Pass the same mask to all three
+ * calls of a step.  H passed to qlora_bwd_lora_dropout must come from qlora_fwd_dropout with that mask (or be NULL: it
+ * is then recomputed with the mask).  The backward-input call runs the dense kernel without the branch and adds the masked
+ * LoRA term in a second, elementwise pass over dX.  Everything else is as for the calls without dropout. */
+int qlora_fwd_dropout(const qlora_desc* desc, int M, const void* X, const uint8_t* mask, float keep_scale, const int32_t* Q,
+                      const void* scales, const void* zeros, const void* A, const void* B, void* Y, float* H_out,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+int qlora_bwd_input_dropout(const qlora_desc* desc, int M, const void* dY, const uint8_t* mask, float keep_scale,
+                            const int32_t* Q, const void* scales, const void* zeros, const void* A, const void* B, void* dX,
+                            float* G_out, void* workspace, size_t workspace_bytes, void* cuda_stream);
+int qlora_bwd_lora_dropout(const qlora_desc* desc, int M, const void* X, const uint8_t* mask, float keep_scale, const void* dY,
+                           const void* A, const void* B, const float* H, const float* G, float* dA, float* dB, int accumulate,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Size of the scratch array built into the library for qlora_bwd_lora_static (16 MiB, held by every GPU that loads
  * the library until the process exits). */
 #define QLORA_STATIC_SCRATCH_BYTES (16u << 20)

@@ -204,6 +204,39 @@ def backward_stacked(X, dY, W, A, B, alpha, A2, B2, alpha2):
     return dX + s2 * ((dY @ B2) @ A2), dA, dB, G
 
 
+# ----------------------------------------------------------------------------------------------
+# LoRA dropout (Appendix B: dropout 0.05 on the LoRA branch).  The mask is an input (the draw is
+# not part of the layer's arithmetic): D(X) = mask * X / (1 - p).
+# ----------------------------------------------------------------------------------------------
+def forward_dropout(X, W, A, B, alpha, mask, p):
+    """Y = X W^T + s (D(X) A^T) B^T.  Returns (Y, H) with H = D(X) A^T.  float64."""
+    X = np.asarray(X, dtype=np.float64)
+    W = np.asarray(W, dtype=np.float64)
+    A = np.asarray(A, dtype=np.float64)
+    B = np.asarray(B, dtype=np.float64)
+    Xd = X * (np.asarray(mask) != 0) / (1.0 - p)
+    H = Xd @ A.T
+    s = lora_scale(alpha, A.shape[0])
+    return X @ W.T + s * (H @ B.T), H
+
+
+def backward_dropout(X, dY, W, A, B, alpha, mask, p):
+    """dX = dY W + D'(s (dY B) A) with D'(Z) = mask * Z / (1 - p);  dA = s (dY B)^T D(X);  dB = s dY^T (D(X) A^T)."""
+    X = np.asarray(X, dtype=np.float64)
+    dY = np.asarray(dY, dtype=np.float64)
+    W = np.asarray(W, dtype=np.float64)
+    A = np.asarray(A, dtype=np.float64)
+    B = np.asarray(B, dtype=np.float64)
+    keep = (np.asarray(mask) != 0) / (1.0 - p)
+    Xd = X * keep
+    s = lora_scale(alpha, A.shape[0])
+    G = dY @ B
+    dX = dY @ W + keep * (s * (G @ A))
+    dA = s * (G.T @ Xd)
+    dB = s * (dY.T @ (Xd @ A.T))
+    return dX, dA, dB, G
+
+
 def layer_reference(inputs: dict, rows=None) -> dict:
     """Convenience wrapper for the tests: takes the dict produced by the synthetic-input module
     (bf16 bit patterns for X, dY, A, B; uint8 codes; fp16 scales / zeros) and returns the oracle's

@@ -47,12 +47,17 @@ def library() -> ctypes.CDLL:
     lib.qlora_fwd.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.qlora_bwd_input.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.qlora_bwd_lora.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
+    f32 = ctypes.c_float
+    lib.qlora_fwd_dropout.argtypes = [dp, i32, vp, vp, f32, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.qlora_bwd_input_dropout.argtypes = [dp, i32, vp, vp, f32, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.qlora_bwd_lora_dropout.argtypes = [dp, i32, vp, vp, f32, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
     lib.qlora_bwd_lora_static.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp]
     lib.qlora_pack.argtypes = [i32, i32, i32, vp, vp, vp]
     lib.qlora_unpack.argtypes = [i32, i32, i32, vp, vp, vp]
     lib.qlora_dequant.argtypes = [dp, vp, vp, vp, vp, vp]
     lib.qlora_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint), i32]
-    for name in ("qlora_workspace_bytes", "qlora_fwd", "qlora_bwd_input", "qlora_bwd_lora", "qlora_bwd_lora_static", "qlora_pack",
+    for name in ("qlora_workspace_bytes", "qlora_fwd", "qlora_bwd_input", "qlora_bwd_lora", "qlora_bwd_lora_static", "qlora_fwd_dropout", "qlora_bwd_input_dropout",
+                 "qlora_bwd_lora_dropout", "qlora_pack",
                  "qlora_unpack", "qlora_dequant", "qlora_device_status"):
         getattr(lib, name).restype = i32
     _lib = lib
@@ -116,6 +121,29 @@ def qlora_bwd_lora(d, M, X, dY, A, B, H, G, dA, dB, accumulate, workspace, strea
     _check(library().qlora_bwd_lora(ctypes.byref(d), int(M), _ptr(X), _ptr(dY), _ptr(A), _ptr(B), _ptr(H), _ptr(G),
                                     _ptr(dA), _ptr(dB), int(accumulate), _ptr(workspace), wb, _stream(stream)),
            "qlora_bwd_lora")
+
+
+def qlora_fwd_dropout(d, M, X, mask, keep_scale, Q, scales, zeros, A, B, Y, H_out, workspace, stream=None, workspace_bytes=None):
+    wb = _nbytes(workspace) if workspace_bytes is None else int(workspace_bytes)
+    _check(library().qlora_fwd_dropout(ctypes.byref(d), int(M), _ptr(X), _ptr(mask), float(keep_scale), _ptr(Q), _ptr(scales),
+                                       _ptr(zeros), _ptr(A), _ptr(B), _ptr(Y), _ptr(H_out), _ptr(workspace), wb, _stream(stream)),
+           "qlora_fwd_dropout")
+
+
+def qlora_bwd_input_dropout(d, M, dY, mask, keep_scale, Q, scales, zeros, A, B, dX, G_out, workspace, stream=None,
+                            workspace_bytes=None):
+    wb = _nbytes(workspace) if workspace_bytes is None else int(workspace_bytes)
+    _check(library().qlora_bwd_input_dropout(ctypes.byref(d), int(M), _ptr(dY), _ptr(mask), float(keep_scale), _ptr(Q), _ptr(scales),
+                                             _ptr(zeros), _ptr(A), _ptr(B), _ptr(dX), _ptr(G_out), _ptr(workspace), wb,
+                                             _stream(stream)), "qlora_bwd_input_dropout")
+
+
+def qlora_bwd_lora_dropout(d, M, X, mask, keep_scale, dY, A, B, H, G, dA, dB, accumulate, workspace, stream=None,
+                           workspace_bytes=None):
+    wb = _nbytes(workspace) if workspace_bytes is None else int(workspace_bytes)
+    _check(library().qlora_bwd_lora_dropout(ctypes.byref(d), int(M), _ptr(X), _ptr(mask), float(keep_scale), _ptr(dY), _ptr(A),
+                                            _ptr(B), _ptr(H), _ptr(G), _ptr(dA), _ptr(dB), int(accumulate), _ptr(workspace), wb,
+                                            _stream(stream)), "qlora_bwd_lora_dropout")
 
 
 STATIC_SCRATCH_BYTES = 16 << 20   # QLORA_STATIC_SCRATCH_BYTES

@@ -111,9 +111,10 @@ int qlora_dequant(const qlora_desc* desc, const int32_t* Q, const void* scales, 
     return launch_dequant(*desc, Q, scales, zeros, W, (cudaStream_t)cuda_stream);
 }
 
-int qlora_fwd(const qlora_desc* desc, int M, const void* X, const int32_t* Q, const void* scales, const void* zeros,
-              const void* A, const void* B, void* Y, float* H_out, void* workspace, size_t workspace_bytes,
-              void* cuda_stream) {
+// mask == NULL: the plain layer.  Otherwise LoRA dropout: the branch sees keep_scale * mask (.) X.
+static int fwd_common(const qlora_desc* desc, int M, const void* X, const uint8_t* mask, float keep_scale, const int32_t* Q,
+                      const void* scales, const void* zeros, const void* A, const void* B, void* Y, float* H_out,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream) {
     int rc = check_desc(desc, true);
     if (rc != QLORA_OK) return rc;
     if (M < 0) return QLORA_ERR_INVALID_ARG;
@@ -129,24 +130,26 @@ int qlora_fwd(const qlora_desc* desc, int M, const void* X, const int32_t* Q, co
     cudaStream_t st = (cudaStream_t)cuda_stream;
     float* H = H_out ? H_out : reinterpret_cast<float*>(static_cast<char*>(workspace) + w.p0_off);
     if (skinny_supported(d, M)) {
-        const bool fused = d.r > 0 && d.r <= 16;      // the down-projection rides along inside the kernel
+        const bool fused = d.r > 0 && d.r <= 16 && mask == nullptr;   // the down-projection rides along inside the kernel
         if (d.r > 0 && !fused) {
-            rc = launch_lora_down(M, d.K, d.r, true, X, A, H, st);
+            rc = launch_lora_down(M, d.K, d.r, true, X, A, H, st, mask, keep_scale);
             if (rc != QLORA_OK) return rc;
         }
         return launch_skinny_gemm(d, M, false, X, Q, scales, zeros, A, B, H, !fused, Y, st);
     }
     if (d.r > 0) {
-        rc = launch_lora_down(M, d.K, d.r, true, X, A, H, st);
+        rc = launch_lora_down(M, d.K, d.r, true, X, A, H, st, mask, keep_scale);
         if (rc != QLORA_OK) return rc;
     }
     if (umma_supported(d, M)) return launch_umma_gemm(d, M, false, X, Q, scales, zeros, B, H, Y, st);
     return launch_simt_gemm(d, M, false, X, Q, scales, zeros, B, H, Y, st);
 }
 
-int qlora_bwd_input(const qlora_desc* desc, int M, const void* dY, const int32_t* Q, const void* scales,
-                    const void* zeros, const void* A, const void* B, void* dX, float* G_out, void* workspace,
-                    size_t workspace_bytes, void* cuda_stream) {
+// mask == NULL: the plain layer.  Otherwise LoRA dropout: the LoRA term of dX is keep_scale * mask (.) (s G A); the dense
+// kernels then run without the branch (rank 0) and an elementwise pass adds the masked term.
+static int bwd_input_common(const qlora_desc* desc, int M, const void* dY, const uint8_t* mask, float keep_scale,
+                            const int32_t* Q, const void* scales, const void* zeros, const void* A, const void* B, void* dX,
+                            float* G_out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
     int rc = check_desc(desc, true);
     if (rc != QLORA_OK) return rc;
     if (M < 0) return QLORA_ERR_INVALID_ARG;
@@ -161,6 +164,17 @@ int qlora_bwd_input(const qlora_desc* desc, int M, const void* dY, const int32_t
     if (workspace == nullptr || workspace_bytes < w.total) return QLORA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     float* G = G_out ? G_out : reinterpret_cast<float*>(static_cast<char*>(workspace) + w.p0_off);
+    if (mask != nullptr && d.r > 0) {
+        rc = launch_lora_down(M, d.N, d.r, false, dY, B, G, st);
+        if (rc != QLORA_OK) return rc;
+        qlora_desc d0 = d;
+        d0.r = 0;
+        if (skinny_supported(d0, M)) rc = launch_skinny_gemm(d0, M, true, dY, Q, scales, zeros, B, A, G, true, dX, st);
+        else if (umma_supported(d0, M)) rc = launch_umma_gemm(d0, M, true, dY, Q, scales, zeros, A, G, dX, st);
+        else rc = launch_simt_gemm(d0, M, true, dY, Q, scales, zeros, A, G, dX, st);
+        if (rc != QLORA_OK) return rc;
+        return launch_lora_masked_update(M, d.K, d.r, keep_scale * d.alpha / (float)d.r, G, A, mask, dX, st);
+    }
     if (skinny_supported(d, M)) {
         const bool fused = d.r > 0 && d.r <= 16;
         if (d.r > 0 && !fused) {
@@ -177,9 +191,10 @@ int qlora_bwd_input(const qlora_desc* desc, int M, const void* dY, const int32_t
     return launch_simt_gemm(d, M, true, dY, Q, scales, zeros, A, G, dX, st);
 }
 
-int qlora_bwd_lora(const qlora_desc* desc, int M, const void* X, const void* dY, const void* A, const void* B,
-                   const float* H, const float* G, float* dA, float* dB, int accumulate, void* workspace,
-                   size_t workspace_bytes, void* cuda_stream) {
+// mask == NULL: the plain layer.  Otherwise LoRA dropout: H (if recomputed) and dA use keep_scale * mask (.) X.
+static int bwd_lora_common(const qlora_desc* desc, int M, const void* X, const uint8_t* mask, float keep_scale, const void* dY,
+                           const void* A, const void* B, const float* H, const float* G, float* dA, float* dB, int accumulate,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
     int rc = check_desc(desc, true);
     if (rc != QLORA_OK) return rc;
     if (M < 0 || (accumulate != 0 && accumulate != 1)) return QLORA_ERR_INVALID_ARG;
@@ -198,7 +213,7 @@ int qlora_bwd_lora(const qlora_desc* desc, int M, const void* X, const void* dY,
     const float s = d.alpha / (float)d.r;
     if (M > 0 && !H) {
         float* Hs = reinterpret_cast<float*>(ws + w.p0_off);
-        rc = launch_lora_down(M, d.K, d.r, true, X, A, Hs, st);
+        rc = launch_lora_down(M, d.K, d.r, true, X, A, Hs, st, mask, keep_scale);
         if (rc != QLORA_OK) return rc;
         H = Hs;
     }
@@ -208,7 +223,56 @@ int qlora_bwd_lora(const qlora_desc* desc, int M, const void* X, const void* dY,
         if (rc != QLORA_OK) return rc;
         G = Gs;
     }
-    return launch_lora_grads(M, d.K, d.N, d.r, s, X, dY, H, G, dA, dB, accumulate, ws + w.grad_off, st);
+    return launch_lora_grads(M, d.K, d.N, d.r, s, X, dY, H, G, dA, dB, accumulate, ws + w.grad_off, st, mask, keep_scale);
+}
+
+static int check_dropout(const void* mask, float keep_scale, int M) {
+    if (M > 0 && mask == nullptr) return QLORA_ERR_INVALID_ARG;
+    if (!(keep_scale >= 1.0f) || !(keep_scale < 1e6f)) return QLORA_ERR_INVALID_ARG;   // 1 / (1 - p), p in [0, 1)
+    if (!aligned16(mask)) return QLORA_ERR_ALIGNMENT;
+    return QLORA_OK;
+}
+
+int qlora_fwd(const qlora_desc* desc, int M, const void* X, const int32_t* Q, const void* scales, const void* zeros,
+              const void* A, const void* B, void* Y, float* H_out, void* workspace, size_t workspace_bytes,
+              void* cuda_stream) {
+    return fwd_common(desc, M, X, nullptr, 1.0f, Q, scales, zeros, A, B, Y, H_out, workspace, workspace_bytes, cuda_stream);
+}
+
+int qlora_bwd_input(const qlora_desc* desc, int M, const void* dY, const int32_t* Q, const void* scales,
+                    const void* zeros, const void* A, const void* B, void* dX, float* G_out, void* workspace,
+                    size_t workspace_bytes, void* cuda_stream) {
+    return bwd_input_common(desc, M, dY, nullptr, 1.0f, Q, scales, zeros, A, B, dX, G_out, workspace, workspace_bytes, cuda_stream);
+}
+
+int qlora_bwd_lora(const qlora_desc* desc, int M, const void* X, const void* dY, const void* A, const void* B,
+                   const float* H, const float* G, float* dA, float* dB, int accumulate, void* workspace,
+                   size_t workspace_bytes, void* cuda_stream) {
+    return bwd_lora_common(desc, M, X, nullptr, 1.0f, dY, A, B, H, G, dA, dB, accumulate, workspace, workspace_bytes, cuda_stream);
+}
+
+int qlora_fwd_dropout(const qlora_desc* desc, int M, const void* X, const uint8_t* mask, float keep_scale, const int32_t* Q,
+                      const void* scales, const void* zeros, const void* A, const void* B, void* Y, float* H_out,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    const int rc = check_dropout(mask, keep_scale, M);
+    if (rc != QLORA_OK) return rc;
+    return fwd_common(desc, M, X, mask, keep_scale, Q, scales, zeros, A, B, Y, H_out, workspace, workspace_bytes, cuda_stream);
+}
+
+int qlora_bwd_input_dropout(const qlora_desc* desc, int M, const void* dY, const uint8_t* mask, float keep_scale,
+                            const int32_t* Q, const void* scales, const void* zeros, const void* A, const void* B, void* dX,
+                            float* G_out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    const int rc = check_dropout(mask, keep_scale, M);
+    if (rc != QLORA_OK) return rc;
+    return bwd_input_common(desc, M, dY, mask, keep_scale, Q, scales, zeros, A, B, dX, G_out, workspace, workspace_bytes, cuda_stream);
+}
+
+int qlora_bwd_lora_dropout(const qlora_desc* desc, int M, const void* X, const uint8_t* mask, float keep_scale, const void* dY,
+                           const void* A, const void* B, const float* H, const float* G, float* dA, float* dB, int accumulate,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    const int rc = check_dropout(mask, keep_scale, M);
+    if (rc != QLORA_OK) return rc;
+    return bwd_lora_common(desc, M, X, mask, keep_scale, dY, A, B, H, G, dA, dB, accumulate, workspace, workspace_bytes, cuda_stream);
 }
 
 }  // extern "C"

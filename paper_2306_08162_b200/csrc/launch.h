@@ -21,12 +21,18 @@ int launch_simt_gemm(const qlora_desc& d, int M, bool transposed, const void* In
                      const void* scales, const void* zeros, const void* L, const float* P, void* Out,
                      cudaStream_t st);
 // P[m, j] = sum_t In[m, t] * L(j, t);  l_is_A: L = A [r, K] (t = k) else L = B [N, r] (t = n).
-int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const void* L, float* P, cudaStream_t st);
+// mask (optional, only with l_is_A): uint8 [M, T] dropout mask on In, non-zero = keep; the result is multiplied by out_scale.
+int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const void* L, float* P, cudaStream_t st,
+                     const uint8_t* mask = nullptr, float out_scale = 1.0f);
 // dB = s dY^T H [N, r] and dA = s G^T X [r, K] in one pair of launches (partial sums per row slice, then a fixed-order
 // reduction); scratch needs lora_grad_scratch_bytes().
 size_t lora_grad_scratch_bytes(int M, int K, int N, int r);
 int launch_lora_grads(int M, int K, int N, int r, float s, const void* X, const void* dY, const float* H, const float* G,
-                      float* dA, float* dB, int accumulate, void* scratch, cudaStream_t st);
+                      float* dA, float* dB, int accumulate, void* scratch, cudaStream_t st, const uint8_t* x_mask = nullptr,
+                      float keep_scale = 1.0f);
+// dX[m, k] += mask[m, k] * c * sum_j G[m, j] A[j, k]: the LoRA term of the backward pass under dropout.
+int launch_lora_masked_update(int M, int K, int r, float c, const float* G, const void* A, const uint8_t* mask, void* dX,
+                              cudaStream_t st);
 
 // umma_kernel.cu -- tcgen05 tensor-core kernel (both directions); same contract as launch_simt_gemm
 bool umma_supported(const qlora_desc& d, int M);

@@ -130,6 +130,14 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 // Transpose an 8 x 8 matrix of 16-bit elements held across the warp (lane l: row l / 4, elements 2 (l % 4), +1).
+// LoRA dropout: keep the bf16 pair elements whose mask byte is non-zero (mask bytes m0, m1 in the low two bytes of `mb`).
+__device__ __forceinline__ uint32_t mask_pair(uint32_t pair, uint32_t mb) {
+    return pair & (((mb & 0xFFu) ? 0x0000FFFFu : 0u) | ((mb & 0xFF00u) ? 0xFFFF0000u : 0u));
+}
+// Eight bf16 (uint4) against eight mask bytes (uint2).
+__device__ __forceinline__ uint4 mask_eight(uint4 x, uint2 m) {
+    return make_uint4(mask_pair(x.x, m.x), mask_pair(x.y, m.x >> 16), mask_pair(x.z, m.y), mask_pair(x.w, m.y >> 16));
+}
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
     uint32_t d;
     asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
@@ -139,7 +147,7 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
 template <bool L_IS_A, int NT, int WARPS>
 __global__ void __launch_bounds__(WARPS * 32)
 lora_down_kernel(int M, int T, int r, const __nv_bfloat16* __restrict__ In, const __nv_bfloat16* __restrict__ L,
-                 float* __restrict__ P) {
+                 float* __restrict__ P, const uint8_t* __restrict__ mask, float out_scale) {
     __shared__ float red[WARPS][NT][4][32];
     pdl_launch_dependents();
     pdl_wait();
@@ -161,6 +169,10 @@ lora_down_kernel(int M, int T, int r, const __nv_bfloat16* __restrict__ In, cons
             const int k = kk + u * WARPS * 32 + q * 8;         // T is a multiple of 8: 8 elements are all-in or all-out
             xlo[u] = (v0 && k < T) ? *reinterpret_cast<const uint4*>(row0 + k) : zero4;
             xhi[u] = (v1 && k < T) ? *reinterpret_cast<const uint4*>(row1 + k) : zero4;
+            if (mask != nullptr) {   // dropout on the branch input: dropped elements contribute nothing
+                if (v0 && k < T) xlo[u] = mask_eight(xlo[u], __ldg(reinterpret_cast<const uint2*>(mask + (size_t)r0 * T + k)));
+                if (v1 && k < T) xhi[u] = mask_eight(xhi[u], __ldg(reinterpret_cast<const uint2*>(mask + (size_t)r1 * T + k)));
+            }
         }
 #pragma unroll
         for (int u = 0; u < LD_UNROLL; ++u) {
@@ -203,11 +215,12 @@ lora_down_kernel(int M, int T, int r, const __nv_bfloat16* __restrict__ In, cons
         for (int w = 0; w < WARPS; ++w) v += red[w][nt][c][ln];
         const int row = m_base + (ln >> 2) + ((c & 2) ? 8 : 0);
         const int col = nt * 8 + (ln & 3) * 2 + (c & 1);
-        if (row < M && col < r) P[(size_t)row * r + col] = v;
+        if (row < M && col < r) P[(size_t)row * r + col] = v * out_scale;
     }
 }
 
-int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const void* L, float* P, cudaStream_t st) {
+int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const void* L, float* P, cudaStream_t st,
+                     const uint8_t* mask, float out_scale) {
     if (M == 0 || r == 0) return QLORA_OK;
     const unsigned grid = (unsigned)((M + 15) / 16);
     const __nv_bfloat16* in = (const __nv_bfloat16*)In;
@@ -216,8 +229,8 @@ int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const voi
     cudaError_t err = cudaSuccess;
 #define QLORA_LD(NTV, W)                                                                              \
     do {                                                                                              \
-        if (l_is_A) err = launch_pdl(lora_down_kernel<true, NTV, W>, dim3(grid), dim3(W * 32), 0, st, 1, M, T, r, in, l, P);   \
-        else        err = launch_pdl(lora_down_kernel<false, NTV, W>, dim3(grid), dim3(W * 32), 0, st, 1, M, T, r, in, l, P);  \
+        if (l_is_A) err = launch_pdl(lora_down_kernel<true, NTV, W>, dim3(grid), dim3(W * 32), 0, st, 1, M, T, r, in, l, P, mask, out_scale);   \
+        else        err = launch_pdl(lora_down_kernel<false, NTV, W>, dim3(grid), dim3(W * 32), 0, st, 1, M, T, r, in, l, P, mask, out_scale);  \
     } while (0)
     if (nt <= 1) QLORA_LD(1, 32);
     else if (nt <= 2) QLORA_LD(2, 32);
@@ -271,6 +284,8 @@ struct GradSide {
     float* partial;            // [slices][C][r]
     float* Out;
     int C;
+    const uint8_t* mask;       // [M, C] dropout mask on In (non-zero = keep), or NULL
+    float scale;               // s (times the dropout keep scale on the masked side)
 };
 
 template <int RT>   // rank tiles of 16
@@ -316,6 +331,10 @@ lora_grad_partial_kernel(int M, int r, int rows_per_slice, GradSide side0, GradS
             const int ma = mm + 16 * u + g, mb = ma + 8;
             x0[u] = (live && ma < m_stop) ? *reinterpret_cast<const uint4*>(src + (size_t)ma * C) : zero4;
             x1[u] = (live && mb < m_stop) ? *reinterpret_cast<const uint4*>(src + (size_t)mb * C) : zero4;
+            if (sd.mask != nullptr) {
+                if (live && ma < m_stop) x0[u] = mask_eight(x0[u], __ldg(reinterpret_cast<const uint2*>(sd.mask + (size_t)ma * C + c0)));
+                if (live && mb < m_stop) x1[u] = mask_eight(x1[u], __ldg(reinterpret_cast<const uint2*>(sd.mask + (size_t)mb * C + c0)));
+            }
         }
 #pragma unroll
         for (int u = 0; u < LG_UNROLL; ++u) {
@@ -352,7 +371,7 @@ lora_grad_partial_kernel(int M, int r, int rows_per_slice, GradSide side0, GradS
             }
 }
 
-__global__ void lora_grad_reduce_kernel(int r, int slices, float s, int accumulate, GradSide dB_side, GradSide dA_side) {
+__global__ void lora_grad_reduce_kernel(int r, int slices, int accumulate, GradSide dB_side, GradSide dA_side) {
     // elements [0, N*r): dB[n, j]; elements [N*r, N*r + K*r): dA (stored [r, K])
     pdl_launch_dependents();
     pdl_wait();
@@ -371,14 +390,14 @@ __global__ void lora_grad_reduce_kernel(int r, int slices, float s, int accumula
         v = (((v + p0) + p1) + p2) + p3;
     }
     for (; sl < slices; ++sl) v += sd.partial[(size_t)sl * step + e];
-    v *= s;
+    v *= sd.scale;
     const int c = (int)(e / r), j = (int)(e % r);
     float* dst = is_dB ? sd.Out + e : sd.Out + (size_t)j * sd.C + c;
     *dst = accumulate ? (*dst + v) : v;
 }
 
 int launch_lora_grads(int M, int K, int N, int r, float s, const void* X, const void* dY, const float* H, const float* G,
-                      float* dA, float* dB, int accumulate, void* scratch, cudaStream_t st) {
+                      float* dA, float* dB, int accumulate, void* scratch, cudaStream_t st, const uint8_t* x_mask, float keep_scale) {
     if (r == 0) return QLORA_OK;
     if (M == 0) {   // empty sums: dA = dB = 0 unless accumulating
         if (!accumulate) {
@@ -390,8 +409,8 @@ int launch_lora_grads(int M, int K, int N, int r, float s, const void* X, const 
     const GradPlan plan = lora_grad_plan(M, K, N);
     float* part_dB = (float*)scratch;
     float* part_dA = part_dB + (size_t)plan.slices * N * r;
-    GradSide sB{(const __nv_bfloat16*)dY, H, part_dB, dB, N};
-    GradSide sA{(const __nv_bfloat16*)X, G, part_dA, dA, K};
+    GradSide sB{(const __nv_bfloat16*)dY, H, part_dB, dB, N, nullptr, s};
+    GradSide sA{(const __nv_bfloat16*)X, G, part_dA, dA, K, x_mask, x_mask ? s * keep_scale : s};
     const int cols = (N > K ? N : K);
     dim3 grid((cols + LG_COLS - 1) / LG_COLS, plan.slices, 2);
     const int rt = (r + 15) / 16;
@@ -416,7 +435,58 @@ int launch_lora_grads(int M, int K, int N, int r, float s, const void* X, const 
 #undef QLORA_LG
     if (err != cudaSuccess) return QLORA_ERR_CUDA;
     const size_t total = (size_t)(N + K) * r;
-    err = launch_pdl(lora_grad_reduce_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st, 1, r, plan.slices, s, accumulate, sB, sA);
+    err = launch_pdl(lora_grad_reduce_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st, 1, r, plan.slices, accumulate, sB, sA);
+    return err == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// LoRA dropout, backward through the branch input: dX[m, k] += mask[m, k] * c * sum_j G[m, j] A[j, k]   (c = s * keep scale).
+// The tensor-core kernels add the LoRA term inside the accumulator, where a per-element mask cannot be applied, so with
+// dropout they run without the branch and this elementwise pass adds the masked term (dX is read and rounded once more).
+// One thread = 8 consecutive k of one token row.
+// ------------------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+lora_masked_update_kernel(int M, int K, int r, float c, const float* __restrict__ G, const __nv_bfloat16* __restrict__ A,
+                          const uint8_t* __restrict__ mask, __nv_bfloat16* __restrict__ dX) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int kchunks = K / 8;
+    if (idx >= (size_t)M * kchunks) return;
+    const int m = (int)(idx / kchunks), k = (int)(idx % kchunks) * 8;
+    const uint2 mb = __ldg(reinterpret_cast<const uint2*>(mask + (size_t)m * K + k));
+    if ((mb.x | mb.y) == 0u) return;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int j = 0; j < r; ++j) {
+        const float gj = __ldg(G + (size_t)m * r + j);
+        const uint4 av = __ldg(reinterpret_cast<const uint4*>(A + (size_t)j * K + k));
+        acc[0] = fmaf(gj, bf16_lo(av.x), acc[0]); acc[1] = fmaf(gj, bf16_hi(av.x), acc[1]);
+        acc[2] = fmaf(gj, bf16_lo(av.y), acc[2]); acc[3] = fmaf(gj, bf16_hi(av.y), acc[3]);
+        acc[4] = fmaf(gj, bf16_lo(av.z), acc[4]); acc[5] = fmaf(gj, bf16_hi(av.z), acc[5]);
+        acc[6] = fmaf(gj, bf16_lo(av.w), acc[6]); acc[7] = fmaf(gj, bf16_hi(av.w), acc[7]);
+    }
+    uint4* px = reinterpret_cast<uint4*>(dX + (size_t)m * K + k);
+    const uint4 xv = *px;
+    const uint32_t xin[4] = {xv.x, xv.y, xv.z, xv.w};
+    const uint32_t mbytes[2] = {mb.x, mb.y};
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t m2 = mbytes[i >> 1] >> (16 * (i & 1));
+        const float lo = bf16_lo(xin[i]) + ((m2 & 0xFFu) ? c * acc[2 * i] : 0.f);
+        const float hi = bf16_hi(xin[i]) + ((m2 & 0xFF00u) ? c * acc[2 * i + 1] : 0.f);
+        const __nv_bfloat162 pr = __floats2bfloat162_rn(lo, hi);
+        o[i] = *reinterpret_cast<const uint32_t*>(&pr);
+    }
+    *px = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+int launch_lora_masked_update(int M, int K, int r, float c, const float* G, const void* A, const uint8_t* mask, void* dX,
+                              cudaStream_t st) {
+    if (M == 0 || K == 0 || r == 0) return QLORA_OK;
+    const size_t total = (size_t)M * (K / 8);
+    const cudaError_t err = launch_pdl(lora_masked_update_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st, 1, M, K, r,
+                                       c, G, (const __nv_bfloat16*)A, mask, (__nv_bfloat16*)dX);
     return err == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
 }
 

@@ -145,7 +145,7 @@ __device__ __forceinline__ void sk_cluster_epilogue(const SkinnyParams& p, uint3
     uint32_t peer[SK_SPLIT];
 #pragma unroll
     for (int rk = 0; rk < SK_SPLIT; ++rk) peer[rk] = map_to_cta(part_addr, (uint32_t)rk);
-    if (NTL > 0) {
+    if constexpr (NTL > 0) {
         for (int e = tid; e < 16 * 8 * NTL; e += SK_THREADS) {
             const int m = e / (8 * NTL), j = e % (8 * NTL);
             float v = 0.f;

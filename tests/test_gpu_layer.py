@@ -142,6 +142,38 @@ def test_stacked_adapters_through_rank_concatenation():
     assert rel_err(to_f64(out["dA"])[:r], dA) <= REL_TOL and rel_err(to_f64(out["dB"])[:, :r], dB) <= REL_TOL
 
 
+@pytest.mark.parametrize("M,K,N,bits,g,r", [(16, 512, 384, 4, 128, 8), (100, 1024, 256, 2, 64, 16), (600, 512, 512, 4, 128, 8),
+                                              (70, 352, 264, 3, 32, 8), (300, 256, 512, 8, 128, 24)])
+def test_lora_dropout_against_the_oracle(M, K, N, bits, g, r):
+    """LoRA dropout (mask passed in, p = 0.25) through every kernel path: streaming (16 tokens), split single-CTA (100),
+    CTA pair (600), CUDA-core fallback (N = 264), rank 24; saved and recomputed H / G."""
+    import paper_2306_08162_b200 as ql
+    layer = qi.random_codes_layer(K=K, N=N, bits=bits, group_size=g, r=r, alpha=2.0 * r, M=M, seed=900 + M)
+    gl = GpuLayer(layer)
+    p = 0.25
+    mask_np = (np.random.default_rng(M).random((M, K)) >= p).astype(np.uint8)
+    mask = torch.from_numpy(mask_np).cuda()
+    keep = 1.0 / (1.0 - p)
+    Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda"); dX = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    H = torch.empty((M, r), dtype=torch.float32, device="cuda"); G = torch.empty_like(H)
+    dA = torch.empty((r, K), dtype=torch.float32, device="cuda"); dB = torch.empty((N, r), dtype=torch.float32, device="cuda")
+    ql.qlora_fwd_dropout(gl.desc, M, gl.X, mask, keep, gl.Q, gl.scales, gl.zeros, gl.A, gl.B, Y, H, gl.ws)
+    ql.qlora_bwd_input_dropout(gl.desc, M, gl.dY, mask, keep, gl.Q, gl.scales, gl.zeros, gl.A, gl.B, dX, G, gl.ws)
+    ql.qlora_bwd_lora_dropout(gl.desc, M, gl.X, mask, keep, gl.dY, gl.A, gl.B, H, G, dA, dB, 0, gl.ws)
+    dA2 = torch.empty_like(dA); dB2 = torch.empty_like(dB)
+    ql.qlora_bwd_lora_dropout(gl.desc, M, gl.X, mask, keep, gl.dY, gl.A, gl.B, None, None, dA2, dB2, 0, gl.ws)
+    torch.cuda.synchronize()
+    assert ql.qlora_device_status() == 0
+    f64 = orc.bf16_bits_to_f64
+    W = orc.dequant(orc.pack(layer["codes"], bits), layer["scales"], layer["zeros"], bits, g)
+    Xr, dYr, Ar, Br = f64(layer["X"]), f64(layer["dY"]), f64(layer["A"]), f64(layer["B"])
+    Yo, Ho = orc.forward_dropout(Xr, W, Ar, Br, layer["alpha"], mask_np, p)
+    dXo, dAo, dBo, Go = orc.backward_dropout(Xr, dYr, W, Ar, Br, layer["alpha"], mask_np, p)
+    for name, got, want in (("Y", Y, Yo), ("H", H, Ho), ("dX", dX, dXo), ("G", G, Go), ("dA", dA, dAo), ("dB", dB, dBo)):
+        assert rel_err(to_f64(got), want) <= REL_TOL, name
+    assert torch.equal(dA, dA2) and torch.equal(dB, dB2)
+
+
 def test_recompute_h_g_matches_saved():
     layer = qi.random_codes_layer(K=512, N=256, bits=4, group_size=128, r=8, alpha=16.0, M=200, seed=3)
     _, saved, gl = check_layer(layer, save_hg=True)

@@ -254,3 +254,43 @@ def test_stacked_adapters_gradients_and_reductions():
     dXc, dAc, dBc, _ = orc.backward(X, dY, W, A_cat, B_cat, alpha_cat)
     assert np.allclose(Yc, Y, rtol=1e-12, atol=1e-12) and np.allclose(dXc, dX, rtol=1e-12, atol=1e-12)
     assert np.allclose(dAc[:4], dA, rtol=1e-12, atol=1e-12) and np.allclose(dBc[:, :4], dB, rtol=1e-12, atol=1e-12)
+
+
+def test_dropout_gradients_and_reductions():
+    """LoRA dropout with the mask as an input (Appendix B): central differences of <dY, Y> for dX, dA, dB with the mask
+    held fixed; an all-ones mask with p = 0 is the plain layer; an all-zero mask removes the branch (dA = 0, dB = 0, Y and
+    dX those of the pure quantized layer); dropped positions of X get no gradient through the branch."""
+    codes, scales, zeros, X, dY, A, B = tiny(51, M=4, K=32, N=8, r=4)
+    rng = np.random.default_rng(52)
+    mask = (rng.random(X.shape) > 0.3).astype(np.uint8)
+    p, alpha = 0.3, 6.0
+    W = orc.dequant(orc.pack(codes, 4), scales, zeros, 4, 32)
+    dX, dA, dB, _ = orc.backward_dropout(X, dY, W, A, B, alpha, mask, p)
+
+    def loss(X_, A_, B_):
+        return float(np.sum(dY * orc.forward_dropout(X_, W, A_, B_, alpha, mask, p)[0]))
+
+    eps = 1e-4
+    for pos, (arr, grad) in enumerate(((X, dX), (A, dA), (B, dB))):
+        num = np.zeros_like(arr)
+        for idx in np.ndindex(*arr.shape):
+            up, dn = arr.copy(), arr.copy()
+            up[idx] += eps
+            dn[idx] -= eps
+            au, ad = [X, A, B], [X, A, B]
+            au[pos], ad[pos] = up, dn
+            num[idx] = (loss(*au) - loss(*ad)) / (2 * eps)
+        assert rel_err(grad, num) < 1e-6
+    ones = np.ones_like(mask)
+    assert np.allclose(orc.forward_dropout(X, W, A, B, alpha, ones, 0.0)[0], orc.forward(X, W, A, B, alpha)[0], rtol=0, atol=1e-12)
+    for got, want in zip(orc.backward_dropout(X, dY, W, A, B, alpha, ones, 0.0), orc.backward(X, dY, W, A, B, alpha)):
+        assert np.allclose(got, want, rtol=0, atol=1e-12)
+    none = np.zeros_like(mask)
+    assert np.allclose(orc.forward_dropout(X, W, A, B, alpha, none, p)[0], X @ W.T, rtol=0, atol=1e-12)
+    dX0, dA0, dB0, _ = orc.backward_dropout(X, dY, W, A, B, alpha, none, p)
+    assert np.allclose(dX0, dY @ W, rtol=0, atol=1e-12) and not dA0.any() and not dB0.any()
+    # where the mask is zero, dX is the frozen weight's term alone
+    assert np.allclose(dX[mask == 0], (dY @ W)[mask == 0], rtol=0, atol=1e-12)
+    # scaling: E-preserving 1 / (1 - p) on kept elements
+    Yk, Hk = orc.forward_dropout(X, W, A, B, alpha, mask, p)
+    assert np.allclose(Hk, ((X * mask) / 0.7) @ A.T, rtol=1e-12, atol=1e-12)
