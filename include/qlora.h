@@ -141,6 +141,16 @@ int qlora_bwd_lora_static(const qlora_desc* desc, int M, const void* X, const vo
 int qlora_pack(int bits, int K, int N, const uint8_t* codes, int32_t* Q, void* cuda_stream);
 int qlora_unpack(int bits, int K, int N, const int32_t* Q, uint8_t* codes, void* cuda_stream);
 
+/* Column gather  out[m, j] = in[m, perm[j]]  for 2-byte (bf16) or 4-byte (fp32) elements; perm: int32 [cols] device
+ * pointer holding a permutation of 0 .. cols-1 (not checked); in and out must not overlap.
+ * This is the per-call step of the activation-order format (Appendix A, "activation order": the group of input feature k
+ * is g_idx[k], not k / group_size).  With perm = a stable sort of the features by g_idx, the packed matrix whose code
+ * rows are permuted once (codes[perm, :] re-packed) has contiguous groups, and
+ *     Y = gather(X, perm) W'^T + s (gather(X, perm) gather(A, perm)^T) B^T
+ * is the activation-order layer's Y; dX and dA come back in the permuted order and are un-permuted with the inverse
+ * permutation (the same call). */
+int qlora_gather_columns(int elem_bytes, int rows, int cols, const void* in, const int32_t* perm, void* out, void* cuda_stream);
+
 /* Full dequantisation to the bf16 weight the tensor-core kernels stage:  W[n,k] = bf16_rne(fp32(scale) * (q - zero)),
  * bf16 [N, K].  The fp32 product is exact (an 11-bit significand times an integer of at most 9 bits), so the result
  * is a single rounding of the closed form.  desc->r and desc->alpha are ignored. */

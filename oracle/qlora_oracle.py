@@ -109,6 +109,18 @@ def dequant(Q: np.ndarray, scales: np.ndarray, zeros: np.ndarray, bits: int, gro
     return np.ascontiguousarray((s_full * (q - z_full)).T)      # [N, K]
 
 
+def dequant_gidx(Q: np.ndarray, scales: np.ndarray, zeros: np.ndarray, bits: int, g_idx: np.ndarray) -> np.ndarray:
+    """Activation-order format (Appendix A): the group of input feature k is g_idx[k] instead of k // g.
+    W[n, k] = scales[g_idx[k], n] * (q[k, n] - zeros[g_idx[k], n]).  float64 [N, K]."""
+    q = unpack(Q, bits).astype(np.float64)                      # [K, N]
+    g_idx = np.asarray(g_idx)
+    if g_idx.shape != (q.shape[0],):
+        raise ValueError("g_idx must have one entry per input feature")
+    s = np.asarray(scales, dtype=np.float16).astype(np.float64)[g_idx]   # [K, N]
+    z = np.asarray(zeros, dtype=np.float16).astype(np.float64)[g_idx]
+    return np.ascontiguousarray((s * (q - z)).T)
+
+
 def round_to_bf16_bits(x: np.ndarray) -> np.ndarray:
     """Round float values (exactly representable in float32) to bf16, nearest-even; returns uint16 bit patterns."""
     f32 = np.asarray(x, dtype=np.float64).astype(np.float32)

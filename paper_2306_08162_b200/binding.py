@@ -55,10 +55,11 @@ def library() -> ctypes.CDLL:
     lib.qlora_pack.argtypes = [i32, i32, i32, vp, vp, vp]
     lib.qlora_unpack.argtypes = [i32, i32, i32, vp, vp, vp]
     lib.qlora_dequant.argtypes = [dp, vp, vp, vp, vp, vp]
+    lib.qlora_gather_columns.argtypes = [i32, i32, i32, vp, vp, vp, vp]
     lib.qlora_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint), i32]
     for name in ("qlora_workspace_bytes", "qlora_fwd", "qlora_bwd_input", "qlora_bwd_lora", "qlora_bwd_lora_static", "qlora_fwd_dropout", "qlora_bwd_input_dropout",
                  "qlora_bwd_lora_dropout", "qlora_pack",
-                 "qlora_unpack", "qlora_dequant", "qlora_device_status"):
+                 "qlora_unpack", "qlora_dequant", "qlora_gather_columns", "qlora_device_status"):
         getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -163,6 +164,13 @@ def qlora_pack(bits, K, N, codes, Q, stream=None):
 
 def qlora_unpack(bits, K, N, Q, codes, stream=None):
     _check(library().qlora_unpack(int(bits), int(K), int(N), _ptr(Q), _ptr(codes), _stream(stream)), "qlora_unpack")
+
+
+def qlora_gather_columns(inp, perm, out, stream=None):
+    """out[m, j] = inp[m, perm[j]] for 2-D bf16 / fp16 / fp32 tensors; perm int32 [cols]."""
+    rows, cols = inp.shape
+    _check(library().qlora_gather_columns(inp.element_size(), int(rows), int(cols), _ptr(inp), _ptr(perm), _ptr(out),
+                                          _stream(stream)), "qlora_gather_columns")
 
 
 def qlora_dequant(d, Q, scales, zeros, W, stream=None):

@@ -101,6 +101,15 @@ int qlora_unpack(int bits, int K, int N, const int32_t* Q, uint8_t* codes, void*
     return launch_unpack(bits, K, N, Q, codes, (cudaStream_t)cuda_stream);
 }
 
+int qlora_gather_columns(int elem_bytes, int rows, int cols, const void* in, const int32_t* perm, void* out, void* cuda_stream) {
+    if (rows < 0 || cols < 0) return QLORA_ERR_INVALID_ARG;
+    if (elem_bytes != 2 && elem_bytes != 4) return QLORA_ERR_UNSUPPORTED;
+    if (rows == 0 || cols == 0) return QLORA_OK;
+    if (!in || !perm || !out || in == out) return QLORA_ERR_INVALID_ARG;
+    if (!aligned16(in) || !aligned16(perm) || !aligned16(out)) return QLORA_ERR_ALIGNMENT;
+    return launch_gather_columns(elem_bytes, rows, cols, in, perm, out, (cudaStream_t)cuda_stream);
+}
+
 int qlora_dequant(const qlora_desc* desc, const int32_t* Q, const void* scales, const void* zeros, void* W,
                   void* cuda_stream) {
     const int rc = check_desc(desc, false);

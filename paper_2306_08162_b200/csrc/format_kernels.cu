@@ -53,6 +53,27 @@ __global__ void dequant_kernel(int g, int K, int N, const uint32_t* __restrict__
     for (int c = 0; c < 4; ++c) dst[c] = make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
 }
 
+// Column gather out[m, j] = in[m, perm[j]] for 2- or 4-byte elements: the per-call step of the activation-order format
+// (Appendix A: GPTQ "activation order" leaves the input features of a group scattered; permuting the packed rows once so
+// that groups become contiguous, and gathering the activation columns with the same permutation, gives the same layer).
+template <typename T>
+__global__ void gather_columns_kernel(int rows, int cols, const T* __restrict__ in, const int32_t* __restrict__ perm, T* __restrict__ out) {
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)rows * cols) return;
+    const int m = (int)(idx / cols), j = (int)(idx % cols);
+    out[idx] = in[(size_t)m * cols + __ldg(perm + j)];
+}
+
+int launch_gather_columns(int elem_bytes, int rows, int cols, const void* in, const int32_t* perm, void* out, cudaStream_t st) {
+    const size_t total = (size_t)rows * cols;
+    if (total == 0) return QLORA_OK;
+    const unsigned grid = (unsigned)((total + 255) / 256);
+    if (elem_bytes == 2) gather_columns_kernel<uint16_t><<<grid, 256, 0, st>>>(rows, cols, (const uint16_t*)in, perm, (uint16_t*)out);
+    else if (elem_bytes == 4) gather_columns_kernel<uint32_t><<<grid, 256, 0, st>>>(rows, cols, (const uint32_t*)in, perm, (uint32_t*)out);
+    else return QLORA_ERR_UNSUPPORTED;
+    return cudaGetLastError() == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
+}
+
 int launch_pack(int bits, int K, int N, const uint8_t* codes, int32_t* Q, cudaStream_t st) {
     const int rows = K * bits / 32;
     const size_t total = (size_t)rows * N;

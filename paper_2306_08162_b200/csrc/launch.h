@@ -11,6 +11,7 @@ namespace qlora {
 // format_kernels.cu
 int launch_pack(int bits, int K, int N, const uint8_t* codes, int32_t* Q, cudaStream_t st);
 int launch_unpack(int bits, int K, int N, const int32_t* Q, uint8_t* codes, cudaStream_t st);
+int launch_gather_columns(int elem_bytes, int rows, int cols, const void* in, const int32_t* perm, void* out, cudaStream_t st);
 int launch_dequant(const qlora_desc& d, const int32_t* Q, const void* scales, const void* zeros, void* W,
                    cudaStream_t st);
 

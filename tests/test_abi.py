@@ -111,6 +111,18 @@ def test_calls_reject_bad_arguments_before_launch(ql):
     with pytest.raises(ql.QloraError) as e:
         ql.qlora_dequant(ql.desc(4, 128, 256, 256, 0, 0.0), ok, ok, None, ok, stream=0)
     assert e.value.status == -1
+    # dropout variants: the mask is required, the keep scale is 1 / (1 - p) >= 1
+    with pytest.raises(ql.QloraError) as e:
+        ql.qlora_fwd_dropout(d, 4, ok, None, 1.25, ok, ok, ok, ok, ok, ok, None, ok, stream=0, workspace_bytes=need)
+    assert e.value.status == -1
+    with pytest.raises(ql.QloraError) as e:
+        ql.qlora_bwd_input_dropout(d, 4, ok, ok, 0.5, ok, ok, ok, ok, ok, ok, None, ok, stream=0, workspace_bytes=need)
+    assert e.value.status == -1
+    # column gather: element size, NULL, in-place
+    lib = ql.library()
+    assert lib.qlora_gather_columns(3, 4, 8, ok, ok, ok + 64, 0) == -2
+    assert lib.qlora_gather_columns(2, 4, 8, ok, None, ok + 64, 0) == -1
+    assert lib.qlora_gather_columns(2, 4, 8, ok, ok, ok, 0) == -1
 
 
 def test_missing_library_fails_loudly(ql, monkeypatch, tmp_path):

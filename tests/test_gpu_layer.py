@@ -174,6 +174,40 @@ def test_lora_dropout_against_the_oracle(M, K, N, bits, g, r):
     assert torch.equal(dA, dA2) and torch.equal(dB, dB2)
 
 
+@pytest.mark.parametrize("M", [20, 400])
+def test_activation_order_through_row_permutation_and_column_gather(M):
+    """GPTQ activation order: group of feature k = g_idx[k], scattered.  The library runs it as a contiguous-group layer:
+    code rows permuted once by a stable sort of g_idx, activation and adapter columns gathered with the same permutation
+    (qlora_gather_columns), dX and dA un-permuted with the inverse.  Checked against the oracle evaluated with g_idx."""
+    import paper_2306_08162_b200 as ql
+    K, N, bits, g, r, alpha = 512, 384, 4, 128, 8, 16.0
+    layer = qi.random_codes_layer(K=K, N=N, bits=bits, group_size=g, r=r, alpha=alpha, M=M, seed=300 + M)
+    rng = np.random.default_rng(M)
+    g_idx = rng.permutation(np.arange(K) // g)
+    perm = np.argsort(g_idx, kind="stable").astype(np.int32)
+    inv = np.argsort(perm).astype(np.int32)
+    f64 = orc.bf16_bits_to_f64
+    W = orc.dequant_gidx(orc.pack(layer["codes"], bits), layer["scales"], layer["zeros"], bits, g_idx)
+    Xr, dYr, Ar, Br = f64(layer["X"]), f64(layer["dY"]), f64(layer["A"]), f64(layer["B"])
+    Yo, _ = orc.forward(Xr, W, Ar, Br, alpha)
+    dXo, dAo, dBo, _ = orc.backward(Xr, dYr, W, Ar, Br, alpha)
+    # device side: permuted layer
+    gl = GpuLayer(dict(layer, codes=np.ascontiguousarray(layer["codes"][perm])))
+    d_perm, d_inv = torch.from_numpy(perm).cuda(), torch.from_numpy(inv).cuda()
+    Xp, Ap = torch.empty_like(gl.X), torch.empty_like(gl.A)
+    ql.qlora_gather_columns(gl.X, d_perm, Xp)
+    ql.qlora_gather_columns(gl.A, d_perm, Ap)
+    gl.A = Ap
+    out = gl.run(X=Xp)
+    dX, dA = torch.empty_like(out["dX"]), torch.empty_like(out["dA"])
+    ql.qlora_gather_columns(out["dX"].contiguous(), d_inv, dX)
+    ql.qlora_gather_columns(out["dA"], d_inv, dA)
+    torch.cuda.synchronize()
+    assert torch.equal(Xp.cpu(), gl.X.cpu()[:, torch.from_numpy(perm.astype(np.int64))])          # the gather itself is exact
+    assert rel_err(to_f64(out["Y"]), Yo) <= REL_TOL and rel_err(to_f64(dX), dXo) <= REL_TOL
+    assert rel_err(to_f64(dA), dAo) <= REL_TOL and rel_err(to_f64(out["dB"]), dBo) <= REL_TOL
+
+
 def test_recompute_h_g_matches_saved():
     layer = qi.random_codes_layer(K=512, N=256, bits=4, group_size=128, r=8, alpha=16.0, M=200, seed=3)
     _, saved, gl = check_layer(layer, save_hg=True)

@@ -141,3 +141,25 @@ def test_dequant_rejects_bad_shapes():
         orc.pack(np.full((32, 1), 16, np.uint8), 4)
     with pytest.raises(ValueError):
         orc.pack(codes[:33], 4)
+
+
+def test_dequant_with_activation_order_index():
+    """g_idx[k] = k // g gives the contiguous-group dequant; a scattered g_idx matches loops written from the index form;
+    and permuting the code rows by a stable sort of g_idx turns it into a contiguous-group matrix with permuted columns
+    (the identity the CUDA library's activation-order recipe rests on)."""
+    rng = np.random.default_rng(9)
+    bits, K, N, g = 3, 96, 8, 32
+    codes = rng.integers(0, 1 << bits, size=(K, N), dtype=np.uint8)
+    scales = rng.uniform(0.01, 0.1, size=(K // g, N)).astype(np.float16)
+    zeros = rng.integers(0, 1 << bits, size=(K // g, N)).astype(np.float16)
+    Q = orc.pack(codes, bits)
+    assert np.array_equal(orc.dequant_gidx(Q, scales, zeros, bits, np.arange(K) // g), orc.dequant(Q, scales, zeros, bits, g))
+    g_idx = rng.permutation(np.arange(K) // g)
+    W = orc.dequant_gidx(Q, scales, zeros, bits, g_idx)
+    for n in range(N):
+        for k in range(K):
+            assert W[n, k] == float(scales[g_idx[k], n]) * (int(codes[k, n]) - float(zeros[g_idx[k], n]))
+    perm = np.argsort(g_idx, kind="stable")
+    assert np.array_equal(g_idx[perm], np.arange(K) // g)
+    Wp = orc.dequant(orc.pack(codes[perm], bits), scales, zeros, bits, g)
+    assert np.array_equal(Wp, W[:, perm])
