@@ -408,6 +408,48 @@ def run_ours(args):
     return 0
 
 
+def run_loss(args):
+    """--workload lrec_loss: the fused KL + cross-entropy loss of the error-correction objective (Section 3.2) and its
+    gradient over T = 4096 tokens (8 x 512) x V = 32000 bf16 logits, an HBM-bound second workload.  Reported in GB/s of
+    algorithmic bytes (two logit matrices read, one gradient written); every call touches 786 MB, far more than the L2."""
+    import torch
+    import paper_2306_08162_b200 as ql
+    import qlora_inputs as qi
+    T, V = 4096, 32000
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    ql.library()
+    z = torch.from_numpy(qi.normal_bf16(7, 0, (T, V), 3.0).view(np.int16)).to(dev).view(torch.bfloat16)
+    t = torch.from_numpy(qi.normal_bf16(7, 1, (T, V), 3.0).view(np.int16)).to(dev).view(torch.bfloat16)
+    labels = torch.from_numpy(np.random.default_rng(7).integers(0, V, size=T).astype(np.int32)).to(dev)
+    loss = torch.empty(T, dtype=torch.float32, device=dev)
+    grad = torch.empty((T, V), dtype=torch.bfloat16, device=dev)
+    for _ in range(args.warmup):
+        ql.qlora_lrec_loss(z, t, labels, 1.0, 1.0, 1.0 / T, loss, grad)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(dev.index or 0)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    e0.record()
+    for _ in range(args.steps):
+        ql.qlora_lrec_loss(z, t, labels, 1.0, 1.0, 1.0 / T, loss, grad)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    alg_bytes = 6.0 * T * V + 8.0 * T
+    peaks = measured_peaks()
+    gbs = alg_bytes / (ms * 1e-3) / 1e9
+    print(json.dumps({"metric": "fused LREC loss fwd+bwd, GB/s of algorithmic bytes", "value": gbs, "unit": "GB/s", "n_gpus": 1,
+                      "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+                      "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                      "config": {"workload": "LREC objective: T=4096 tokens x V=32000 bf16 student + teacher logits -> per-token loss + bf16 gradient"},
+                      "roofline": {"bound": "hbm", "kernel": "lrec_loss_kernel", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s",
+                                   "frac": gbs / peaks["hbm"], "traffic": None, "peak_kind": f"{peaks['source']} HBM copy bandwidth"},
+                      "gpu_launches": args.steps, "clocks": clocks}))
+    return 0
+
+
 def launches_per_step(M: int, r: int) -> int:
     """Kernels the library launches for one fwd + bwd_input + bwd_lora (H, G saved).  Up to 32 tokens the LoRA
     down-projection is fused into the streaming kernel for r <= 16 (one launch per call); otherwise each of fwd and
@@ -424,7 +466,7 @@ def main():
     ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="config2",
+    ap.add_argument("--workload", choices=sorted(WORKLOADS) + ["lrec_loss"], default="config2",
                     help="layer shape to run (default: configs[1], the headline workload)")
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="time the K steps as issued call by call from Python instead of as one CUDA-graph replay "
@@ -434,6 +476,8 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if args.workload == "lrec_loss":
+        return run_loss(args)
     global WORKLOAD, WORKLOAD_NAME, ROTATION
     WORKLOAD, WORKLOAD_NAME = WORKLOADS[args.workload]
     ROTATION = max(4, -(-300 * 2**20 // layer_bytes(WORKLOAD)))     # > 126 MB of L2 with margin

@@ -141,6 +141,19 @@ int qlora_bwd_lora_static(const qlora_desc* desc, int M, const void* X, const vo
 int qlora_pack(int bits, int K, int N, const uint8_t* codes, int32_t* Q, void* cuda_stream);
 int qlora_unpack(int bits, int K, int N, const int32_t* Q, uint8_t* codes, void* cuda_stream);
 
+/* Fused LREC training loss and its gradient (Section 3.2, Eq. 1-2): per token, with p = softmax(student logits) and
+ * q = softmax(teacher logits) over the V vocabulary entries,
+ *     loss_tokens[t] = lambda_kl * sum_i p_i log(p_i / q_i)  +  lambda_ce * ( -log p[labels[t]] )
+ *     dlogits[t, j]  = grad_scale * ( lambda_kl * p_j ((log p_j - log q_j) - KL_t) + lambda_ce * (p_j - [j == labels[t]]) )
+ * (the paper prints the cross-entropy with its arguments exchanged; this is the usual next-token cross-entropy).
+ * student_logits, teacher_logits: bf16 [T, V] (the teacher's are the cached targets of the full-precision model,
+ * Appendix C); labels: int32 [T] or NULL, entries outside [0, V) drop the cross-entropy term of that token;
+ * loss_tokens: fp32 [T] (the mean over the batch is left to the caller: pass grad_scale = 1 / n for the gradient of the
+ * mean); dlogits: bf16 [T, V] or NULL (loss only).  V % 8 == 0 and V <= 32768, else QLORA_ERR_UNSUPPORTED.
+ * fp32 arithmetic, fixed-order reductions (bitwise reproducible).  Each logit matrix is read once. */
+int qlora_lrec_loss(int T, int V, const void* student_logits, const void* teacher_logits, const int32_t* labels, float lambda_kl,
+                    float lambda_ce, float grad_scale, float* loss_tokens, void* dlogits, void* cuda_stream);
+
 /* Column gather  out[m, j] = in[m, perm[j]]  for 2-byte (bf16) or 4-byte (fp32) elements; perm: int32 [cols] device
  * pointer holding a permutation of 0 .. cols-1 (not checked); in and out must not overlap.
  * This is the per-call step of the activation-order format (Appendix A, "activation order": the group of input feature k

@@ -249,6 +249,38 @@ def backward_dropout(X, dY, W, A, B, alpha, mask, p):
     return dX, dA, dB, G
 
 
+# ----------------------------------------------------------------------------------------------
+# LREC objective (Section 3.2, Eq. 1-2): lambda_KL * KL(student || teacher) + lambda_CE * CE(student, label).
+# The paper prints the cross-entropy with its two arguments exchanged (log of a one-hot target);
+# the reading taken is the usual next-token cross-entropy, -log p[label].
+# ----------------------------------------------------------------------------------------------
+def lrec_loss(student_logits, teacher_logits, labels, lambda_kl: float, lambda_ce: float):
+    """Per-token loss [T] and its gradient with respect to the student logits [T, V], float64.
+
+    p = softmax(z), q = softmax(t);  loss_t = lambda_kl * sum_i p_i (log p_i - log q_i) + lambda_ce * (-log p[label_t]).
+    Labels outside [0, V) drop the cross-entropy term of that token."""
+    z = np.asarray(student_logits, dtype=np.float64)
+    t = np.asarray(teacher_logits, dtype=np.float64)
+    T, V = z.shape
+    logp = z - z.max(axis=1, keepdims=True)
+    logp = logp - np.log(np.exp(logp).sum(axis=1, keepdims=True))
+    logq = t - t.max(axis=1, keepdims=True)
+    logq = logq - np.log(np.exp(logq).sum(axis=1, keepdims=True))
+    p = np.exp(logp)
+    kl = (p * (logp - logq)).sum(axis=1)
+    loss = lambda_kl * kl
+    grad = lambda_kl * p * ((logp - logq) - kl[:, None])
+    if labels is not None:
+        labels = np.asarray(labels)
+        for tok in range(T):
+            lab = int(labels[tok])
+            if 0 <= lab < V:
+                loss[tok] += lambda_ce * (-logp[tok, lab])
+                grad[tok] += lambda_ce * p[tok]
+                grad[tok, lab] -= lambda_ce
+    return loss, grad
+
+
 def layer_reference(inputs: dict, rows=None) -> dict:
     """Convenience wrapper for the tests: takes the dict produced by the synthetic-input module
     (bf16 bit patterns for X, dY, A, B; uint8 codes; fp16 scales / zeros) and returns the oracle's

@@ -56,10 +56,11 @@ def library() -> ctypes.CDLL:
     lib.qlora_unpack.argtypes = [i32, i32, i32, vp, vp, vp]
     lib.qlora_dequant.argtypes = [dp, vp, vp, vp, vp, vp]
     lib.qlora_gather_columns.argtypes = [i32, i32, i32, vp, vp, vp, vp]
+    lib.qlora_lrec_loss.argtypes = [i32, i32, vp, vp, vp, ctypes.c_float, ctypes.c_float, ctypes.c_float, vp, vp, vp]
     lib.qlora_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint), i32]
     for name in ("qlora_workspace_bytes", "qlora_fwd", "qlora_bwd_input", "qlora_bwd_lora", "qlora_bwd_lora_static", "qlora_fwd_dropout", "qlora_bwd_input_dropout",
                  "qlora_bwd_lora_dropout", "qlora_pack",
-                 "qlora_unpack", "qlora_dequant", "qlora_gather_columns", "qlora_device_status"):
+                 "qlora_unpack", "qlora_dequant", "qlora_gather_columns", "qlora_lrec_loss", "qlora_device_status"):
         getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -164,6 +165,14 @@ def qlora_pack(bits, K, N, codes, Q, stream=None):
 
 def qlora_unpack(bits, K, N, Q, codes, stream=None):
     _check(library().qlora_unpack(int(bits), int(K), int(N), _ptr(Q), _ptr(codes), _stream(stream)), "qlora_unpack")
+
+
+def qlora_lrec_loss(student_logits, teacher_logits, labels, lambda_kl, lambda_ce, grad_scale, loss_tokens, dlogits, stream=None):
+    """Fused KL + cross-entropy loss of the error-correction objective and its gradient; logits bf16 [T, V]."""
+    T, V = student_logits.shape
+    _check(library().qlora_lrec_loss(int(T), int(V), _ptr(student_logits), _ptr(teacher_logits), _ptr(labels), float(lambda_kl),
+                                     float(lambda_ce), float(grad_scale), _ptr(loss_tokens), _ptr(dlogits), _stream(stream)),
+           "qlora_lrec_loss")
 
 
 def qlora_gather_columns(inp, perm, out, stream=None):

@@ -101,6 +101,20 @@ int qlora_unpack(int bits, int K, int N, const int32_t* Q, uint8_t* codes, void*
     return launch_unpack(bits, K, N, Q, codes, (cudaStream_t)cuda_stream);
 }
 
+int qlora_lrec_loss(int T, int V, const void* student_logits, const void* teacher_logits, const int32_t* labels, float lambda_kl,
+                    float lambda_ce, float grad_scale, float* loss_tokens, void* dlogits, void* cuda_stream) {
+    if (T < 0 || V < 0) return QLORA_ERR_INVALID_ARG;
+    if (V == 0 || V % 8 != 0 || V > 32768) return QLORA_ERR_UNSUPPORTED;
+    if (T == 0) return QLORA_OK;
+    if (!student_logits || !teacher_logits || !loss_tokens) return QLORA_ERR_INVALID_ARG;
+    if (!(lambda_kl == lambda_kl) || !(lambda_ce == lambda_ce) || !(grad_scale == grad_scale)) return QLORA_ERR_INVALID_ARG;
+    if (!aligned16(student_logits) || !aligned16(teacher_logits) || !aligned16(labels) || !aligned16(loss_tokens) ||
+        !aligned16(dlogits))
+        return QLORA_ERR_ALIGNMENT;
+    return launch_lrec_loss(T, V, student_logits, teacher_logits, labels, lambda_kl, lambda_ce, grad_scale, loss_tokens, dlogits,
+                            (cudaStream_t)cuda_stream);
+}
+
 int qlora_gather_columns(int elem_bytes, int rows, int cols, const void* in, const int32_t* perm, void* out, void* cuda_stream) {
     if (rows < 0 || cols < 0) return QLORA_ERR_INVALID_ARG;
     if (elem_bytes != 2 && elem_bytes != 4) return QLORA_ERR_UNSUPPORTED;

@@ -15,6 +15,10 @@ int launch_gather_columns(int elem_bytes, int rows, int cols, const void* in, co
 int launch_dequant(const qlora_desc& d, const int32_t* Q, const void* scales, const void* zeros, void* W,
                    cudaStream_t st);
 
+// loss_kernel.cu -- fused KL + cross-entropy loss and its gradient over [T, V] logits (V % 8 == 0, V <= 32768)
+int launch_lrec_loss(int T, int V, const void* Z, const void* Tt, const int32_t* labels, float lambda_kl, float lambda_ce,
+                     float grad_scale, float* loss_tokens, void* dZ, cudaStream_t st);
+
 // simt_kernels.cu -- CUDA-core kernels, correct for every supported shape
 // In [M, T] bf16 times the dequantised weight, plus s * P L.  transposed = false: forward (T = K, C = N);
 // true: backward-input (T = N, C = K).  P fp32 [M, r] (H or G) may be NULL when r == 0.
