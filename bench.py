@@ -64,7 +64,7 @@ KERNELS_PER_STEP = None           # filled from the library's dispatch (see laun
 
 # DRAM traffic (read + write) per launch of the dominant kernel of the default workload, from the ncu capture
 # summarised in profiles/umma_pair_config2_int4_m2048.md.  Set back to None whenever that kernel changes.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 25.98e6
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 25.93e6
 
 
 def layer_flops(M, K, N, r):
@@ -399,7 +399,7 @@ def run_ours(args):
             "cpu_baseline": {"value": cpu["value"], "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": cpu["sample"]},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
-            "gpu_launches": launches_per_step(M, r) * args.steps,
+            "gpu_launches": launches_per_step(M, r, K, N) * args.steps,
             "clocks": clocks,
         }
         print(json.dumps(line))
@@ -450,14 +450,27 @@ def run_loss(args):
     return 0
 
 
-def launches_per_step(M: int, r: int) -> int:
-    """Kernels the library launches for one fwd + bwd_input + bwd_lora (H, G saved).  Up to 32 tokens the LoRA
-    down-projection is fused into the streaming kernel for r <= 16 (one launch per call); otherwise each of fwd and
-    bwd_input is a down-projection launch plus the dequant-GEMM.  The gradients are a partial-sum and a reduction launch."""
+def pair_kernel_computes_p(M: int, C: int, r: int, sms: int = 148) -> bool:
+    """Mirror of the library's dispatch: above 256 tokens the CTA-pair kernel runs the LoRA down-projection on SM pairs
+    its tiles (512 tokens x 256 of the C output columns) leave idle, when there are enough of them."""
+    if M <= 256 or r == 0 or r > 16:
+        return False
+    tiles = -(-M // 512) * -(-C // 256)
+    blocks = -(-M // 16)
+    n_prod = min(sms // 2 - tiles, -(-blocks // 4))
+    return n_prod > 0 and n_prod * 16 >= blocks
+
+
+def launches_per_step(M: int, r: int, K: int, N: int) -> int:
+    """Kernels the library launches for one fwd + bwd_input + bwd_lora (H, G saved).  Each of fwd and bwd_input is a
+    down-projection launch plus the dequant-GEMM, or the dequant-GEMM alone where it computes H / G itself (up to 32
+    tokens with r <= 16; above 256 tokens where the tiles leave SM pairs idle).  The gradients are a partial-sum and a
+    reduction launch."""
     if r == 0:
         return 2
-    per_call = 1 if (M <= 32 and r <= 16) else 2
-    return 2 * per_call + 2
+    fwd = 1 if (M <= 32 and r <= 16) or pair_kernel_computes_p(M, N, r) else 2
+    bwd = 1 if (M <= 32 and r <= 16) or pair_kernel_computes_p(M, K, r) else 2
+    return fwd + bwd + 2
 
 
 def main():

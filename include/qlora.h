@@ -32,6 +32,9 @@
  *     Section 3.1).
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = the legacy default stream) of
  *     the current device.  No call synchronises the device; outputs are valid in stream order.
+ *   - Calls given the same workspace must be ordered one after the other (same stream, or events): they share
+ *     its contents, and the library keys the few words of device-side bookkeeping some kernels need (counters that
+ *     a launch leaves zeroed) by the workspace address.  Calls with different workspaces may overlap freely.
  *   - Return value: QLORA_OK or a negative QLORA_ERR_* code.  Arguments are validated before anything is
  *     launched; on error nothing has been enqueued.  Nothing is printed, nothing throws.
  *   - Same inputs give bitwise the same outputs on every run (fixed-order reductions, no floating-point atomics).

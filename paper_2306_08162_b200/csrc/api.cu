@@ -160,6 +160,8 @@ static int fwd_common(const qlora_desc* desc, int M, const void* X, const uint8_
         }
         return launch_skinny_gemm(d, M, false, X, Q, scales, zeros, A, B, H, !fused, Y, st);
     }
+    // the tensor-core path computes H itself when given A (beside its tiles where SM pairs are idle, else ahead of them)
+    if (umma_supported(d, M) && mask == nullptr) return launch_umma_gemm(d, M, false, X, Q, scales, zeros, B, H, Y, st, A, workspace);
     if (d.r > 0) {
         rc = launch_lora_down(M, d.K, d.r, true, X, A, H, st, mask, keep_scale);
         if (rc != QLORA_OK) return rc;
@@ -206,11 +208,11 @@ static int bwd_input_common(const qlora_desc* desc, int M, const void* dY, const
         }
         return launch_skinny_gemm(d, M, true, dY, Q, scales, zeros, B, A, G, !fused, dX, st);
     }
+    if (umma_supported(d, M)) return launch_umma_gemm(d, M, true, dY, Q, scales, zeros, A, G, dX, st, B, workspace);   // computes G
     if (d.r > 0) {
         rc = launch_lora_down(M, d.N, d.r, false, dY, B, G, st);
         if (rc != QLORA_OK) return rc;
     }
-    if (umma_supported(d, M)) return launch_umma_gemm(d, M, true, dY, Q, scales, zeros, A, G, dX, st);
     return launch_simt_gemm(d, M, true, dY, Q, scales, zeros, A, G, dX, st);
 }
 

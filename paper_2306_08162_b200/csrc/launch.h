@@ -27,8 +27,9 @@ int launch_simt_gemm(const qlora_desc& d, int M, bool transposed, const void* In
                      cudaStream_t st);
 // P[m, j] = sum_t In[m, t] * L(j, t);  l_is_A: L = A [r, K] (t = k) else L = B [N, r] (t = n).
 // mask (optional, only with l_is_A): uint8 [M, T] dropout mask on In, non-zero = keep; the result is multiplied by out_scale.
+// warps15: sum the contraction in the order of the copy that runs inside the CTA-pair kernel (r <= 16 only).
 int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const void* L, float* P, cudaStream_t st,
-                     const uint8_t* mask = nullptr, float out_scale = 1.0f);
+                     const uint8_t* mask = nullptr, float out_scale = 1.0f, bool warps15 = false);
 // dB = s dY^T H [N, r] and dA = s G^T X [r, K] in one pair of launches (partial sums per row slice, then a fixed-order
 // reduction); scratch needs lora_grad_scratch_bytes().
 size_t lora_grad_scratch_bytes(int M, int K, int N, int r);
@@ -40,10 +41,14 @@ int launch_lora_masked_update(int M, int K, int r, float c, const float* G, cons
                               cudaStream_t st);
 
 // umma_kernel.cu -- tcgen05 tensor-core kernel (both directions); same contract as launch_simt_gemm
+// Ldown == NULL: P is an input.  Ldown != NULL (the adapter applied first: A forward, B backward): P is an output,
+// computed on the way -- by SM pairs the tiles of the CTA-pair kernel leave idle when there are some (they signal the
+// tiles through a pair of counters in device memory chosen by `sync_key`: calls that may overlap in time must pass
+// different keys; the layer calls pass their workspace), otherwise by a down-projection launch ahead of the kernel.
 bool umma_supported(const qlora_desc& d, int M);
 int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q,
-                     const void* scales, const void* zeros, const void* L, const float* P, void* Out,
-                     cudaStream_t st);
+                     const void* scales, const void* zeros, const void* L, float* P, void* Out,
+                     cudaStream_t st, const void* Ldown = nullptr, const void* sync_key = nullptr);
 // Small token counts (M <= 32): TMA-fed mma.sync streaming kernels.  Ldown / Lup: the adapter applied first / second
 // (forward A, B; backward B, A).  P = H or G, fp32 [M, r]: read when p_is_input, otherwise computed inside the kernel
 // (ranks 8 and 16 only) and written out.

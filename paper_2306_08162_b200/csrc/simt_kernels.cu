@@ -3,6 +3,7 @@
 // HBM traffic rather than by arithmetic (Figure 1 of the paper: the green "MM" blocks and their gradients).
 #include "common.cuh"
 #include "launch.h"
+#include "lora_down.cuh"
 
 namespace qlora {
 
@@ -113,114 +114,20 @@ int launch_simt_gemm(const qlora_desc& d, int M, bool transposed, const void* In
 
 // ------------------------------------------------------------------------------------------------------------
 // LoRA down-projections: H = X A^T (contraction over K) and G = dY B (contraction over N), fp32 [M, r].
-// Skinny products bound by reading the activations once, so they use the warp-level mma.sync (m16n8k16, bf16 in,
-// fp32 accumulate) fed straight from 16-byte row loads: a block owns 16 token rows, its warps stride over the
-// contraction in steps of 32 and keep four steps of loads in flight.  The 32 contraction indices of a step are assigned
-// to the fragments in a permuted order (lane q of a quad owns indices 8q..8q+7); activation and adapter fragments use the
-// same permutation, so the sum is unchanged.  A [r, K] is contraction-contiguous and loads directly; B [N, r] is
-// rank-contiguous, so its 8 x 8 fragment tiles are loaded row-wise and transposed across the warp with movmatrix.
-// The per-warp partial tiles are added in warp order through shared memory (fixed order: deterministic).
+// Skinny products bound by reading the activations once: a block owns 16 token rows (lora_down.cuh has the method).
 // ------------------------------------------------------------------------------------------------------------
-constexpr int LD_UNROLL = 4;
-
-__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                               uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-// Transpose an 8 x 8 matrix of 16-bit elements held across the warp (lane l: row l / 4, elements 2 (l % 4), +1).
-// LoRA dropout: keep the bf16 pair elements whose mask byte is non-zero (mask bytes m0, m1 in the low two bytes of `mb`).
-__device__ __forceinline__ uint32_t mask_pair(uint32_t pair, uint32_t mb) {
-    return pair & (((mb & 0xFFu) ? 0x0000FFFFu : 0u) | ((mb & 0xFF00u) ? 0xFFFF0000u : 0u));
-}
-// Eight bf16 (uint4) against eight mask bytes (uint2).
-__device__ __forceinline__ uint4 mask_eight(uint4 x, uint2 m) {
-    return make_uint4(mask_pair(x.x, m.x), mask_pair(x.y, m.x >> 16), mask_pair(x.z, m.y), mask_pair(x.w, m.y >> 16));
-}
-__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
-    uint32_t d;
-    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
-    return d;
-}
-
 template <bool L_IS_A, int NT, int WARPS>
 __global__ void __launch_bounds__(WARPS * 32)
 lora_down_kernel(int M, int T, int r, const __nv_bfloat16* __restrict__ In, const __nv_bfloat16* __restrict__ L,
                  float* __restrict__ P, const uint8_t* __restrict__ mask, float out_scale) {
-    __shared__ float red[WARPS][NT][4][32];
+    __shared__ float red[WARPS * NT * 128];
     pdl_launch_dependents();
     pdl_wait();
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int g = lane >> 2, q = lane & 3;
-    const int m_base = blockIdx.x * 16;
-    const int r0 = m_base + g, r1 = r0 + 8;
-    const __nv_bfloat16* row0 = In + (size_t)r0 * T;
-    const __nv_bfloat16* row1 = In + (size_t)r1 * T;
-    const bool v0 = r0 < M, v1 = r1 < M;
-    float acc[NT][4];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-    const uint4 zero4 = make_uint4(0, 0, 0, 0);
-    for (int kk = warp * 32; kk < T; kk += WARPS * 32 * LD_UNROLL) {
-        uint4 xlo[LD_UNROLL], xhi[LD_UNROLL];
-#pragma unroll
-        for (int u = 0; u < LD_UNROLL; ++u) {                 // all activation loads of the unrolled steps first
-            const int k = kk + u * WARPS * 32 + q * 8;         // T is a multiple of 8: 8 elements are all-in or all-out
-            xlo[u] = (v0 && k < T) ? *reinterpret_cast<const uint4*>(row0 + k) : zero4;
-            xhi[u] = (v1 && k < T) ? *reinterpret_cast<const uint4*>(row1 + k) : zero4;
-            if (mask != nullptr) {   // dropout on the branch input: dropped elements contribute nothing
-                if (v0 && k < T) xlo[u] = mask_eight(xlo[u], __ldg(reinterpret_cast<const uint2*>(mask + (size_t)r0 * T + k)));
-                if (v1 && k < T) xhi[u] = mask_eight(xhi[u], __ldg(reinterpret_cast<const uint2*>(mask + (size_t)r1 * T + k)));
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < LD_UNROLL; ++u) {
-            const int k0 = kk + u * WARPS * 32;                // warp-uniform
-            if (k0 >= T) break;
-            const int k = k0 + q * 8;
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-                uint4 lv = zero4;
-                if (L_IS_A) {
-                    const int j = nt * 8 + g;                  // rank index of this lane's adapter fragment
-                    if (k < T && j < r) lv = __ldg(reinterpret_cast<const uint4*>(L + (size_t)j * T + k));   // A[j, k..k+7]
-                } else {
-                    // tile t: row rho (0..7) <-> n = k0 + 8 (rho / 2) + (rho % 2) + 2 t, columns = ranks 8 nt .. 8 nt + 7;
-                    // after the transpose lane (g, q) holds B[k0 + 8q + 2t, 8nt + g], B[k0 + 8q + 2t + 1, 8nt + g]
-                    uint32_t w[4];
-#pragma unroll
-                    for (int t = 0; t < 4; ++t) {
-                        const int n = k0 + 8 * (g >> 1) + (g & 1) + 2 * t;
-                        uint32_t v = 0;
-                        if (n < T && nt * 8 < r) v = __ldg(reinterpret_cast<const uint32_t*>(L + (size_t)n * r + nt * 8 + 2 * q));
-                        w[t] = movmatrix_trans(v);
-                    }
-                    lv = make_uint4(w[0], w[1], w[2], w[3]);
-                }
-                mma_bf16_16816(acc[nt], xlo[u].x, xhi[u].x, xlo[u].y, xhi[u].y, lv.x, lv.y);
-                mma_bf16_16816(acc[nt], xlo[u].z, xhi[u].z, xlo[u].w, xhi[u].w, lv.z, lv.w);
-            }
-        }
-    }
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-        for (int c = 0; c < 4; ++c) red[warp][nt][c][lane] = acc[nt][c];
-    __syncthreads();
-    for (int idx = threadIdx.x; idx < NT * 128; idx += WARPS * 32) {
-        const int nt = idx >> 7, c = (idx >> 5) & 3, ln = idx & 31;
-        float v = 0.f;
-#pragma unroll
-        for (int w = 0; w < WARPS; ++w) v += red[w][nt][c][ln];
-        const int row = m_base + (ln >> 2) + ((c & 2) ? 8 : 0);
-        const int col = nt * 8 + (ln & 3) * 2 + (c & 1);
-        if (row < M && col < r) P[(size_t)row * r + col] = v * out_scale;
-    }
+    lora_down_rows<L_IS_A, NT>(M, T, r, In, L, P, mask, out_scale, (int)blockIdx.x * 16, WARPS, red);
 }
 
 int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const void* L, float* P, cudaStream_t st,
-                     const uint8_t* mask, float out_scale) {
+                     const uint8_t* mask, float out_scale, bool warps15) {
     if (M == 0 || r == 0) return QLORA_OK;
     const unsigned grid = (unsigned)((M + 15) / 16);
     const __nv_bfloat16* in = (const __nv_bfloat16*)In;
@@ -232,7 +139,10 @@ int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const voi
         if (l_is_A) err = launch_pdl(lora_down_kernel<true, NTV, W>, dim3(grid), dim3(W * 32), 0, st, 1, M, T, r, in, l, P, mask, out_scale);   \
         else        err = launch_pdl(lora_down_kernel<false, NTV, W>, dim3(grid), dim3(W * 32), 0, st, 1, M, T, r, in, l, P, mask, out_scale);  \
     } while (0)
-    if (nt <= 1) QLORA_LD(1, 32);
+    if (warps15 && nt <= 2) {   // the summation order of the copy that runs inside the CTA-pair kernel (15 warps)
+        if (nt <= 1) QLORA_LD(1, 15);
+        else QLORA_LD(2, 15);
+    } else if (nt <= 1) QLORA_LD(1, 32);
     else if (nt <= 2) QLORA_LD(2, 32);
     else if (nt <= 4) QLORA_LD(4, 8);
     else QLORA_LD(8, 8);

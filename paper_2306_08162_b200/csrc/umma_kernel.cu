@@ -20,12 +20,21 @@
 // Every mbarrier wait is bounded; on a timeout the kernel records a status word, drains and returns.
 #include <cuda.h>
 
+#include <mutex>
+#include <unordered_map>
+
 #include "common.cuh"
 #include "launch.h"
+#include "lora_down.cuh"
 
 namespace qlora {
 
 __device__ unsigned int g_device_status = 0;   // sticky; bit 0: an mbarrier wait timed out
+
+// Counter pairs of the CTA-pair kernel's producer clusters: [0] producer CTAs that have published their rows,
+// [1] tile CTAs that have seen the full count.  Zero whenever no launch is using the pair (the kernel restores that).
+constexpr int kSyncSlots = 4096;
+__device__ unsigned int g_pair_sync[kSyncSlots][2];
 
 namespace {
 
@@ -656,8 +665,23 @@ bool umma_supported(const qlora_desc& d, int M) {
 }
 
 // CTA-pair kernel: 512 tokens x 256 weight rows per pair of SMs.  Used when there are more than 256 tokens.
+// One counter pair per key (the caller's workspace address), handed out on first sight and kept: two launches that can
+// overlap in time have different workspaces, hence different pairs.  -1 when the table is full.
+static int sync_slot_for(const void* key) {
+    static std::mutex mu;
+    static std::unordered_map<const void*, int> table;
+    std::lock_guard<std::mutex> lock(mu);
+    const auto it = table.find(key);
+    if (it != table.end()) return it->second;
+    if ((int)table.size() >= kSyncSlots) return -1;
+    const int slot = (int)table.size();
+    table.emplace(key, slot);
+    return slot;
+}
+
 static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
-                            const void* zeros, const void* L, const float* Pmat, void* Out, cudaStream_t st) {
+                            const void* zeros, const void* L, float* Pmat, void* Out, cudaStream_t st, const void* Ldown,
+                            const void* sync_key) {
     PairParams p{};
     p.M = M; p.N = d.N; p.K = d.K; p.bits = d.bits; p.g = d.group_size; p.r = d.r; p.r_pad = (d.r + 15) / 16 * 16;
     p.C = transposed ? d.K : d.N;
@@ -701,7 +725,27 @@ static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const v
         return QLORA_ERR_CUDA;
 
     const int pairs = sm_count() / 2;
-    const int grid = 2 * (p.n_tiles < pairs ? p.n_tiles : pairs);
+    // P = In * Ldown still to be computed: on SM pairs the tiles leave idle when there are enough of them to be done well
+    // before the tiles' contractions are (a 16-row block of the down-projection costs about five pipeline stages of a
+    // tile, so 16 blocks per producer pair keeps it under half of the main loop), else by a launch ahead of this one.
+    p.n_prod = 0; p.T = T; p.slot = 0;
+    p.In = (const __nv_bfloat16*)In; p.Ldown = (const __nv_bfloat16*)Ldown; p.Pout = Pmat;
+    if (Ldown != nullptr && d.r > 0) {
+        const int n_blocks = (M + 15) / 16;
+        const int idle = pairs - p.n_tiles;
+        int n_prod = (n_blocks + 3) / 4;
+        if (n_prod > idle) n_prod = idle;
+        const int slot = (d.r <= 16 && n_prod > 0 && n_prod * 16 >= n_blocks && sync_key != nullptr) ? sync_slot_for(sync_key) : -1;
+        if (slot >= 0) {
+            p.n_prod = n_prod;
+            p.slot = slot;
+        } else {
+            const int rc = launch_lora_down(M, T, d.r, !transposed, In, Ldown, Pmat, st, nullptr, 1.0f,
+                                            /*warps15=*/d.r <= 16 && n_prod > 0 && n_prod * 16 >= n_blocks);
+            if (rc != QLORA_OK) return rc;
+        }
+    }
+    const int grid = 2 * ((p.n_tiles < pairs ? p.n_tiles : pairs) + p.n_prod);
 #define QLORA_LAUNCH_PAIR(B)                                                                              \
     return transposed ? launch_pair_impl<B, true>(ta, tq, ts, tz, p, smem_bytes, grid, st)                \
                       : launch_pair_impl<B, false>(ta, tq, ts, tz, p, smem_bytes, grid, st)
@@ -716,8 +760,13 @@ static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const v
 }
 
 int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
-                     const void* zeros, const void* L, const float* Pmat, void* Out, cudaStream_t st) {
-    if (M > 256) return launch_umma_pair(d, M, transposed, In, Q, scales, zeros, L, Pmat, Out, st);
+                     const void* zeros, const void* L, float* Pmat, void* Out, cudaStream_t st, const void* Ldown,
+                     const void* sync_key) {
+    if (M > 256) return launch_umma_pair(d, M, transposed, In, Q, scales, zeros, L, Pmat, Out, st, Ldown, sync_key);
+    if (Ldown != nullptr && d.r > 0) {
+        const int rc = launch_lora_down(M, transposed ? d.N : d.K, d.r, !transposed, In, Ldown, Pmat, st);
+        if (rc != QLORA_OK) return rc;
+    }
     Params p{};
     p.M = M; p.N = d.N; p.K = d.K; p.bits = d.bits; p.g = d.group_size; p.r = d.r; p.r_pad = (d.r + 15) / 16 * 16;
     p.C = transposed ? d.K : d.N;
@@ -796,6 +845,10 @@ int read_device_status(unsigned int* out, int clear) {
     if (clear && v != 0) {
         const unsigned int zero = 0;
         if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(zero)) != cudaSuccess) return QLORA_ERR_CUDA;
+        // a launch that gave up may have left its counter pair non-zero (the caller has synchronised the device)
+        void* sync = nullptr;
+        if (cudaGetSymbolAddress(&sync, g_pair_sync) != cudaSuccess || cudaMemset(sync, 0, sizeof(unsigned int) * 2 * kSyncSlots) != cudaSuccess)
+            return QLORA_ERR_CUDA;
     }
     *out = v;
     return QLORA_OK;

@@ -15,6 +15,13 @@
 // and collect arrivals from both CTAs (remote mbarrier arrive / TMA complete_tx); barriers that both CTAs wait on
 // (stage free, accumulators complete) exist in both and are signalled by one multicast tcgen05.commit.
 // Every wait is bounded, as in the single-CTA kernel; the CTAs leave together through a cluster barrier.
+//
+// When the tiles leave SM pairs idle (fewer tiles than pairs), the launch can add `n_prod` producer clusters in front of
+// the tile clusters (lowest block indices, so they are dispatched first and wait for nobody): their CTAs compute the LoRA
+// down-projection P = In * Ldown (lora_down.cuh) beside the main loops and publish it through a counter in device
+// memory; a tile's epilogue warps wait for that counter before they stage P for the LoRA update, which is only needed
+// once the tile's contraction is through.  The counter pair belongs to one launch at a time (the host hands out one
+// pair per workspace) and the last CTA to have seen the count zeroes it again.
 
 constexpr int kPairTok = 128;                          // token rows per CTA per accumulator
 constexpr int kPairW = 128;                            // weight rows per CTA (256 per pair tile)
@@ -33,7 +40,32 @@ struct PairParams {
     const float* Pmat;           // H (forward) or G (backward), fp32 [M, r]
     const __nv_bfloat16* L;      // B [N, r] (forward) or A [r, K] (backward)
     __nv_bfloat16* Out;
+    // producer clusters (n_prod > 0): P = In * Ldown is computed by this launch and written to Pout (== Pmat)
+    int n_prod, T, slot;
+    const __nv_bfloat16* In;     // [M, T]
+    const __nv_bfloat16* Ldown;  // A [r, K] (forward) or B [N, r] (backward)
+    float* Pout;
 };
+
+// Bounded wait until a counter in global memory reaches `target` (written by other CTAs of the same launch).
+__device__ __forceinline__ bool wait_counter(const unsigned* ctr, unsigned target, volatile int* abort_flag) {
+    uint64_t t0 = 0;
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        unsigned v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+        if (v >= target) return true;
+        __nanosleep(256);
+        if ((i & 63u) == 63u) {
+            if (*abort_flag) return false;
+            const uint64_t now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) break;
+        }
+    }
+    *abort_flag = 1;
+    atomicOr(&g_device_status, 1u);
+    return false;
+}
 
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
@@ -114,7 +146,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t S = (uint32_t)p.S, P = (uint32_t)p.P;
     const uint32_t cta = cluster_ctarank();            // 0 = leader (issues the MMAs), 1 = follower
-    const int first_tile = (int)(blockIdx.x >> 1), tile_stride = (int)(gridDim.x >> 1);
+    const int first_tile = (int)(blockIdx.x >> 1) - p.n_prod, tile_stride = (int)(gridDim.x >> 1) - p.n_prod;
 
     // barriers (same offsets in both CTAs)
     const uint32_t bar_full_x = smem0 + p.off_bar;          // [S] leader's: activation sub-tiles of both CTAs landed (TMA)
@@ -153,7 +185,18 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     const uint32_t tmem_base = tmem_base_slot;
     pdl_wait();                // set-up done; from here on global memory is touched
 
-    if (warp == 0) {
+    if (first_tile < 0) {
+        // ------------------------------------------------------------------ producer cluster: LoRA down-projection
+        float* red = reinterpret_cast<float*>(smem_gen);
+        const int n_blocks = (p.M + 15) / 16;
+        for (int b = (int)blockIdx.x; b < n_blocks; b += 2 * p.n_prod) {
+            if (p.r <= 8) lora_down_rows<!TRANSPOSED, 1>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, nullptr, 1.0f, b * 16, kThreads / 32, red);
+            else          lora_down_rows<!TRANSPOSED, 2>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, nullptr, 1.0f, b * 16, kThreads / 32, red);
+        }
+        __threadfence();       // every thread's rows of P are visible device-wide before the CTA is counted
+        __syncthreads();
+        if (threadIdx.x == 0) atomicAdd(&g_pair_sync[p.slot][0], 1u);
+    } else if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer: activation sub-tiles
         if (lane == 0) {
             Ring ring;
@@ -258,6 +301,19 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             const int wt = tile / p.n_tok_tiles, tt = tile % p.n_tok_tiles;
             const int w0 = wt * (2 * kPairW);                          // first weight row (output column) of the pair tile
             const int m0 = tt * (4 * kPairTok) + (int)cta * kPairTok;  // this CTA's first token row of accumulator 0
+            if (p.n_prod > 0 && tile_it == 0) {
+                // P is being computed by the producer clusters of this launch: one thread waits for all of their CTAs, is
+                // counted as done with the counter, and the last such CTA of the launch zeroes the pair for the next one.
+                if (et == 0 && wait_counter(&g_pair_sync[p.slot][0], 2u * (unsigned)p.n_prod, abort_flag)) {
+                    const unsigned n_cons = gridDim.x - 2u * (unsigned)p.n_prod;
+                    if (atomicAdd(&g_pair_sync[p.slot][1], 1u) == n_cons - 1u) {
+                        atomicExch(&g_pair_sync[p.slot][0], 0u);
+                        atomicExch(&g_pair_sync[p.slot][1], 0u);
+                    }
+                }
+                asm volatile("bar.sync 2, %0;" ::"r"(kEpiWarps * 32) : "memory");
+                if (*abort_flag) break;
+            }
             if (p.r > 0) {
                 // (the previous tile's LoRA MMA has completed: its accumulator-full barrier was observed below)
                 uint8_t* ll = smem_gen + p.off_lora_l;
@@ -286,8 +342,9 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                     for (int jc = 0; jc < p.r_pad / 8; ++jc) {
                         uint4 v = make_uint4(0, 0, 0, 0);
                         if (jc * 8 < p.r && m < p.M) {
-                            const float4 x = __ldg(reinterpret_cast<const float4*>(p.Pmat + (size_t)m * p.r + jc * 8));
-                            const float4 y = __ldg(reinterpret_cast<const float4*>(p.Pmat + (size_t)m * p.r + jc * 8 + 4));
+                            // (not the read-only path: P may have been written by this launch's producer clusters)
+                            const float4 x = __ldcg(reinterpret_cast<const float4*>(p.Pmat + (size_t)m * p.r + jc * 8));
+                            const float4 y = __ldcg(reinterpret_cast<const float4*>(p.Pmat + (size_t)m * p.r + jc * 8 + 4));
                             __nv_bfloat162 h0 = __floats2bfloat162_rn(p.s * x.x, p.s * x.y), h1 = __floats2bfloat162_rn(p.s * x.z, p.s * x.w);
                             __nv_bfloat162 h2 = __floats2bfloat162_rn(p.s * y.x, p.s * y.y), h3 = __floats2bfloat162_rn(p.s * y.z, p.s * y.w);
                             v = make_uint4(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1),

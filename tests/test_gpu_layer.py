@@ -208,6 +208,44 @@ def test_activation_order_through_row_permutation_and_column_gather(M):
     assert rel_err(to_f64(dA), dAo) <= REL_TOL and rel_err(to_f64(out["dB"]), dBo) <= REL_TOL
 
 
+def test_down_projection_beside_the_tiles_repeats_bitwise_and_on_two_streams():
+    """Above 256 tokens with few tiles the pair kernel's spare SM pairs compute H / G during the main loop and publish them
+    through a counter pair that the launch zeroes again: repeated launches, and launches of two layers (two workspaces)
+    overlapping on two streams, give the same bits as a first, serial run."""
+    la = qi.random_codes_layer(K=512, N=512, bits=4, group_size=128, r=8, alpha=16.0, M=600, seed=11)
+    lb = qi.random_codes_layer(K=768, N=256, bits=2, group_size=64, r=16, alpha=32.0, M=1000, seed=12)
+    _, ra, ga = check_layer(la)
+    _, rb, gb = check_layer(lb)
+    keys = ("Y", "dX", "H", "G", "dA", "dB")
+    bits = lambda t: t.view(torch.int16) if t.dtype == torch.bfloat16 else t
+    for _ in range(3):
+        again = ga.run()
+        for k in keys:
+            assert torch.equal(bits(again[k]), bits(ra[k])), k
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    outs = []
+    for _ in range(6):
+        with torch.cuda.stream(sa):
+            Ya = torch.empty_like(ra["Y"]); Ha = torch.empty_like(ra["H"])
+            ql_fwd(ga, Ya, Ha)
+        with torch.cuda.stream(sb):
+            Yb = torch.empty_like(rb["Y"]); Hb = torch.empty_like(rb["H"])
+            ql_fwd(gb, Yb, Hb)
+        outs.append((Ya, Ha, Yb, Hb))
+    torch.cuda.synchronize()
+    import paper_2306_08162_b200 as ql
+    assert ql.qlora_device_status() == 0
+    for Ya, Ha, Yb, Hb in outs:
+        assert torch.equal(bits(Ya), bits(ra["Y"])) and torch.equal(Ha, ra["H"])
+        assert torch.equal(bits(Yb), bits(rb["Y"])) and torch.equal(Hb, rb["H"])
+
+
+def ql_fwd(gl, Y, H):
+    import paper_2306_08162_b200 as ql
+    ql.qlora_fwd(gl.desc, gl.M, gl.X, gl.Q, gl.scales, gl.zeros, gl.A, gl.B, Y, H, gl.ws)
+
+
 def test_recompute_h_g_matches_saved():
     layer = qi.random_codes_layer(K=512, N=256, bits=4, group_size=128, r=8, alpha=16.0, M=200, seed=3)
     _, saved, gl = check_layer(layer, save_hg=True)
