@@ -27,9 +27,11 @@ int launch_simt_gemm(const qlora_desc& d, int M, bool transposed, const void* In
                      cudaStream_t st);
 // P[m, j] = sum_t In[m, t] * L(j, t);  l_is_A: L = A [r, K] (t = k) else L = B [N, r] (t = n).
 // mask (optional, only with l_is_A): uint8 [M, T] dropout mask on In, non-zero = keep; the result is multiplied by out_scale.
-// warps15: sum the contraction in the order of the copy that runs inside the CTA-pair kernel (r <= 16 only).
 int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const void* L, float* P, cudaStream_t st,
-                     const uint8_t* mask = nullptr, float out_scale = 1.0f, bool warps15 = false);
+                     const uint8_t* mask = nullptr, float out_scale = 1.0f);
+// umma_kernel.cu -- the same product for many rows and r <= 16: activations streamed through shared memory by bulk
+// copies (launch_lora_down routes there above 256 rows; the CTA-pair kernel runs the same code on idle SM pairs).
+int launch_lora_down_stream(int M, int T, int r, bool l_is_A, const void* In, const void* L, float* P, cudaStream_t st);
 // dB = s dY^T H [N, r] and dA = s G^T X [r, K] in one pair of launches (partial sums per row slice, then a fixed-order
 // reduction); scratch needs lora_grad_scratch_bytes().
 size_t lora_grad_scratch_bytes(int M, int K, int N, int r);

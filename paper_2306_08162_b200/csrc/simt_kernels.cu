@@ -127,8 +127,11 @@ lora_down_kernel(int M, int T, int r, const __nv_bfloat16* __restrict__ In, cons
 }
 
 int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const void* L, float* P, cudaStream_t st,
-                     const uint8_t* mask, float out_scale, bool warps15) {
+                     const uint8_t* mask, float out_scale) {
     if (M == 0 || r == 0) return QLORA_OK;
+    // Many rows, low rank: the streaming kernel (also the form that runs inside the CTA-pair kernel, so H / G have the
+    // same bits whichever call produced them).
+    if (mask == nullptr && out_scale == 1.0f && M > 256 && r <= 16) return launch_lora_down_stream(M, T, r, l_is_A, In, L, P, st);
     const unsigned grid = (unsigned)((M + 15) / 16);
     const __nv_bfloat16* in = (const __nv_bfloat16*)In;
     const __nv_bfloat16* l = (const __nv_bfloat16*)L;
@@ -139,10 +142,7 @@ int launch_lora_down(int M, int T, int r, bool l_is_A, const void* In, const voi
         if (l_is_A) err = launch_pdl(lora_down_kernel<true, NTV, W>, dim3(grid), dim3(W * 32), 0, st, 1, M, T, r, in, l, P, mask, out_scale);   \
         else        err = launch_pdl(lora_down_kernel<false, NTV, W>, dim3(grid), dim3(W * 32), 0, st, 1, M, T, r, in, l, P, mask, out_scale);  \
     } while (0)
-    if (warps15 && nt <= 2) {   // the summation order of the copy that runs inside the CTA-pair kernel (15 warps)
-        if (nt <= 1) QLORA_LD(1, 15);
-        else QLORA_LD(2, 15);
-    } else if (nt <= 1) QLORA_LD(1, 32);
+    if (nt <= 1) QLORA_LD(1, 32);
     else if (nt <= 2) QLORA_LD(2, 32);
     else if (nt <= 4) QLORA_LD(4, 8);
     else QLORA_LD(8, 8);

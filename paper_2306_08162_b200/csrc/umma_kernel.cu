@@ -573,10 +573,15 @@ int launch_impl(const CUtensorMap& ta, const CUtensorMap& tq, const CUtensorMap&
                ? QLORA_OK : QLORA_ERR_CUDA;
 }
 
+#include "lora_down_stream.cuh"
 #include "umma_pair.cuh"
 #include "skinny_kernel.cuh"
 
 }  // namespace
+
+int launch_lora_down_stream(int M, int T, int r, bool l_is_A, const void* In, const void* L, float* P, cudaStream_t st) {
+    return launch_lora_down_stream_impl(M, T, r, l_is_A, In, L, P, st);
+}
 
 bool skinny_supported(const qlora_desc& d, int M) {
     if (M < 1 || M > 32) return false;
@@ -725,23 +730,24 @@ static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const v
         return QLORA_ERR_CUDA;
 
     const int pairs = sm_count() / 2;
-    // P = In * Ldown still to be computed: on SM pairs the tiles leave idle when there are enough of them to be done well
-    // before the tiles' contractions are (a 16-row block of the down-projection costs about five pipeline stages of a
-    // tile, so 16 blocks per producer pair keeps it under half of the main loop), else by a launch ahead of this one.
+    // P = In * Ldown still to be computed: on SM pairs the tiles leave idle when they can take all row blocks (they are
+    // then done well before the tiles' contractions are), else by a launch ahead of this one.  Both sum in the same order.
     p.n_prod = 0; p.T = T; p.slot = 0;
     p.In = (const __nv_bfloat16*)In; p.Ldown = (const __nv_bfloat16*)Ldown; p.Pout = Pmat;
+    p.lds_stages = (int)((p.off_bar - LDS_BAR_BYTES) / LDS_STAGE_BYTES);
+    if (p.lds_stages > 6) p.lds_stages = 6;
     if (Ldown != nullptr && d.r > 0) {
         const int n_blocks = (M + 15) / 16;
         const int idle = pairs - p.n_tiles;
-        int n_prod = (n_blocks + 3) / 4;
+        int n_prod = (n_blocks + 3) / 4;                     // four row blocks per producer CTA pair when there is room
         if (n_prod > idle) n_prod = idle;
-        const int slot = (d.r <= 16 && n_prod > 0 && n_prod * 16 >= n_blocks && sync_key != nullptr) ? sync_slot_for(sync_key) : -1;
+        const bool fits = d.r <= 16 && n_prod > 0 && n_prod * 2 * LDS_MAXB >= n_blocks && p.lds_stages >= LDS_MIN_STAGES;
+        const int slot = (fits && sync_key != nullptr) ? sync_slot_for(sync_key) : -1;
         if (slot >= 0) {
             p.n_prod = n_prod;
             p.slot = slot;
         } else {
-            const int rc = launch_lora_down(M, T, d.r, !transposed, In, Ldown, Pmat, st, nullptr, 1.0f,
-                                            /*warps15=*/d.r <= 16 && n_prod > 0 && n_prod * 16 >= n_blocks);
+            const int rc = launch_lora_down(M, T, d.r, !transposed, In, Ldown, Pmat, st);
             if (rc != QLORA_OK) return rc;
         }
     }

@@ -18,7 +18,7 @@
 //
 // When the tiles leave SM pairs idle (fewer tiles than pairs), the launch can add `n_prod` producer clusters in front of
 // the tile clusters (lowest block indices, so they are dispatched first and wait for nobody): their CTAs compute the LoRA
-// down-projection P = In * Ldown (lora_down.cuh) beside the main loops and publish it through a counter in device
+// down-projection P = In * Ldown (lora_down_stream.cuh) beside the main loops and publish it through a counter in device
 // memory; a tile's epilogue warps wait for that counter before they stage P for the LoRA update, which is only needed
 // once the tile's contraction is through.  The counter pair belongs to one launch at a time (the host hands out one
 // pair per workspace) and the last CTA to have seen the count zeroes it again.
@@ -41,7 +41,7 @@ struct PairParams {
     const __nv_bfloat16* L;      // B [N, r] (forward) or A [r, K] (backward)
     __nv_bfloat16* Out;
     // producer clusters (n_prod > 0): P = In * Ldown is computed by this launch and written to Pout (== Pmat)
-    int n_prod, T, slot;
+    int n_prod, T, slot, lds_stages;
     const __nv_bfloat16* In;     // [M, T]
     const __nv_bfloat16* Ldown;  // A [r, K] (forward) or B [N, r] (backward)
     float* Pout;
@@ -187,12 +187,9 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
 
     if (first_tile < 0) {
         // ------------------------------------------------------------------ producer cluster: LoRA down-projection
-        float* red = reinterpret_cast<float*>(smem_gen);
-        const int n_blocks = (p.M + 15) / 16;
-        for (int b = (int)blockIdx.x; b < n_blocks; b += 2 * p.n_prod) {
-            if (p.r <= 8) lora_down_rows<!TRANSPOSED, 1>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, nullptr, 1.0f, b * 16, kThreads / 32, red);
-            else          lora_down_rows<!TRANSPOSED, 2>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, nullptr, 1.0f, b * 16, kThreads / 32, red);
-        }
+        // (this CTA's row blocks: blockIdx.x, blockIdx.x + 2 n_prod, ...; the ring takes the operand area, below the barriers)
+        if (p.r <= 8) lora_down_stream<!TRANSPOSED, 1>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, 2 * p.n_prod, smem_gen, p.lds_stages, abort_flag);
+        else          lora_down_stream<!TRANSPOSED, 2>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, 2 * p.n_prod, smem_gen, p.lds_stages, abort_flag);
         __threadfence();       // every thread's rows of P are visible device-wide before the CTA is counted
         __syncthreads();
         if (threadIdx.x == 0) atomicAdd(&g_pair_sync[p.slot][0], 1u);
