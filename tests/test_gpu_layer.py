@@ -49,6 +49,45 @@ def test_config2_q_proj_int4():
     check_layer(qi.config2())
 
 
+def test_config2_as_a_replayed_cuda_graph():
+    """The launch configuration the benchmark times: the three calls of several steps captured in one CUDA graph
+    (programmatic dependent launches, the pair kernel's self-zeroing counters) and replayed twice; every replay's
+    outputs are checked against the oracle on sampled rows and are bitwise those of the call-by-call run."""
+    layer = qi.config2(seed=3)
+    rows = sample_rows(layer["M"], seed=5)
+    _, eager, gl = check_layer(layer, rows=rows)
+    import paper_2306_08162_b200 as ql
+    M, dev = gl.M, gl.X.device
+    bufs = [dict(Y=torch.empty((M, gl.N), dtype=torch.bfloat16, device=dev), dX=torch.empty((M, gl.K), dtype=torch.bfloat16, device=dev),
+                 H=torch.empty((M, gl.r), dtype=torch.float32, device=dev), G=torch.empty((M, gl.r), dtype=torch.float32, device=dev),
+                 dA=torch.empty((gl.r, gl.K), dtype=torch.float32, device=dev), dB=torch.empty((gl.N, gl.r), dtype=torch.float32, device=dev))
+            for _ in range(3)]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for b in bufs:
+                ql.qlora_fwd(gl.desc, M, gl.X, gl.Q, gl.scales, gl.zeros, gl.A, gl.B, b["Y"], b["H"], gl.ws)
+                ql.qlora_bwd_input(gl.desc, M, gl.dY, gl.Q, gl.scales, gl.zeros, gl.A, gl.B, b["dX"], b["G"], gl.ws)
+                ql.qlora_bwd_lora(gl.desc, M, gl.X, gl.dY, gl.A, gl.B, b["H"], b["G"], b["dA"], b["dB"], 0, gl.ws)
+    ref = orc.layer_reference(layer, rows=rows)
+    sel = np.asarray(rows)
+    bits = lambda t: t.view(torch.int16) if t.dtype == torch.bfloat16 else t
+    for replay in range(2):
+        for b in bufs:
+            for t in b.values():
+                t.view(torch.int16 if t.dtype == torch.bfloat16 else torch.int32).fill_(-1)      # NaN patterns: nothing is left over
+        graph.replay()
+        torch.cuda.synchronize()
+        assert ql.qlora_device_status() == 0
+        for b in bufs:
+            assert rel_err(to_f64(b["Y"])[sel], ref["Y"]) <= REL_TOL and rel_err(to_f64(b["dX"])[sel], ref["dX"]) <= REL_TOL
+            assert rel_err(to_f64(b["dA"]), ref["dA"]) <= REL_TOL and rel_err(to_f64(b["dB"]), ref["dB"]) <= REL_TOL
+            for k in ("Y", "dX", "H", "G", "dA", "dB"):
+                assert torch.equal(bits(b[k]), bits(eager[k])), (replay, k)
+
+
 @pytest.mark.parametrize("which", ["gate", "up", "down"])
 def test_config3_mlp_int2_outliers(which):
     layer = qi.config3(which)
