@@ -492,15 +492,30 @@ def pair_kernel_computes_p(M: int, C: int, r: int, sms: int = 148) -> bool:
     return n_prod > 0 and n_prod * 16 >= blocks
 
 
+def mid_kernel_computes_p(M: int, C: int, T: int, r: int, sms: int = 148) -> bool:
+    """Mirror of the dispatch for 33..256 tokens: tiles of 128 output columns, the contraction split over clusters of 4 or
+    2 CTAs when that still fits the GPU; producer clusters are added while the GPU can hold more clusters of that width
+    (33 of width 4, 74 of width 2) and two row blocks of 16 tokens per producer CTA cover the batch."""
+    if not (32 < M <= 256) or r == 0 or r > 16:
+        return False
+    tiles, steps, bt = -(-C // 128), T // 64, (256 if M > 128 else 128 if M > 64 else 64)
+    split = next((sp for sp in (4, 2) if tiles * sp <= sms and steps % sp == 0 and steps // sp >= 4 and bt % sp == 0), 1)
+    clusters = tiles if split > 1 else min(tiles, sms)
+    idle = {1: sms, 2: sms // 2, 4: 33}[split] - clusters
+    blocks = -(-M // 16)
+    n_prod = min(idle, -(-blocks // split))
+    return n_prod > 0 and n_prod * split * 2 >= blocks
+
+
 def launches_per_step(M: int, r: int, K: int, N: int) -> int:
     """Kernels the library launches for one fwd + bwd_input + bwd_lora (H, G saved).  Each of fwd and bwd_input is a
     down-projection launch plus the dequant-GEMM, or the dequant-GEMM alone where it computes H / G itself (up to 32
-    tokens with r <= 16; above 256 tokens where the tiles leave SM pairs idle).  The gradients are a partial-sum and a
-    reduction launch."""
+    tokens with r <= 16; above that where the tiles leave SMs idle).  The gradients are a partial-sum and a reduction
+    launch."""
     if r == 0:
         return 2
-    fwd = 1 if (M <= 32 and r <= 16) or pair_kernel_computes_p(M, N, r) else 2
-    bwd = 1 if (M <= 32 and r <= 16) or pair_kernel_computes_p(M, K, r) else 2
+    fwd = 1 if (M <= 32 and r <= 16) or pair_kernel_computes_p(M, N, r) or mid_kernel_computes_p(M, N, K, r) else 2
+    bwd = 1 if (M <= 32 and r <= 16) or pair_kernel_computes_p(M, K, r) or mid_kernel_computes_p(M, K, N, r) else 2
     return fwd + bwd + 2
 
 

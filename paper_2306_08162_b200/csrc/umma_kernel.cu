@@ -35,6 +35,7 @@ __device__ unsigned int g_device_status = 0;   // sticky; bit 0: an mbarrier wai
 // [1] tile CTAs that have seen the full count.  Zero whenever no launch is using the pair (the kernel restores that).
 constexpr int kSyncSlots = 4096;
 __device__ unsigned int g_pair_sync[kSyncSlots][2];
+int sync_slot_for(const void* key);   // host: the counter pair of a workspace address (-1: table full)
 
 namespace {
 
@@ -64,6 +65,12 @@ struct Params {
     const float* Pmat;               // H (forward) or G (backward), fp32 [M, r]
     const __nv_bfloat16* L;          // B [N, r] (forward) or A [r, K] (backward)
     __nv_bfloat16* Out;
+    // producer clusters (n_prod > 0, as in the CTA-pair kernel): the first n_prod clusters of the grid compute
+    // P = In * Ldown into Pout (== Pmat) beside the tiles and publish it through counter pair `slot`
+    int n_prod, T, slot, lds_stages;
+    const __nv_bfloat16* In;         // [M, T]
+    const __nv_bfloat16* Ldown;      // A [r, K] (forward) or B [N, r] (backward)
+    float* Pout;
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -167,6 +174,29 @@ __device__ __forceinline__ float ld_cluster_f32(uint32_t cluster_addr) {
 }
 
 
+// Bounded wait until a counter in global memory reaches `target` (written by other CTAs of the same launch).
+__device__ __forceinline__ bool wait_counter(const unsigned* ctr, unsigned target, volatile int* abort_flag) {
+    uint64_t t0 = 0;
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        unsigned v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+        if (v >= target) return true;
+        __nanosleep(256);
+        if ((i & 63u) == 63u) {
+            if (*abort_flag) return false;
+            const uint64_t now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) break;
+        }
+    }
+    *abort_flag = 1;
+    atomicOr(&g_device_status, 1u);
+    return false;
+}
+
+int sm_count();
+#include "lora_down_stream.cuh"
+
 // Shared-memory matrix descriptor (version 1).  Offsets in bytes; layout 0 = no swizzle, 2 = 128-byte swizzle.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo, uint32_t layout) {
     return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) |
@@ -242,10 +272,19 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     // i * p.steps ...), each accumulates its part in tensor memory, and the parts are added through distributed shared
     // memory at the end.  One tile per cluster in that mode.
     const int rank = p.split > 1 ? (int)cluster_ctarank() : 0;
-    const int first_tile = blockIdx.x / p.split, tile_stride = gridDim.x / p.split;
+    const int first_tile = (int)blockIdx.x / p.split - p.n_prod, tile_stride = (int)gridDim.x / p.split - p.n_prod;
     const int step0 = rank * p.steps;
 
-    if (warp == 0) {
+    if (first_tile < 0) {
+        // ------------------------------------------------------------------ producer cluster: LoRA down-projection on SMs
+        // the tiles leave idle (one CTA per row block or more; lowest block indices, so they wait for nobody)
+        const int n_ctas = p.n_prod * p.split;
+        if (p.r <= 8) lora_down_stream<!TRANSPOSED, 1>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, n_ctas, smem_gen, p.lds_stages, abort_flag);
+        else          lora_down_stream<!TRANSPOSED, 2>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, n_ctas, smem_gen, p.lds_stages, abort_flag);
+        __threadfence();       // every thread's rows of P are visible device-wide before the CTA is counted
+        __syncthreads();
+        if (threadIdx.x == 0) atomicAdd(&g_pair_sync[p.slot][0], 1u);
+    } else if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer: activation tiles
         if (lane == 0) {
             Ring ring;
@@ -346,7 +385,20 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             const int wt = tile / p.n_tok_tiles, tt = tile % p.n_tok_tiles;
             const int w0 = wt * kWRows, m0 = tt * p.BT;
             const uint32_t buf = tile_it & 1u;
-            if (p.r > 0) {
+            if (p.n_prod > 0 && tile_it == 0 && rank == 0) {
+                // P is being computed by this launch's producer clusters: one thread waits for all of their CTAs, is counted
+                // as done with the counter, and the last such CTA of the launch zeroes the pair for the next one.
+                if (et == 0 && wait_counter(&g_pair_sync[p.slot][0], (unsigned)(p.n_prod * p.split), abort_flag)) {
+                    const unsigned n_cons = gridDim.x / (unsigned)p.split - (unsigned)p.n_prod;   // one waiting CTA per tile cluster
+                    if (atomicAdd(&g_pair_sync[p.slot][1], 1u) == n_cons - 1u) {
+                        atomicExch(&g_pair_sync[p.slot][0], 0u);
+                        atomicExch(&g_pair_sync[p.slot][1], 0u);
+                    }
+                }
+                asm volatile("bar.sync 2, %0;" ::"r"(kEpiWarps * 32) : "memory");
+                if (*abort_flag) break;
+            }
+            if (p.r > 0 && rank == 0) {   // (the LoRA update goes into rank 0's part only)
                 // (the previous tile's LoRA MMA has completed: its accumulator-full barrier was observed below)
                 uint8_t* la = smem_gen + p.off_lora_a;
                 uint8_t* lp = smem_gen + p.off_lora_p;
@@ -371,8 +423,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                     for (int jc = 0; jc < p.r_pad / 8; ++jc) {
                         uint4 v = make_uint4(0, 0, 0, 0);
                         if (jc * 8 < p.r && m < p.M) {
-                            const float4 a = __ldg(reinterpret_cast<const float4*>(p.Pmat + (size_t)m * p.r + jc * 8));
-                            const float4 b = __ldg(reinterpret_cast<const float4*>(p.Pmat + (size_t)m * p.r + jc * 8 + 4));
+                            // (not the read-only path: P may have been written by this launch's producer clusters)
+                            const float4 a = __ldcg(reinterpret_cast<const float4*>(p.Pmat + (size_t)m * p.r + jc * 8));
+                            const float4 b = __ldcg(reinterpret_cast<const float4*>(p.Pmat + (size_t)m * p.r + jc * 8 + 4));
                             __nv_bfloat162 h0 = __floats2bfloat162_rn(p.s * a.x, p.s * a.y), h1 = __floats2bfloat162_rn(p.s * a.z, p.s * a.w);
                             __nv_bfloat162 h2 = __floats2bfloat162_rn(p.s * b.x, p.s * b.y), h3 = __floats2bfloat162_rn(p.s * b.z, p.s * b.w);
                             v = make_uint4(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1),
@@ -498,7 +551,7 @@ done:
         // Add the ranks' parts in rank order (fixed order: deterministic); rank i finishes tokens i * BT / split ...
         __syncwarp();
         cluster_sync_all();
-        if (!*abort_flag && first_tile < p.n_tiles) {
+        if (!*abort_flag && first_tile >= 0 && first_tile < p.n_tiles) {
             const int wt = first_tile / p.n_tok_tiles, tt = first_tile % p.n_tok_tiles;
             const int w0 = wt * kWRows, m0 = tt * p.BT;
             const int tok_per_rank = p.BT / p.split;
@@ -559,21 +612,56 @@ int sm_count() {
     return n;
 }
 
+// Ldown != NULL: P = In * Ldown is still to be computed.  Where the tile clusters leave room for more clusters on the GPU
+// (cudaOccupancyMaxActiveClusters: 33 clusters of 4 fit on 148 SMs, 74 of 2), producer clusters in front of the grid do
+// it beside the tiles; else a down-projection launch goes ahead of the kernel.
 template <int BITS, bool TRANSPOSED>
-int launch_impl(const CUtensorMap& ta, const CUtensorMap& tq, const CUtensorMap& ts, const CUtensorMap& tz, const Params& p,
-                size_t smem_bytes, int grid, cudaStream_t st) {
+int launch_impl(const CUtensorMap& ta, const CUtensorMap& tq, const CUtensorMap& ts, const CUtensorMap& tz, const Params& p_in,
+                size_t smem_bytes, int grid, cudaStream_t st, const void* Ldown, const void* sync_key) {
     static bool configured = false;   // raising the dynamic shared-memory limit is a per-function, per-process setting
+    static int max_clusters[5] = {0, 0, 0, 0, 0};   // by cluster width
     auto kern = umma_gemm_kernel<BITS, TRANSPOSED>;
     if (!configured) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024) != cudaSuccess) return QLORA_ERR_CUDA;
         configured = true;
+    }
+    Params p = p_in;
+    p.n_prod = 0; p.slot = 0;
+    if (Ldown != nullptr && p.r > 0) {
+        if (max_clusters[p.split] == 0) {
+            cudaLaunchConfig_t cfg{};
+            cfg.gridDim = dim3((unsigned)(sm_count() / p.split * p.split));
+            cfg.blockDim = dim3(kThreads);
+            cfg.dynamicSmemBytes = 232448 - 1024;
+            cudaLaunchAttribute attr;
+            attr.id = cudaLaunchAttributeClusterDimension;
+            attr.val.clusterDim.x = (unsigned)p.split; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+            cfg.attrs = &attr;
+            cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) { (void)cudaGetLastError(); n = -1; }
+            max_clusters[p.split] = n;
+        }
+        const int n_blocks = (p.M + 15) / 16;
+        const int idle = max_clusters[p.split] - grid / p.split;
+        int n_prod = (n_blocks + p.split - 1) / p.split;           // one row block per producer CTA when there is room
+        if (n_prod > idle) n_prod = idle;
+        const bool fits = p.r <= 16 && n_prod > 0 && n_prod * p.split * 2 >= n_blocks && p.lds_stages >= LDS_MIN_STAGES;
+        const int slot = (fits && sync_key != nullptr) ? sync_slot_for(sync_key) : -1;
+        if (slot >= 0) {
+            p.n_prod = n_prod;
+            p.slot = slot;
+            grid += n_prod * p.split;
+        } else {
+            const int rc = launch_lora_down(p.M, p.T, p.r, !TRANSPOSED, p.In, p.Ldown, p.Pout, st);
+            if (rc != QLORA_OK) return rc;
+        }
     }
     // one cluster of p.split CTAs per tile when the contraction is split
     return launch_pdl(kern, dim3((unsigned)grid), dim3(kThreads), smem_bytes, st, (unsigned)p.split, ta, tq, ts, tz, p) == cudaSuccess
                ? QLORA_OK : QLORA_ERR_CUDA;
 }
 
-#include "lora_down_stream.cuh"
 #include "umma_pair.cuh"
 #include "skinny_kernel.cuh"
 
@@ -672,7 +760,7 @@ bool umma_supported(const qlora_desc& d, int M) {
 // CTA-pair kernel: 512 tokens x 256 weight rows per pair of SMs.  Used when there are more than 256 tokens.
 // One counter pair per key (the caller's workspace address), handed out on first sight and kept: two launches that can
 // overlap in time have different workspaces, hence different pairs.  -1 when the table is full.
-static int sync_slot_for(const void* key) {
+int sync_slot_for(const void* key) {
     static std::mutex mu;
     static std::unordered_map<const void*, int> table;
     std::lock_guard<std::mutex> lock(mu);
@@ -769,10 +857,6 @@ int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In
                      const void* zeros, const void* L, float* Pmat, void* Out, cudaStream_t st, const void* Ldown,
                      const void* sync_key) {
     if (M > 256) return launch_umma_pair(d, M, transposed, In, Q, scales, zeros, L, Pmat, Out, st, Ldown, sync_key);
-    if (Ldown != nullptr && d.r > 0) {
-        const int rc = launch_lora_down(M, transposed ? d.N : d.K, d.r, !transposed, In, Ldown, Pmat, st);
-        if (rc != QLORA_OK) return rc;
-    }
     Params p{};
     p.M = M; p.N = d.N; p.K = d.K; p.bits = d.bits; p.g = d.group_size; p.r = d.r; p.r_pad = (d.r + 15) / 16 * 16;
     p.C = transposed ? d.K : d.N;
@@ -832,9 +916,12 @@ int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In
     }
     p.steps /= p.split;
     const int grid = p.split > 1 ? p.n_tiles * p.split : (p.n_tiles < sm_count() ? p.n_tiles : sm_count());
+    p.T = T; p.In = (const __nv_bfloat16*)In; p.Ldown = (const __nv_bfloat16*)Ldown; p.Pout = Pmat;
+    p.lds_stages = (int)((p.off_bar - LDS_BAR_BYTES) / LDS_STAGE_BYTES);
+    if (p.lds_stages > 6) p.lds_stages = 6;
 #define QLORA_LAUNCH(B)                                                                              \
-    return transposed ? launch_impl<B, true>(ta, tq, ts, tz, p, smem_bytes, grid, st)                \
-                      : launch_impl<B, false>(ta, tq, ts, tz, p, smem_bytes, grid, st)
+    return transposed ? launch_impl<B, true>(ta, tq, ts, tz, p, smem_bytes, grid, st, Ldown, sync_key)  \
+                      : launch_impl<B, false>(ta, tq, ts, tz, p, smem_bytes, grid, st, Ldown, sync_key)
     switch (d.bits) {
         case 2: QLORA_LAUNCH(2);
         case 3: QLORA_LAUNCH(3);

@@ -47,25 +47,6 @@ struct PairParams {
     float* Pout;
 };
 
-// Bounded wait until a counter in global memory reaches `target` (written by other CTAs of the same launch).
-__device__ __forceinline__ bool wait_counter(const unsigned* ctr, unsigned target, volatile int* abort_flag) {
-    uint64_t t0 = 0;
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        unsigned v;
-        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
-        if (v >= target) return true;
-        __nanosleep(256);
-        if ((i & 63u) == 63u) {
-            if (*abort_flag) return false;
-            const uint64_t now = global_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) break;
-        }
-    }
-    *abort_flag = 1;
-    atomicOr(&g_device_status, 1u);
-    return false;
-}
 
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
