@@ -29,7 +29,7 @@ constexpr size_t lds_smem_bytes(int stages) { return (size_t)stages * LDS_STAGE_
 constexpr int LDS_MIN_STAGES = (LDS_CWARPS * LDS_MAXB * 2 * 128 * 4 + LDS_STAGE_BYTES - 1) / LDS_STAGE_BYTES;   // room for the reduction
 
 // Row blocks first_block, first_block + block_stride, ... (at most LDS_MAXB of them below ceil(M / 16)).
-// Called by all 480 threads of the CTA; `smem` is 128-byte aligned with room for lds_smem_bytes(stages), stages >=
+// Called by all threads of the CTA (15 warps or more; the first 15 work); `smem` is 128-byte aligned with room for lds_smem_bytes(stages), stages >=
 // LDS_MIN_STAGES.  Returns with no copy in flight (every issued stage has been waited for) unless the kernel is aborting.
 template <bool L_IS_A, int NT>
 __device__ __forceinline__ void lora_down_stream(int M, int T, int r, const __nv_bfloat16* __restrict__ In,
@@ -84,8 +84,8 @@ __device__ __forceinline__ void lora_down_stream(int M, int T, int r, const __nv
                 if (++slot == (uint32_t)stages) { slot = 0; phase ^= 1u; }
             }
         }
-    } else {
-        // ---------------------------------------------------------------- consumers
+    } else if (warp < LDS_CWARPS) {
+        // ---------------------------------------------------------------- consumers (warps beyond the issuer's have no part)
         uint32_t slot = 0, phase = 0;
         const uint4 zero4 = make_uint4(0, 0, 0, 0);
         bool live = true;

@@ -231,9 +231,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     const uint32_t S = (uint32_t)p.S, P = (uint32_t)p.P;
 
     // barrier addresses
-    const uint32_t bar_full_x = smem0 + p.off_bar;          // [S]  activation tile landed (TMA)
-    const uint32_t bar_full_w = bar_full_x + 8 * S;         // [S]  weight tile written by one dequant group
-    const uint32_t bar_empty = bar_full_w + 8 * S;          // [S]  MMAs reading the stage have completed
+    const uint32_t bar_full_x = smem0 + p.off_bar;          // [S]  stage full: activation tile landed (TMA) and weight tile
+    const uint32_t bar_full_w = bar_full_x;                 //      written by one dequant group (one wait for the MMA issuer)
+    const uint32_t bar_empty = bar_full_x + 8 * S;          // [S]  MMAs reading the stage have completed
     const uint32_t bar_full_p = bar_empty + 8 * S;          // [P]  packed words + group parameters landed (TMA)
     const uint32_t bar_empty_p = bar_full_p + 8 * P;        // [P]  the dequant group has read them into registers
     const uint32_t bar_acc_full = bar_empty_p + 8 * P;      // [2]  accumulator buffer complete
@@ -243,8 +243,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     if (threadIdx.x == 0) {
         abort_flag_s = 0;
         for (uint32_t i = 0; i < S; ++i) {
-            mbar_init(bar_full_x + 8 * i, 1);
-            mbar_init(bar_full_w + 8 * i, kGroupWarps);
+            mbar_init(bar_full_x + 8 * i, 1 + kGroupWarps);
             mbar_init(bar_empty + 8 * i, 1);
         }
         for (uint32_t i = 0; i < P; ++i) {
@@ -351,7 +350,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                 uint32_t acc = 0;
                 for (int step = 0; step < p.steps; ++step) {
                     if (!mbar_wait(bar_full_x + 8 * ring.slot, ring.phase, abort_flag)) goto done;
-                    if (!mbar_wait(bar_full_w + 8 * ring.slot, ring.phase, abort_flag)) goto done;
                     tc_fence_after();
                     const uint64_t b_desc = b_desc0 + ring.slot * x_step;
                     const uint64_t a_desc = a_desc0 + ring.slot * (uint32_t)(kWStageBytes >> 4);

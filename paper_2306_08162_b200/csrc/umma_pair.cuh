@@ -130,9 +130,12 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     const int first_tile = (int)(blockIdx.x >> 1) - p.n_prod, tile_stride = (int)(gridDim.x >> 1) - p.n_prod;
 
     // barriers (same offsets in both CTAs)
-    const uint32_t bar_full_x = smem0 + p.off_bar;          // [S] leader's: activation sub-tiles of both CTAs landed (TMA)
-    const uint32_t bar_full_w = bar_full_x + 8 * S;         // [S] leader's: weight tiles of both CTAs written
-    const uint32_t bar_empty = bar_full_w + 8 * S;          // [S] both: MMAs reading the stage have completed (multicast commit)
+    // One "stage full" barrier per slot collects both operand streams -- the TMA bytes of both CTAs' activation sub-tiles
+    // (one expect_tx arrival) and the arrivals of both CTAs' dequant warps: the MMA-issuing thread's per-stage work (eight
+    // tcgen05.mma, one wait, one commit) is what paces the main loop, and a second wait per stage cost 4 % of the kernel.
+    const uint32_t bar_full_x = smem0 + p.off_bar;          // [S] leader's: activation sub-tiles landed (TMA) + weight tiles written
+    const uint32_t bar_full_w = bar_full_x;                 //     (the same barriers: dequant warps arrive on them)
+    const uint32_t bar_empty = bar_full_x + 8 * S;          // [S] both: MMAs reading the stage have completed (multicast commit)
     const uint32_t bar_full_p = bar_empty + 8 * S;          // [P] local: packed words + group parameters landed (TMA)
     const uint32_t bar_empty_p = bar_full_p + 8 * P;        // [P] local: the dequant group has read them into registers
     const uint32_t bar_acc_full = bar_empty_p + 8 * P;      // [1] both: accumulators complete (multicast commit)
@@ -142,8 +145,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     if (threadIdx.x == 0) {
         abort_flag_s = 0;
         for (uint32_t i = 0; i < S; ++i) {
-            mbar_init(bar_full_x + 8 * i, 1);
-            mbar_init(bar_full_w + 8 * i, 2 * kGroupWarps);
+            mbar_init(bar_full_x + 8 * i, 1 + 2 * kGroupWarps);
             mbar_init(bar_empty + 8 * i, 1);
         }
         for (uint32_t i = 0; i < P; ++i) {
@@ -238,8 +240,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                 tc_fence_after();
                 uint32_t acc = 0;
                 for (int step = 0; step < p.steps; ++step) {
-                    if (!mbar_wait(bar_full_x + 8 * ring.slot, ring.phase, abort_flag)) goto done;
-                    if (!mbar_wait_cluster(bar_full_w + 8 * ring.slot, ring.phase, abort_flag)) goto done;
+                    if (!mbar_wait_cluster(bar_full_x + 8 * ring.slot, ring.phase, abort_flag)) goto done;
                     tc_fence_after();
                     const uint64_t a_desc = a_desc0 + ring.slot * (uint32_t)(kPairXStage >> 4);
                     const uint64_t b_desc = b_desc0 + ring.slot * (uint32_t)(kWStageBytes >> 4);
