@@ -167,6 +167,11 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t ran
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+__device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t cluster_addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(cluster_addr) : "memory");
+    return v;
+}
 __device__ __forceinline__ float ld_cluster_f32(uint32_t cluster_addr) {
     float v;
     asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr) : "memory");
@@ -554,12 +559,20 @@ done:
             const int w0 = wt * kWRows, m0 = tt * p.BT;
             const int tok_per_rank = p.BT / p.split;
             const uint32_t part_addr = smem0;
-            for (int e = threadIdx.x; e < tok_per_rank * kWRows; e += kThreads) {
-                const int t = rank * tok_per_rank + e / kWRows, cw = e % kWRows;
-                float v = 0.f;
-                for (int rk = 0; rk < p.split; ++rk)
-                    v += ld_cluster_f32(map_to_cta(part_addr, (uint32_t)rk) + (uint32_t)((t * kWRows + cw) * 4));
-                if (m0 + t < p.M && w0 + cw < p.C) p.Out[(size_t)(m0 + t) * p.C + w0 + cw] = __float2bfloat16_rn(v);
+            uint32_t peer[4];
+            for (int rk = 0; rk < 4; ++rk) peer[rk] = map_to_cta(part_addr, (uint32_t)(rk < p.split ? rk : 0));
+            for (int e = threadIdx.x; e < tok_per_rank * (kWRows / 4); e += kThreads) {   // four weight rows (output columns) at a time
+                const int t = rank * tok_per_rank + e / (kWRows / 4), cw = (e % (kWRows / 4)) * 4;
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int rk = 0; rk < p.split; ++rk) {
+                    const float4 x = ld_cluster_f32x4(peer[rk] + (uint32_t)((t * kWRows + cw) * 4));
+                    v.x += x.x; v.y += x.y; v.z += x.z; v.w += x.w;
+                }
+                if (m0 + t < p.M && w0 + cw < p.C) {     // C is a multiple of 8: four columns are all-in or all-out
+                    const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+                    *reinterpret_cast<uint2*>(p.Out + (size_t)(m0 + t) * p.C + w0 + cw) =
+                        make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+                }
             }
         }
         __syncwarp();
