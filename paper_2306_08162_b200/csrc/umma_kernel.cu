@@ -119,6 +119,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // Whole-warp wait: lane 0 polls (so a waiting warp costs one lane's issue slots), the outcome is broadcast, and every
 // lane then observes the completed phase itself before touching the data the barrier guards.
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int lane) {
+    if (__all_sync(0xFFFFFFFFu, mbar_try_wait(bar, parity) != 0u)) return true;   // already complete: one instruction per lane
     uint32_t ok = 1;
     if (lane == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1u : 0u;
     ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
