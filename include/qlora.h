@@ -30,6 +30,10 @@
  *     descriptor is a HOST pointer.  The library allocates no device memory, keeps no per-call state and never
  *     frees anything.  Q, scales, zeros, A, B are read-only (theta_q is frozen and there is no gradient for it;
  *     Section 3.1).
+ *     Because they are read-only for every call of the library, a call may start loading Q, scales, zeros, A and B
+ *     while the library's own preceding call in the stream is still finishing (programmatic dependent launch); it waits
+ *     for that call before it touches activations, H / G or outputs.  Work of other origin in the stream (a kernel
+ *     that repacks Q or updates A / B) is always complete before a call starts.
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = the legacy default stream) of
  *     the current device.  No call synchronises the device; outputs are valid in stream order.
  *   - Calls given the same workspace must be ordered one after the other (same stream, or events): they share

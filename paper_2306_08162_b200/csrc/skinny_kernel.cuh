@@ -103,6 +103,7 @@ __device__ __forceinline__ void sk_producer(const SkinnyParams& p, const CUtenso
                                             uint32_t bar_empty, int c0, int mrow0, int rank, int lane, volatile int* abort_flag) {
     const int slot = lane >> 2, job = lane & 3;
     if (slot >= p.S || job == 3 || (job == 2 && NTL == 0)) return;
+    if (job == 1) pdl_wait();                                            // the activations may come from the preceding kernel
     int it = slot;                                                       // this CTA's it-th stage
     for (int st = rank + SK_SPLIT * slot; st < p.stages_total; st += SK_SPLIT * p.S, it += p.S) {
         const uint32_t lap = (uint32_t)(it / p.S);
@@ -201,8 +202,9 @@ __device__ __forceinline__ void sk_cluster_epilogue(const SkinnyParams& p, uint3
         for (int i = 0; i < p.S; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, SK_WARPS / 2); } \
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");                                          \
     }                                                                                                               \
-    __syncthreads();                                                                                                \
-    pdl_wait();   /* set-up done; from here on global memory is touched */
+    __syncthreads();   /* set-up done.  The frozen weights and the adapters are read-only for every call of the library, so  \
+                          their loads start at once; whatever the preceding work in the stream may have produced (the      \
+                          activations, P) or may still be reading (the outputs) is touched only after pdl_wait().  */
 
 // After the main loop: every consumer warp has read every stage this CTA loaded, so no TMA write is still to come and
 // the ring's memory can hold the partial tiles; then the cluster reduces them.  On an abort nothing is stored.
@@ -211,6 +213,7 @@ __device__ __forceinline__ void sk_cluster_epilogue(const SkinnyParams& p, uint3
     if (*abort_flag) for (int i = 0; i < 200; ++i) __nanosleep(1000);   /* let copies in flight land */               \
     __syncwarp();                                                                                                   \
     cluster_sync_all();                    /* all eight partial tiles are written */                                \
+    pdl_wait();                            /* P may come from, and Out may still be read by, the preceding kernel */ \
     if (!*abort_flag) sk_cluster_epilogue<TRANSPOSED_, NTL>(p, smem0, ps, c0, mrow0, rank);                          \
     __syncwarp();                                                                                                   \
     cluster_sync_all();                    /* nobody leaves while a peer may still read its partial tile */

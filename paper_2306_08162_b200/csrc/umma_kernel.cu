@@ -271,7 +271,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
-    pdl_wait();   // set-up done; from here on global memory is touched
+    // Set-up done.  The frozen weights are read-only for every call of the library, so their producer starts at once; the
+    // roles that touch what the preceding work in the stream may have produced (activations, P) or may still be reading
+    // (the output) call pdl_wait() first.
 
     // Few tokens give few tiles: the contraction of a tile is then split over a cluster of p.split CTAs (rank i takes steps
     // i * p.steps ...), each accumulates its part in tensor memory, and the parts are added through distributed shared
@@ -284,6 +286,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         // ------------------------------------------------------------------ producer cluster: LoRA down-projection on SMs
         // the tiles leave idle (one CTA per row block or more; lowest block indices, so they wait for nobody)
         const int n_ctas = p.n_prod * p.split;
+        pdl_wait();
         if (p.r <= 8) lora_down_stream<!TRANSPOSED, 1>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, n_ctas, smem_gen, p.lds_stages, abort_flag);
         else          lora_down_stream<!TRANSPOSED, 2>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, n_ctas, smem_gen, p.lds_stages, abort_flag);
         __threadfence();       // every thread's rows of P are visible device-wide before the CTA is counted
@@ -292,6 +295,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     } else if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer: activation tiles
         if (lane == 0) {
+            pdl_wait();
             Ring ring;
             for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride) {
                 const int m0 = (tile % p.n_tok_tiles) * p.BT;
@@ -384,6 +388,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         // ------------------------------------------------------------------ epilogue (+ LoRA operand staging)
         const int q = warp & 3;                      // tensor-memory lane quarter this warp may read
         const int et = threadIdx.x - kEpiWarp0 * 32; // 0..127
+        pdl_wait();
         uint32_t tile_it = 0;
         for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride, ++tile_it) {
             const int wt = tile / p.n_tok_tiles, tt = tile % p.n_tok_tiles;
@@ -555,6 +560,7 @@ done:
         // Add the ranks' parts in rank order (fixed order: deterministic); rank i finishes tokens i * BT / split ...
         __syncwarp();
         cluster_sync_all();
+        pdl_wait();            // every thread stores part of the output below
         if (!*abort_flag && first_tile >= 0 && first_tile < p.n_tiles) {
             const int wt = first_tile / p.n_tok_tiles, tt = first_tile % p.n_tok_tiles;
             const int w0 = wt * kWRows, m0 = tt * p.BT;

@@ -166,11 +166,13 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     cluster_sync_all();        // the peer's barriers are initialised before anything arrives on them
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
-    pdl_wait();                // set-up done; from here on global memory is touched
+    // Set-up done.  The weight producer starts at once (the frozen weights are read-only for every call of the library);
+    // the roles that touch activations, P or the output call pdl_wait() first.
 
     if (first_tile < 0) {
         // ------------------------------------------------------------------ producer cluster: LoRA down-projection
         // (this CTA's row blocks: blockIdx.x, blockIdx.x + 2 n_prod, ...; the ring takes the operand area, below the barriers)
+        pdl_wait();
         if (p.r <= 8) lora_down_stream<!TRANSPOSED, 1>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, 2 * p.n_prod, smem_gen, p.lds_stages, abort_flag);
         else          lora_down_stream<!TRANSPOSED, 2>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, 2 * p.n_prod, smem_gen, p.lds_stages, abort_flag);
         __threadfence();       // every thread's rows of P are visible device-wide before the CTA is counted
@@ -179,6 +181,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     } else if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer: activation sub-tiles
         if (lane == 0) {
+            pdl_wait();
             Ring ring;
             const uint32_t leader_full_x = map_to_cta(bar_full_x, 0);
             for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride) {
@@ -275,6 +278,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         const int et = threadIdx.x - kEpiWarp0 * 32; // 0..127
         const uint32_t leader_acc_empty = map_to_cta(bar_acc_empty, 0);
         const uint32_t leader_lora_full = map_to_cta(bar_lora_full, 0);
+        pdl_wait();
         uint32_t tile_it = 0;
         for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride, ++tile_it) {
             const int wt = tile / p.n_tok_tiles, tt = tile % p.n_tok_tiles;
