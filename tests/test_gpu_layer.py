@@ -303,6 +303,13 @@ def test_down_projection_has_the_same_bits_inside_the_kernel_and_as_a_launch(M, 
     assert torch.equal(saved["dA"], recomputed["dA"]) and torch.equal(saved["dB"], recomputed["dB"])
 
 
+def test_many_tokens_narrow_layer():
+    """20000 tokens through a narrow layer: 40 token tiles of the pair kernel on a single column tile, and a down-projection
+    launch with more 16-row blocks (1250) than one wave of CTAs holds (148 x 8), so its grid goes over several waves."""
+    layer = qi.random_codes_layer(K=256, N=128, bits=4, group_size=64, r=8, alpha=16.0, M=20000, seed=23)
+    check_layer(layer)
+
+
 def test_accumulate_adds_to_existing_gradients():
     layer = qi.random_codes_layer(K=256, N=256, bits=4, group_size=128, r=8, alpha=16.0, M=96, seed=4)
     gl = GpuLayer(layer)
