@@ -46,6 +46,7 @@ struct SkinnyParams {
     uint32_t off_p, off_bar;
     float s;
     const __nv_bfloat16* Lup;    // B [N, r] (forward) or A [r, K] (backward): the adapter applied second
+    const __nv_bfloat16* Ldown;  // A [r, K] (forward) or B [N, r] (backward): the adapter applied first (fused ranks only)
     float* P;                    // H / G fp32 [M, r]: written by one CTA when fused, read otherwise
     int p_is_input;
     __nv_bfloat16* Out;
@@ -102,7 +103,7 @@ __device__ __forceinline__ void sk_producer(const SkinnyParams& p, const CUtenso
                                             const CUtensorMap* tact, const CUtensorMap* tl, uint32_t smem0, uint32_t bar_full,
                                             uint32_t bar_empty, int c0, int mrow0, int rank, int lane, volatile int* abort_flag) {
     const int slot = lane >> 2, job = lane & 3;
-    if (slot >= p.S || job == 3 || (job == 2 && NTL == 0)) return;
+    if (slot >= p.S || job == 3 || (job == 2 && (NTL == 0 || !TRANSPOSED))) return;   // (forward: the consumers read A themselves)
     if (job == 1) pdl_wait();                                            // the activations may come from the preceding kernel
     int it = slot;                                                       // this CTA's it-th stage
     for (int st = rank + SK_SPLIT * slot; st < p.stages_total; st += SK_SPLIT * p.S, it += p.S) {
@@ -112,7 +113,7 @@ __device__ __forceinline__ void sk_producer(const SkinnyParams& p, const CUtenso
         const uint32_t bar = bar_full + 8 * slot;
         const int t0 = st * SK_STAGE;                                   // first contraction index of the stage
         if (job == 0) {
-            mbar_expect_tx(bar, p.words_bytes + 2 * p.scale_bytes + p.act_bytes + (NTL > 0 ? p.l_bytes : 0u));
+            mbar_expect_tx(bar, p.words_bytes + 2 * p.scale_bytes + p.act_bytes + (NTL > 0 && TRANSPOSED ? p.l_bytes : 0u));
             if (!TRANSPOSED) {   // c0 = first output column n; packed rows walk K
                 tma_load_2d(dst, tq, bar, c0, st * (SK_STAGE / 32) * p.bits);
                 tma_load_2d(dst + p.off_scale, ts, bar, c0, t0 / p.g);
@@ -127,13 +128,7 @@ __device__ __forceinline__ void sk_producer(const SkinnyParams& p, const CUtenso
             for (int sb = 0; sb < SK_STAGE / 64; ++sb)                   // 16 token rows x 64 contraction elements per box
                 tma_load_2d(dst + p.off_act + sb * 2048, tact, bar, t0 + 64 * sb, mrow0);
         } else {
-            if (!TRANSPOSED) {
-#pragma unroll
-                for (int sb = 0; sb < SK_STAGE / 64; ++sb)               // A[0 .. 8 NTL) x 64 k per box
-                    tma_load_2d(dst + p.off_l + sb * (1024 * NTL), tl, bar, t0 + 64 * sb, 0);
-            } else {
-                tma_load_2d(dst + p.off_l, tl, bar, 0, t0);             // B[n, 0 .. r) for the stage's 256 n
-            }
+            tma_load_2d(dst + p.off_l, tl, bar, 0, t0);                 // backward: B[n, 0 .. r) for the stage's 256 n
         }
     }
 }
@@ -146,40 +141,67 @@ __device__ __forceinline__ void sk_cluster_epilogue(const SkinnyParams& p, uint3
     uint32_t peer[SK_SPLIT];
 #pragma unroll
     for (int rk = 0; rk < SK_SPLIT; ++rk) peer[rk] = map_to_cta(part_addr, (uint32_t)rk);
+    // This thread's output element (threads 0 .. 511), its row of the second adapter (requested first, so that the global
+    // loads are in flight during the reductions) and its sum over the partial tiles.
+    const bool has_out = tid < 16 * 32;
+    const int m = tid >> 5, c = tid & 31;
+    const int row = mrow0 + m, col = c0 + 32 * rank + c;
+    const bool live = has_out && row < p.M && col < p.C;
+    float lup[8 * (NTL > 0 ? NTL : 1)];
     if constexpr (NTL > 0) {
-        for (int e = tid; e < 16 * 8 * NTL; e += SK_THREADS) {
-            const int m = e / (8 * NTL), j = e % (8 * NTL);
-            float v = 0.f;
 #pragma unroll
-            for (int rk = 0; rk < SK_SPLIT; ++rk)
+        for (int j = 0; j < 8 * NTL; ++j) lup[j] = 0.f;
+        if (live) {
+            if (!TRANSPOSED) {        // B[n, 0 .. r): 16 bytes per eight ranks (backward: A[j, k] is strided, read below)
 #pragma unroll
-                for (int h = 0; h < SK_PLANES; ++h) v += ld_cluster_f32(peer[rk] + (uint32_t)(((h * 16 + m) * SK_PW + SK_TILE + j) * 4));
-            ps[m * 16 + j] = v;
-            if (blockIdx.y == 0 && rank == 0 && mrow0 + m < p.M && j < p.r) p.P[(size_t)(mrow0 + m) * p.r + j] = v;
+                for (int lt = 0; lt < NTL; ++lt)
+                    if (lt * 8 < p.r) {
+                        const uint4 b = __ldg(reinterpret_cast<const uint4*>(p.Lup + (size_t)col * p.r + lt * 8));
+                        lup[lt * 8 + 0] = bf16_lo(b.x); lup[lt * 8 + 1] = bf16_hi(b.x); lup[lt * 8 + 2] = bf16_lo(b.y); lup[lt * 8 + 3] = bf16_hi(b.y);
+                        lup[lt * 8 + 4] = bf16_lo(b.z); lup[lt * 8 + 5] = bf16_hi(b.z); lup[lt * 8 + 6] = bf16_lo(b.w); lup[lt * 8 + 7] = bf16_hi(b.w);
+                    }
+            }
         }
-        __syncthreads();
     }
-    for (int e = tid; e < 16 * 32; e += SK_THREADS) {
-        const int m = e >> 5, c = e & 31;
-        const int row = mrow0 + m, col = c0 + 32 * rank + c;
-        float v = 0.f;
+    float v = 0.f;
+    if (has_out) {
 #pragma unroll
         for (int rk = 0; rk < SK_SPLIT; ++rk)
 #pragma unroll
             for (int h = 0; h < SK_PLANES; ++h) v += ld_cluster_f32(peer[rk] + (uint32_t)(((h * 16 + m) * SK_PW + 32 * rank + c) * 4));
-        if (row >= p.M || col >= p.C) continue;
-        if (p.r > 0) {
-            float lo = 0.f;
+    }
+    if constexpr (NTL > 0) {
+        for (int e = tid; e < 16 * 8 * NTL; e += SK_THREADS) {
+            const int mm = e / (8 * NTL), j = e % (8 * NTL);
+            float h = 0.f;
+#pragma unroll
+            for (int rk = 0; rk < SK_SPLIT; ++rk)
+#pragma unroll
+                for (int pl = 0; pl < SK_PLANES; ++pl) h += ld_cluster_f32(peer[rk] + (uint32_t)(((pl * 16 + mm) * SK_PW + SK_TILE + j) * 4));
+            ps[mm * 16 + j] = h;
+            if (blockIdx.y == 0 && rank == 0 && mrow0 + mm < p.M && j < p.r) p.P[(size_t)(mrow0 + mm) * p.r + j] = h;
+        }
+        __syncthreads();
+    }
+    if (!live) return;
+    if (p.r > 0) {
+        float lo = 0.f;
+        if constexpr (NTL > 0 && !TRANSPOSED) {
+#pragma unroll
+            for (int j = 0; j < 8 * NTL; ++j) lo = fmaf(ps[m * 16 + j], lup[j], lo);     // ranks beyond r: zero times zero
+        } else if constexpr (NTL > 0) {
+            for (int j = 0; j < p.r; ++j) lo = fmaf(ps[m * 16 + j], __bfloat162float(p.Lup[(size_t)j * p.K + col]), lo);   // A[j, k]
+        } else {
             for (int j = 0; j < p.r; ++j) {
-                const float pj = NTL > 0 ? ps[m * 16 + j] : __ldg(p.P + (size_t)row * p.r + j);
+                const float pj = __ldg(p.P + (size_t)row * p.r + j);
                 const float l = TRANSPOSED ? __bfloat162float(p.Lup[(size_t)j * p.K + col])     // A[j, k]
                                            : __bfloat162float(p.Lup[(size_t)col * p.r + j]);    // B[n, j]
                 lo = fmaf(pj, l, lo);
             }
-            v += p.s * lo;
         }
-        p.Out[(size_t)row * p.C + col] = __float2bfloat16_rn(v);
+        v += p.s * lo;
     }
+    p.Out[(size_t)row * p.C + col] = __float2bfloat16_rn(v);
 }
 
 #define SK_COMMON_PROLOGUE()                                                                                         \
@@ -236,6 +258,20 @@ skinny_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const int blk = 4 * kh + q;                               // this lane's 32-code block inside the stage
         for (int it = sh, st = rank + SK_SPLIT * sh; st < p.stages_total; st += 2 * SK_SPLIT, it += 2) {
             const uint32_t slot = (uint32_t)(it % p.S), lap = (uint32_t)(it / p.S);
+            // the fused H tile (computed once per cluster column block): this lane's A fragments -- rank lt * 8 + g, its 32 k
+            // -- come straight from global memory (A is small, read-only and shared by every CTA, so it sits in L2),
+            // requested before the wait for the stage, which hides their latency
+            uint4 la[NTL > 0 ? NTL : 1][4];
+            if (NTL > 0 && cg == 0) {
+                const int k0 = st * SK_STAGE + 32 * blk;
+#pragma unroll
+                for (int lt = 0; lt < NTL; ++lt)
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj)
+                        la[lt][jj] = (lt * 8 + g < p.r && k0 + 8 * jj < p.K)
+                                         ? __ldg(reinterpret_cast<const uint4*>(p.Ldown + (size_t)(lt * 8 + g) * p.K + k0 + 8 * jj))
+                                         : make_uint4(0, 0, 0, 0);
+            }
             if (!warp_wait(bar_full + 8 * slot, lap & 1u, abort_flag, lane)) break;
             const uint8_t* stg = smem_gen + slot * p.stage_bytes;
             uint4 w4[BITS];
@@ -254,15 +290,6 @@ skinny_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 const int off = (((4 * (blk & 1) + jj) ^ g) << 4);
                 xa[jj] = *reinterpret_cast<const uint4*>(xrow + off);
                 xb[jj] = *reinterpret_cast<const uint4*>(xrow + 1024 + off);
-            }
-            uint4 la[NTL > 0 ? NTL : 1][4];
-            if (NTL > 0 && cg == 0) {                             // the fused H tile: computed once per cluster column block
-#pragma unroll
-                for (int lt = 0; lt < NTL; ++lt) {
-                    const uint8_t* arow = stg + p.off_l + (blk >> 1) * (1024 * NTL) + (lt * 8 + g) * 128;
-#pragma unroll
-                    for (int jj = 0; jj < 4; ++jj) la[lt][jj] = *reinterpret_cast<const uint4*>(arow + (((4 * (blk & 1) + jj) ^ g) << 4));
-                }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty + 8 * slot);

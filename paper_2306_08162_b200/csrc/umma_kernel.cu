@@ -732,6 +732,7 @@ int launch_skinny_gemm(const qlora_desc& d, int M, bool transposed, const void* 
     const size_t smem_bytes = (size_t)p.off_bar + 2 * 8 * SK_MAX_STAGES + 1024;
     p.s = d.r > 0 ? d.alpha / (float)d.r : 0.f;
     p.Lup = (const __nv_bfloat16*)Lup;
+    p.Ldown = (const __nv_bfloat16*)Ldown;
     p.P = P; p.p_is_input = p_is_input ? 1 : 0; p.Out = (__nv_bfloat16*)Out;
 
     CUtensorMap tq, ts, tz, ta, tl;
