@@ -510,13 +510,13 @@ def mid_kernel_computes_p(M: int, C: int, T: int, r: int, sms: int = 148) -> boo
 def launches_per_step(M: int, r: int, K: int, N: int) -> int:
     """Kernels the library launches for one fwd + bwd_input + bwd_lora (H, G saved).  Each of fwd and bwd_input is a
     down-projection launch plus the dequant-GEMM, or the dequant-GEMM alone where it computes H / G itself (up to 32
-    tokens with r <= 16; above that where the tiles leave SMs idle).  The gradients are a partial-sum and a reduction
-    launch."""
+    tokens with r <= 16; above that where the tiles leave SMs idle).  The gradients are one launch up to 256 tokens (the row
+    slices of a column block form a cluster and reduce through distributed shared memory), else two."""
     if r == 0:
         return 2
     fwd = 1 if (M <= 32 and r <= 16) or pair_kernel_computes_p(M, N, r) or mid_kernel_computes_p(M, N, K, r) else 2
     bwd = 1 if (M <= 32 and r <= 16) or pair_kernel_computes_p(M, K, r) or mid_kernel_computes_p(M, K, N, r) else 2
-    return fwd + bwd + 2
+    return fwd + bwd + (1 if M <= 256 else 2)       # gradients: one clustered launch up to 256 tokens
 
 
 def main():
