@@ -430,7 +430,7 @@ def run_ours(args):
             "cpu_baseline": {"value": cpu["value"], "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": cpu["sample"]},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
-            "gpu_launches": launches_per_step(M, r, K, N) * args.steps,
+            "gpu_launches": launches_per_step(M, r, K, N, w["bits"]) * args.steps,
             "clocks": clocks,
         }
         print(json.dumps(line))
@@ -493,12 +493,13 @@ def pair_kernel_computes_p(M: int, C: int, r: int, sms: int = 148) -> bool:
 
 
 def mid_kernel_computes_p(M: int, C: int, T: int, r: int, sms: int = 148) -> bool:
-    """Mirror of the dispatch for 33..256 tokens: tiles of 128 output columns, the contraction split over clusters of 4 or
+    """Mirror of the dispatch for the single-CTA tensor-core kernel (17..256 tokens; all counts up to 256 with 8-bit
+    weights): tiles of 128 output columns, the contraction split over clusters of 4 or
     2 CTAs when that still fits the GPU; producer clusters are added while the GPU can hold more clusters of that width
     (33 of width 4, 74 of width 2) and two row blocks of 16 tokens per producer CTA cover the batch."""
-    if not (32 < M <= 256) or r == 0 or r > 16:
+    if M > 256 or r == 0 or r > 16:
         return False
-    tiles, steps, bt = -(-C // 128), T // 64, (256 if M > 128 else 128 if M > 64 else 64)
+    tiles, steps, bt = -(-C // 128), T // 64, (256 if M > 128 else 128 if M > 64 else 64 if M > 32 else 32)
     split = next((sp for sp in (4, 2) if tiles * sp <= sms and steps % sp == 0 and steps // sp >= 4 and bt % sp == 0), 1)
     clusters = tiles if split > 1 else min(tiles, sms)
     idle = {1: sms, 2: sms // 2, 4: 33}[split] - clusters
@@ -507,15 +508,16 @@ def mid_kernel_computes_p(M: int, C: int, T: int, r: int, sms: int = 148) -> boo
     return n_prod > 0 and n_prod * split * 2 >= blocks
 
 
-def launches_per_step(M: int, r: int, K: int, N: int) -> int:
+def launches_per_step(M: int, r: int, K: int, N: int, bits: int = 4) -> int:
     """Kernels the library launches for one fwd + bwd_input + bwd_lora (H, G saved).  Each of fwd and bwd_input is a
-    down-projection launch plus the dequant-GEMM, or the dequant-GEMM alone where it computes H / G itself (up to 32
-    tokens with r <= 16; above that where the tiles leave SMs idle).  The gradients are one launch up to 256 tokens (the row
+    down-projection launch plus the dequant-GEMM, or the dequant-GEMM alone where it computes H / G itself (the streaming
+    kernels with r <= 16; above that where the tiles leave SMs idle).  The gradients are one launch up to 256 tokens (the row
     slices of a column block form a cluster and reduce through distributed shared memory), else two."""
     if r == 0:
         return 2
-    fwd = 1 if (M <= 32 and r <= 16) or pair_kernel_computes_p(M, N, r) or mid_kernel_computes_p(M, N, K, r) else 2
-    bwd = 1 if (M <= 32 and r <= 16) or pair_kernel_computes_p(M, K, r) or mid_kernel_computes_p(M, K, N, r) else 2
+    streaming = M <= 16 and bits != 8          # (shapes the tensor-core kernels tile; the bench's all are)
+    fwd = 1 if (streaming and r <= 16) or pair_kernel_computes_p(M, N, r) or (not streaming and mid_kernel_computes_p(M, N, K, r)) else 2
+    bwd = 1 if (streaming and r <= 16) or pair_kernel_computes_p(M, K, r) or (not streaming and mid_kernel_computes_p(M, K, N, r)) else 2
     return fwd + bwd + (1 if M <= 256 else 2)       # gradients: one clustered launch up to 256 tokens
 
 

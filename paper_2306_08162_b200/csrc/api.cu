@@ -34,6 +34,13 @@ int check_desc(const qlora_desc* d, bool need_lora) {
     return QLORA_OK;
 }
 
+// Up to 16 tokens (one 16-row MMA tile) the streaming kernels are the fastest form for 2-, 3- and 4-bit weights; from 17
+// to 32 tokens they would stream the weights twice, and with 8-bit weights their unpacking is the slower one (measured
+// 16.3 against 13.5 us at one token), so there the tensor-core kernel takes over wherever it tiles the shape.
+bool use_streaming(const qlora_desc& d, int M) {
+    return skinny_supported(d, M) && !((M > 16 || d.bits == 8) && umma_supported(d, M));
+}
+
 struct Workspace {
     size_t p0_off, p1_off, grad_off, total;
 };
@@ -152,7 +159,7 @@ static int fwd_common(const qlora_desc* desc, int M, const void* X, const uint8_
     if (workspace == nullptr || workspace_bytes < w.total) return QLORA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     float* H = H_out ? H_out : reinterpret_cast<float*>(static_cast<char*>(workspace) + w.p0_off);
-    if (skinny_supported(d, M)) {
+    if (use_streaming(d, M)) {
         const bool fused = d.r > 0 && d.r <= 16 && mask == nullptr;   // the down-projection rides along inside the kernel
         if (d.r > 0 && !fused) {
             rc = launch_lora_down(M, d.K, d.r, true, X, A, H, st, mask, keep_scale);
@@ -194,13 +201,13 @@ static int bwd_input_common(const qlora_desc* desc, int M, const void* dY, const
         if (rc != QLORA_OK) return rc;
         qlora_desc d0 = d;
         d0.r = 0;
-        if (skinny_supported(d0, M)) rc = launch_skinny_gemm(d0, M, true, dY, Q, scales, zeros, B, A, G, true, dX, st);
+        if (use_streaming(d0, M)) rc = launch_skinny_gemm(d0, M, true, dY, Q, scales, zeros, B, A, G, true, dX, st);
         else if (umma_supported(d0, M)) rc = launch_umma_gemm(d0, M, true, dY, Q, scales, zeros, A, G, dX, st);
         else rc = launch_simt_gemm(d0, M, true, dY, Q, scales, zeros, A, G, dX, st);
         if (rc != QLORA_OK) return rc;
         return launch_lora_masked_update(M, d.K, d.r, keep_scale * d.alpha / (float)d.r, G, A, mask, dX, st);
     }
-    if (skinny_supported(d, M)) {
+    if (use_streaming(d, M)) {
         const bool fused = d.r > 0 && d.r <= 16;
         if (d.r > 0 && !fused) {
             rc = launch_lora_down(M, d.N, d.r, false, dY, B, G, st);
