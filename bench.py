@@ -483,12 +483,14 @@ def run_loss(args):
 
 def pair_kernel_computes_p(M: int, C: int, r: int, sms: int = 148) -> bool:
     """Mirror of the library's dispatch: above 256 tokens the CTA-pair kernel runs the LoRA down-projection on SM pairs
-    its tiles (512 tokens x 256 of the C output columns) leave idle, when there are enough of them."""
+    that have less to do than the rest -- no tile (512 tokens x 256 of the C output columns) at all, or one tile fewer
+    because the last wave is partly filled -- when there are enough of them."""
     if M <= 256 or r == 0 or r > 16:
         return False
-    tiles = -(-M // 512) * -(-C // 256)
+    tiles, pairs = -(-M // 512) * -(-C // 256), sms // 2
+    idle = pairs - tiles if tiles < pairs else (pairs - tiles % pairs if tiles % pairs else 0)
     blocks = -(-M // 16)
-    n_prod = min(sms // 2 - tiles, -(-blocks // 4))
+    n_prod = min(idle, -(-blocks // 4))
     return n_prod > 0 and n_prod * 16 >= blocks
 
 

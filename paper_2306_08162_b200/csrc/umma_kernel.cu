@@ -845,7 +845,8 @@ static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const v
     if (p.lds_stages > 6) p.lds_stages = 6;
     if (Ldown != nullptr && d.r > 0) {
         const int n_blocks = (M + 15) / 16;
-        const int idle = pairs - p.n_tiles;
+        // pairs with less to do: no tile at all, or one tile fewer than the rest when the last wave is partly filled
+        const int idle = p.n_tiles < pairs ? pairs - p.n_tiles : (p.n_tiles % pairs ? pairs - p.n_tiles % pairs : 0);
         int n_prod = (n_blocks + 3) / 4;                     // four row blocks per producer CTA pair when there is room
         if (n_prod > idle) n_prod = idle;
         const bool fits = d.r <= 16 && n_prod > 0 && n_prod * 2 * LDS_MAXB >= n_blocks && p.lds_stages >= LDS_MIN_STAGES;
@@ -858,7 +859,7 @@ static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const v
             if (rc != QLORA_OK) return rc;
         }
     }
-    const int grid = 2 * ((p.n_tiles < pairs ? p.n_tiles : pairs) + p.n_prod);
+    const int grid = 2 * (p.n_tiles < pairs ? p.n_tiles + p.n_prod : pairs);
 #define QLORA_LAUNCH_PAIR(B)                                                                              \
     return transposed ? launch_pair_impl<B, true>(ta, tq, ts, tz, p, smem_bytes, grid, st)                \
                       : launch_pair_impl<B, false>(ta, tq, ts, tz, p, smem_bytes, grid, st)

@@ -16,10 +16,11 @@
 // (stage free, accumulators complete) exist in both and are signalled by one multicast tcgen05.commit.
 // Every wait is bounded, as in the single-CTA kernel; the CTAs leave together through a cluster barrier.
 //
-// When the tiles leave SM pairs idle (fewer tiles than pairs), the launch can add `n_prod` producer clusters in front of
-// the tile clusters (lowest block indices, so they are dispatched first and wait for nobody): their CTAs compute the LoRA
-// down-projection P = In * Ldown (lora_down_stream.cuh) beside the main loops and publish it through a counter in device
-// memory; a tile's epilogue warps wait for that counter before they stage P for the LoRA update, which is only needed
+// When some SM pairs have less to do than others -- no tile at all (fewer tiles than pairs), or one tile fewer than the
+// rest (the last wave is partly filled) -- `n_prod` of them are producers: the first clusters of the grid (lowest block
+// indices, so they are dispatched first and wait for nobody) first compute the LoRA down-projection P = In * Ldown
+// (lora_down_stream.cuh) beside the others' main loops, publish it through a counter in device memory, and then take
+// their own (fewer) tiles; a tile's epilogue warps wait for that counter before they stage P for the LoRA update, which is only needed
 // once the tile's contraction is through.  The counter pair belongs to one launch at a time (the host hands out one
 // pair per workspace) and the last CTA to have seen the count zeroes it again.
 
@@ -127,7 +128,12 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t S = (uint32_t)p.S, P = (uint32_t)p.P;
     const uint32_t cta = cluster_ctarank();            // 0 = leader (issues the MMAs), 1 = follower
-    const int first_tile = (int)(blockIdx.x >> 1) - p.n_prod, tile_stride = (int)(gridDim.x >> 1) - p.n_prod;
+    // Work distribution: the launch has `tile_stride` worker pairs; worker w takes tiles w, w + tile_stride, ...  The first
+    // n_prod clusters of the grid are producers (down-projection first, see above) and take the HIGHEST worker indices,
+    // i.e. the workers with the fewest tiles -- none at all when the tiles do not fill a wave.
+    const int tile_stride = (int)(gridDim.x >> 1);
+    const bool is_producer = (int)(blockIdx.x >> 1) < p.n_prod;
+    const int first_tile = is_producer ? tile_stride - 1 - (int)(blockIdx.x >> 1) : (int)(blockIdx.x >> 1) - p.n_prod;
 
     // barriers (same offsets in both CTAs)
     // One "stage full" barrier per slot collects both operand streams -- the TMA bytes of both CTAs' activation sub-tiles
@@ -169,8 +175,8 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     // Set-up done.  The weight producer starts at once (the frozen weights are read-only for every call of the library);
     // the roles that touch activations, P or the output call pdl_wait() first.
 
-    if (first_tile < 0) {
-        // ------------------------------------------------------------------ producer cluster: LoRA down-projection
+    if (is_producer) {
+        // ------------------------------------------------------------------ producer cluster: LoRA down-projection first
         // (this CTA's row blocks: blockIdx.x, blockIdx.x + 2 n_prod, ...; the ring takes the operand area, below the barriers)
         pdl_wait();
         if (p.r <= 8) lora_down_stream<!TRANSPOSED, 1>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, 2 * p.n_prod, smem_gen, p.lds_stages, abort_flag);
@@ -178,7 +184,10 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         __threadfence();       // every thread's rows of P are visible device-wide before the CTA is counted
         __syncthreads();
         if (threadIdx.x == 0) atomicAdd(&g_pair_sync[p.slot][0], 1u);
-    } else if (warp == 0) {
+        fence_proxy_async();   // the shared memory just used goes to the TMA / tensor-core side for this cluster's tiles, if any
+        __syncthreads();
+    }
+    if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer: activation sub-tiles
         if (lane == 0) {
             pdl_wait();
@@ -288,7 +297,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                 // P is being computed by the producer clusters of this launch: one thread waits for all of their CTAs, is
                 // counted as done with the counter, and the last such CTA of the launch zeroes the pair for the next one.
                 if (et == 0 && wait_counter(&g_pair_sync[p.slot][0], 2u * (unsigned)p.n_prod, abort_flag)) {
-                    const unsigned n_cons = gridDim.x - 2u * (unsigned)p.n_prod;
+                    const unsigned n_cons = 2u * (unsigned)(p.n_tiles < tile_stride ? p.n_tiles : tile_stride);   // CTAs that have a tile
                     if (atomicAdd(&g_pair_sync[p.slot][1], 1u) == n_cons - 1u) {
                         atomicExch(&g_pair_sync[p.slot][0], 0u);
                         atomicExch(&g_pair_sync[p.slot][1], 0u);
