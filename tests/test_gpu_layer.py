@@ -292,11 +292,12 @@ def test_recompute_h_g_matches_saved():
     assert torch.equal(saved["dA"], recomputed["dA"]) and torch.equal(saved["dB"], recomputed["dB"])
 
 
-@pytest.mark.parametrize("M,K,N,r", [(600, 512, 512, 8), (1000, 2112, 320, 16), (300, 1024, 11008, 8)])
+@pytest.mark.parametrize("M,K,N,r", [(600, 512, 512, 8), (1000, 2112, 320, 16), (300, 1024, 11008, 8), (1024, 256, 10240, 8)])
 def test_down_projection_has_the_same_bits_inside_the_kernel_and_as_a_launch(M, K, N, r):
     """Above 256 tokens H / G come from the tensor-core kernel's producer clusters when its tiles leave SM pairs idle and
     from a stand-alone launch otherwise (here: the recomputation inside qlora_bwd_lora).  The streaming code sums in an
-    order that depends on the contraction length only, so saved and recomputed H / G give bitwise the same gradients."""
+    order that depends on the contraction length only, so saved and recomputed H / G give bitwise the same gradients.
+    (Last case: 80 forward tiles on 74 pairs, so the producers are pairs with one tile fewer that take tiles afterwards.)"""
     layer = qi.random_codes_layer(K=K, N=N, bits=4, group_size=64, r=r, alpha=2.0 * r, M=M, seed=17)
     _, saved, gl = check_layer(layer, save_hg=True)
     recomputed = gl.run(save_hg=False)
