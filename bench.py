@@ -64,7 +64,7 @@ KERNELS_PER_STEP = None           # filled from the library's dispatch (see laun
 
 # DRAM traffic (read + write) per launch of the dominant kernel of the default workload, from the ncu capture
 # summarised in profiles/umma_pair_config2_int4_m2048.md.  Set back to None whenever that kernel changes.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 26.02e6
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 26.01e6
 
 
 def layer_flops(M, K, N, r):
