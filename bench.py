@@ -482,10 +482,10 @@ def run_loss(args):
 
 
 def pair_kernel_computes_p(M: int, C: int, r: int, sms: int = 148) -> bool:
-    """Mirror of the library's dispatch: above 256 tokens the CTA-pair kernel runs the LoRA down-projection on SM pairs
+    """Mirror of the library's dispatch: above 768 tokens the CTA-pair kernel runs the LoRA down-projection on SM pairs
     that have less to do than the rest -- no tile (512 tokens x 256 of the C output columns) at all, or one tile fewer
     because the last wave is partly filled -- when there are enough of them."""
-    if M <= 256 or r == 0 or r > 16:
+    if M <= 768 or r == 0 or r > 16:
         return False
     tiles, pairs = -(-M // 512) * -(-C // 256), sms // 2
     idle = pairs - tiles if tiles < pairs else (pairs - tiles % pairs if tiles % pairs else 0)
@@ -495,13 +495,13 @@ def pair_kernel_computes_p(M: int, C: int, r: int, sms: int = 148) -> bool:
 
 
 def mid_kernel_computes_p(M: int, C: int, T: int, r: int, sms: int = 148) -> bool:
-    """Mirror of the dispatch for the single-CTA tensor-core kernel (17..256 tokens; all counts up to 256 with 8-bit
+    """Mirror of the dispatch for the single-CTA tensor-core kernel (17..768 tokens; from one token with 8-bit
     weights): tiles of 128 output columns, the contraction split over clusters of 4 or
     2 CTAs when that still fits the GPU; producer clusters are added while the GPU can hold more clusters of that width
     (33 of width 4, 74 of width 2) and two row blocks of 16 tokens per producer CTA cover the batch."""
-    if M > 256 or r == 0 or r > 16:
+    if M > 768 or r == 0 or r > 16:
         return False
-    tiles, steps, bt = -(-C // 128), T // 64, (256 if M > 128 else 128 if M > 64 else 64 if M > 32 else 32)
+    tiles, steps, bt = -(-C // 128) * max(1, -(-M // 256)), T // 64, (256 if M > 128 else 128 if M > 64 else 64 if M > 32 else 32)
     split = next((sp for sp in (4, 2) if tiles * sp <= sms and steps % sp == 0 and steps // sp >= 4 and bt % sp == 0), 1)
     clusters = tiles if split > 1 else min(tiles, sms)
     idle = {1: sms, 2: sms // 2, 4: 33}[split] - clusters

@@ -40,6 +40,7 @@ int sync_slot_for(const void* key);   // host: the counter pair of a workspace a
 namespace {
 
 constexpr int kThreads = 480;
+constexpr int kPairMinTokens = 768;                  // the CTA-pair kernel takes over above this many tokens
 constexpr int kDequantWarp0 = 7, kGroupWarps = 4;   // two dequant groups of four warps
 constexpr int kEpiWarp0 = 3, kEpiWarps = 4;
 constexpr int kWRows = 128;          // weight rows (MMA M) per tile: n in forward, k in backward
@@ -776,7 +777,7 @@ bool umma_supported(const qlora_desc& d, int M) {
     return true;
 }
 
-// CTA-pair kernel: 512 tokens x 256 weight rows per pair of SMs.  Used when there are more than 256 tokens.
+// CTA-pair kernel: 512 tokens x 256 weight rows per pair of SMs.  Used when there are more than kPairMinTokens tokens.
 // One counter pair per key (the caller's workspace address), handed out on first sight and kept: two launches that can
 // overlap in time have different workspaces, hence different pairs.  -1 when the table is full.
 int sync_slot_for(const void* key) {
@@ -876,7 +877,9 @@ static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const v
 int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
                      const void* zeros, const void* L, float* Pmat, void* Out, cudaStream_t st, const void* Ldown,
                      const void* sync_key) {
-    if (M > 256) return launch_umma_pair(d, M, transposed, In, Q, scales, zeros, L, Pmat, Out, st, Ldown, sync_key);
+    // Up to 768 tokens the tiles of the CTA-pair kernel (512 tokens x 256 weight rows) leave most SM pairs without one;
+    // the single-CTA kernel's smaller tiles (and split contraction) are faster there (23 against 42 us at 512 tokens).
+    if (M > kPairMinTokens) return launch_umma_pair(d, M, transposed, In, Q, scales, zeros, L, Pmat, Out, st, Ldown, sync_key);
     Params p{};
     p.M = M; p.N = d.N; p.K = d.K; p.bits = d.bits; p.g = d.group_size; p.r = d.r; p.r_pad = (d.r + 15) / 16 * 16;
     p.C = transposed ? d.K : d.N;
