@@ -481,11 +481,27 @@ def run_loss(args):
     return 0
 
 
-def pair_kernel_computes_p(M: int, C: int, r: int, sms: int = 148) -> bool:
-    """Mirror of the library's dispatch: above 768 tokens the CTA-pair kernel runs the LoRA down-projection on SM pairs
+def prefer_pair_kernel(M: int, C: int, T: int, sms: int = 148) -> bool:
+    """Mirror of the library's choice between its two tensor-core kernels (the cost model in csrc/umma_kernel.cu)."""
+    if M <= 256:
+        return False
+    if M > 1024:
+        return True
+    steps = T // 64
+    tiles_mid = -(-M // 256) * -(-C // 128)
+    split = next((sp for sp in (4, 2) if tiles_mid * sp <= sms and steps % sp == 0 and steps // sp >= 4), 1)
+    waves_mid = 1 if split > 1 else -(-tiles_mid // sms)
+    mid_us = waves_mid * ((steps // split) * 0.29 + 15.0)
+    tiles_pair = -(-M // 512) * -(-C // 256)
+    pair_us = -(-tiles_pair // (sms // 2)) * (steps * 0.62 + 4.0)
+    return pair_us < mid_us
+
+
+def pair_kernel_computes_p(M: int, C: int, T: int, r: int, sms: int = 148) -> bool:
+    """Mirror of the library's dispatch: the CTA-pair kernel (where prefer_pair_kernel picks it) runs the LoRA down-projection on SM pairs
     that have less to do than the rest -- no tile (512 tokens x 256 of the C output columns) at all, or one tile fewer
     because the last wave is partly filled -- when there are enough of them."""
-    if M <= 768 or r == 0 or r > 16:
+    if not prefer_pair_kernel(M, C, T, sms) or r == 0 or r > 16:
         return False
     tiles, pairs = -(-M // 512) * -(-C // 256), sms // 2
     idle = pairs - tiles if tiles < pairs else (pairs - tiles % pairs if tiles % pairs else 0)
@@ -495,11 +511,11 @@ def pair_kernel_computes_p(M: int, C: int, r: int, sms: int = 148) -> bool:
 
 
 def mid_kernel_computes_p(M: int, C: int, T: int, r: int, sms: int = 148) -> bool:
-    """Mirror of the dispatch for the single-CTA tensor-core kernel (17..768 tokens; from one token with 8-bit
-    weights): tiles of 128 output columns, the contraction split over clusters of 4 or
+    """Mirror of the dispatch for the single-CTA tensor-core kernel (from 17 tokens, or one with 8-bit weights, up to
+    where prefer_pair_kernel picks the other): tiles of 128 output columns, the contraction split over clusters of 4 or
     2 CTAs when that still fits the GPU; producer clusters are added while the GPU can hold more clusters of that width
     (33 of width 4, 74 of width 2) and two row blocks of 16 tokens per producer CTA cover the batch."""
-    if M > 768 or r == 0 or r > 16:
+    if prefer_pair_kernel(M, C, T, sms) or r == 0 or r > 16:
         return False
     tiles, steps, bt = -(-C // 128) * max(1, -(-M // 256)), T // 64, (256 if M > 128 else 128 if M > 64 else 64 if M > 32 else 32)
     split = next((sp for sp in (4, 2) if tiles * sp <= sms and steps % sp == 0 and steps // sp >= 4 and bt % sp == 0), 1)
@@ -518,8 +534,8 @@ def launches_per_step(M: int, r: int, K: int, N: int, bits: int = 4) -> int:
     if r == 0:
         return 2
     streaming = M <= 16 and bits != 8          # (shapes the tensor-core kernels tile; the bench's all are)
-    fwd = 1 if (streaming and r <= 16) or pair_kernel_computes_p(M, N, r) or (not streaming and mid_kernel_computes_p(M, N, K, r)) else 2
-    bwd = 1 if (streaming and r <= 16) or pair_kernel_computes_p(M, K, r) or (not streaming and mid_kernel_computes_p(M, K, N, r)) else 2
+    fwd = 1 if (streaming and r <= 16) or pair_kernel_computes_p(M, N, K, r) or (not streaming and mid_kernel_computes_p(M, N, K, r)) else 2
+    bwd = 1 if (streaming and r <= 16) or pair_kernel_computes_p(M, K, N, r) or (not streaming and mid_kernel_computes_p(M, K, N, r)) else 2
     return fwd + bwd + (1 if M <= 256 else 2)       # gradients: one clustered launch up to 256 tokens
 
 

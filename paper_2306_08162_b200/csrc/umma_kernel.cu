@@ -40,7 +40,6 @@ int sync_slot_for(const void* key);   // host: the counter pair of a workspace a
 namespace {
 
 constexpr int kThreads = 480;
-constexpr int kPairMinTokens = 768;                  // the CTA-pair kernel takes over above this many tokens
 constexpr int kDequantWarp0 = 7, kGroupWarps = 4;   // two dequant groups of four warps
 constexpr int kEpiWarp0 = 3, kEpiWarps = 4;
 constexpr int kWRows = 128;          // weight rows (MMA M) per tile: n in forward, k in backward
@@ -777,7 +776,7 @@ bool umma_supported(const qlora_desc& d, int M) {
     return true;
 }
 
-// CTA-pair kernel: 512 tokens x 256 weight rows per pair of SMs.  Used when there are more than kPairMinTokens tokens.
+// CTA-pair kernel: 512 tokens x 256 weight rows per pair of SMs (see prefer_pair_kernel for when it is used).
 // One counter pair per key (the caller's workspace address), handed out on first sight and kept: two launches that can
 // overlap in time have different workspaces, hence different pairs.  -1 when the table is full.
 int sync_slot_for(const void* key) {
@@ -874,12 +873,31 @@ static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const v
     return QLORA_ERR_UNSUPPORTED;
 }
 
+// Between 257 and 1024 tokens either tensor-core kernel may be the faster one: the pair kernel's tiles (512 tokens x 256
+// weight rows) leave most SM pairs without one on a 4096-wide layer (42 us against 23 at 512 tokens), but fill a wave
+// exactly where the single-CTA kernel's 128 x 256 tiles need two (11008 outputs: 45 against 68 us).  The choice follows
+// a small cost model fitted to measurements: waves of tiles times (steps x time per step + fixed part) for each kernel.
+static bool prefer_pair_kernel(const qlora_desc& d, int M, bool transposed) {
+    if (M <= 256) return false;
+    if (M > 1024) return true;
+    const int T = transposed ? d.N : d.K, C = transposed ? d.K : d.N;
+    const int steps = T / kStepC, sms = sm_count();
+    const int tiles_mid = ((M + 255) / 256) * ((C + kWRows - 1) / kWRows);
+    int split = 1;
+    for (int sp = 4; sp >= 2; sp /= 2)
+        if (tiles_mid * sp <= sms && steps % sp == 0 && steps / sp >= 4) { split = sp; break; }
+    const int waves_mid = split > 1 ? 1 : (tiles_mid + sms - 1) / sms;
+    const float mid_us = (float)waves_mid * ((float)(steps / split) * 0.29f + 15.0f);
+    const int tiles_pair = ((M + 4 * kPairTok - 1) / (4 * kPairTok)) * ((C + 2 * kPairW - 1) / (2 * kPairW));
+    const int waves_pair = (tiles_pair + sms / 2 - 1) / (sms / 2);
+    const float pair_us = (float)waves_pair * ((float)steps * 0.62f + 4.0f);
+    return pair_us < mid_us;
+}
+
 int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
                      const void* zeros, const void* L, float* Pmat, void* Out, cudaStream_t st, const void* Ldown,
                      const void* sync_key) {
-    // Up to 768 tokens the tiles of the CTA-pair kernel (512 tokens x 256 weight rows) leave most SM pairs without one;
-    // the single-CTA kernel's smaller tiles (and split contraction) are faster there (23 against 42 us at 512 tokens).
-    if (M > kPairMinTokens) return launch_umma_pair(d, M, transposed, In, Q, scales, zeros, L, Pmat, Out, st, Ldown, sync_key);
+    if (prefer_pair_kernel(d, M, transposed)) return launch_umma_pair(d, M, transposed, In, Q, scales, zeros, L, Pmat, Out, st, Ldown, sync_key);
     Params p{};
     p.M = M; p.N = d.N; p.K = d.K; p.bits = d.bits; p.g = d.group_size; p.r = d.r; p.r_pad = (d.r + 15) / 16 * 16;
     p.C = transposed ? d.K : d.N;
