@@ -311,6 +311,21 @@ def test_many_tokens_narrow_layer():
     check_layer(layer)
 
 
+@pytest.mark.parametrize("seed", range(24))
+def test_seeded_sweep_across_the_dispatch_boundaries(seed):
+    """Seeded random shapes around every switch of the dispatch (16 / 17, 32 / 33, 256 / 257, the cost-model range up to
+    1024, above it), all bit widths, ranks fused and not: each against the oracle."""
+    rng = np.random.default_rng(1234 + seed)
+    M = int(rng.choice([1, 9, 16, 17, 31, 32, 33, 100, 256, 257, 300, 512, 513, 700, 769, 1000, 1024, 1025, 1300]))
+    bits = int(rng.choice([2, 3, 4, 8]))
+    g = int(rng.choice([64, 128]))
+    K = int(rng.choice([128, 256, 384, 640, 1024, 2176]))
+    N = int(rng.choice([64, 128, 320, 704, 1536, 2752]))
+    r = int(rng.choice([0, 8, 16, 24]))
+    layer = qi.random_codes_layer(K=K, N=N, bits=bits, group_size=g, r=r, alpha=2.0 * max(r, 8), M=M, seed=100 + seed)
+    check_layer(layer)
+
+
 def test_accumulate_adds_to_existing_gradients():
     layer = qi.random_codes_layer(K=256, N=256, bits=4, group_size=128, r=8, alpha=16.0, M=96, seed=4)
     gl = GpuLayer(layer)
