@@ -21,6 +21,7 @@ library's definition):
 Pins (tests/test_oracle_*.py): pack/unpack against a big-integer bit-stream and hand-computed words;
 dequant against the closed form on every code value; forward/backward against brute-force loops,
 central finite differences, the adjoint identity and the B=0 / A=0 / q=zero special cases.
+quantize_rtn against hand-worked groups (incl. ties), the half-step error bound and its invariants.
 The choice of bit layout is "format unpinned by the paper" (no example is printed there).
 """
 from __future__ import annotations
@@ -119,6 +120,46 @@ def dequant_gidx(Q: np.ndarray, scales: np.ndarray, zeros: np.ndarray, bits: int
     s = np.asarray(scales, dtype=np.float16).astype(np.float64)[g_idx]   # [K, N]
     z = np.asarray(zeros, dtype=np.float16).astype(np.float64)[g_idx]
     return np.ascontiguousarray((s * (q - z)).T)
+
+
+def quantize_rtn(W: np.ndarray, bits: int, group_size: int):
+    """Asymmetric min-max round-to-nearest quantizer, the "RTN" baseline the paper's quantized models are
+    compared with and the way the benchmark configurations produce their codes ("asymmetric round-to-nearest
+    min-max", group size g along K).  W float32 [N, K]  ->  codes uint8 [K, N], scales fp16 [K/g, N],
+    zeros fp16 [K/g, N] (integer valued).
+
+    For every output row n and every group of g consecutive k (written out one group at a time):
+        lo = min(0, min w)          hi = max(0, max w)           qmax = 2^bits - 1
+        scale = fp16_rne((hi - lo) / qmax);  scale = 1 when that is 0
+        zero  = clamp(rint(-lo / scale), 0, qmax)
+        q[k]  = clamp(rint(w[k] / scale) + zero, 0, qmax)
+    rint rounds halves to even.  The codes are integers decided by floating-point arithmetic, so the
+    precision is part of the definition: float32 throughout, with the fp16-rounded scale, which is what
+    a GPU kernel computes in too (IEEE division and rint give the same bits on both sides).
+    """
+    W = np.asarray(W, dtype=np.float32)
+    N, K = W.shape
+    if K % group_size != 0:
+        raise ValueError("group_size must divide K")
+    qmax = np.float32((1 << bits) - 1)
+    zero32 = np.float32(0.0)
+    G = K // group_size
+    codes = np.empty((K, N), dtype=np.uint8)
+    scales = np.empty((G, N), dtype=np.float16)
+    zeros = np.empty((G, N), dtype=np.float16)
+    for gi in range(G):
+        w = W[:, gi * group_size:(gi + 1) * group_size]                # [N, g]
+        lo = np.minimum(w.min(axis=1), zero32)
+        hi = np.maximum(w.max(axis=1), zero32)
+        sc16 = ((hi - lo) / qmax).astype(np.float16)                   # one rounding, nearest even
+        sc16 = np.where(sc16 == np.float16(0.0), np.float16(1.0), sc16)
+        sc = sc16.astype(np.float32)
+        z = np.clip(np.rint((-lo) / sc), zero32, qmax)
+        q = np.clip(np.rint(w / sc[:, None]) + z[:, None], zero32, qmax)
+        codes[gi * group_size:(gi + 1) * group_size, :] = q.T.astype(np.uint8)
+        scales[gi, :] = sc16
+        zeros[gi, :] = z.astype(np.float16)
+    return codes, scales, zeros
 
 
 def round_to_bf16_bits(x: np.ndarray) -> np.ndarray:
