@@ -159,12 +159,13 @@ static int fwd_common(const qlora_desc* desc, int M, const void* X, const uint8_
     if (workspace == nullptr || workspace_bytes < w.total) return QLORA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     float* H = H_out ? H_out : reinterpret_cast<float*>(static_cast<char*>(workspace) + w.p0_off);
-    if (use_streaming(d, M)) {
+    if (stream_supported(d, M, false) || use_streaming(d, M)) {
         const bool fused = d.r > 0 && d.r <= 16 && mask == nullptr;   // the down-projection rides along inside the kernel
         if (d.r > 0 && !fused) {
             rc = launch_lora_down(M, d.K, d.r, true, X, A, H, st, mask, keep_scale);
             if (rc != QLORA_OK) return rc;
         }
+        if (stream_supported(d, M, false)) return launch_stream_gemm(d, M, false, X, Q, scales, zeros, A, B, H, !fused, Y, st);
         return launch_skinny_gemm(d, M, false, X, Q, scales, zeros, A, B, H, !fused, Y, st);
     }
     // the tensor-core path computes H itself when given A (beside its tiles where SM pairs are idle, else ahead of them)
@@ -201,18 +202,20 @@ static int bwd_input_common(const qlora_desc* desc, int M, const void* dY, const
         if (rc != QLORA_OK) return rc;
         qlora_desc d0 = d;
         d0.r = 0;
-        if (use_streaming(d0, M)) rc = launch_skinny_gemm(d0, M, true, dY, Q, scales, zeros, B, A, G, true, dX, st);
+        if (stream_supported(d0, M, true)) rc = launch_stream_gemm(d0, M, true, dY, Q, scales, zeros, B, A, G, true, dX, st);
+        else if (use_streaming(d0, M)) rc = launch_skinny_gemm(d0, M, true, dY, Q, scales, zeros, B, A, G, true, dX, st);
         else if (umma_supported(d0, M)) rc = launch_umma_gemm(d0, M, true, dY, Q, scales, zeros, A, G, dX, st);
         else rc = launch_simt_gemm(d0, M, true, dY, Q, scales, zeros, A, G, dX, st);
         if (rc != QLORA_OK) return rc;
         return launch_lora_masked_update(M, d.K, d.r, keep_scale * d.alpha / (float)d.r, G, A, mask, dX, st);
     }
-    if (use_streaming(d, M)) {
+    if (stream_supported(d, M, true) || use_streaming(d, M)) {
         const bool fused = d.r > 0 && d.r <= 16;
         if (d.r > 0 && !fused) {
             rc = launch_lora_down(M, d.N, d.r, false, dY, B, G, st);
             if (rc != QLORA_OK) return rc;
         }
+        if (stream_supported(d, M, true)) return launch_stream_gemm(d, M, true, dY, Q, scales, zeros, B, A, G, !fused, dX, st);
         return launch_skinny_gemm(d, M, true, dY, Q, scales, zeros, B, A, G, !fused, dX, st);
     }
     if (umma_supported(d, M)) return launch_umma_gemm(d, M, true, dY, Q, scales, zeros, A, G, dX, st, B, workspace);   // computes G

@@ -58,6 +58,12 @@ bool skinny_supported(const qlora_desc& d, int M);
 int launch_skinny_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
                        const void* zeros, const void* Ldown, const void* Lup, float* P, bool p_is_input, void* Out,
                        cudaStream_t st);
+// stream_kernel.cu -- few tokens (M <= 16): cp.async-fed mma.sync kernels on raw codes, the contraction split over a
+// cluster; same arguments as launch_skinny_gemm (the down-projection is computed inside for ranks up to 16).
+bool stream_supported(const qlora_desc& d, int M, bool transposed);
+int launch_stream_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
+                       const void* zeros, const void* Ldown, const void* Lup, float* P, bool p_is_input, void* Out,
+                       cudaStream_t st);
 int read_device_status(unsigned int* out, int clear);
 
 }  // namespace qlora
