@@ -62,8 +62,8 @@ def weight_bytes(w):
     return w["N"] * w["K"] * w["bits"] / 8 + 4 * w["N"] * w["K"] / w["group_size"]
 KERNELS_PER_STEP = None           # filled from the library's dispatch (see launches_per_step)
 
-# DRAM traffic (read + write) per launch of the dominant kernel of the default workload, from the ncu capture
-# summarised in profiles/umma_pair_config2_int4_m2048.md.  Set back to None whenever that kernel changes.
+# DRAM traffic (read + write) per launch of the dominant kernel of the default workload, from one ncu capture of that
+# kernel (dram__bytes_read.sum + dram__bytes_write.sum).  Set back to None whenever that kernel changes.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = 26.01e6
 
 

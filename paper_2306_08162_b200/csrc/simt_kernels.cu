@@ -47,9 +47,7 @@ simt_gemm_kernel(int bits, int g, int K, int N, int r, float s, int M, const __n
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int e = tid + i * 256;
-                int ti, ci;
-                if (TRANSPOSED) { ti = e / 64; ci = e % 64; }   // ti: n offset, ci: k offset (k fastest: same word for 8 lanes)
-                else            { ti = e / 64; ci = e % 64; }   // ti: k offset, ci: n offset (n fastest: coalesced words)
+                const int ti = e / 64, ci = e % 64;   // ti: contraction offset, ci: output offset (fastest across threads)
                 const int t = t0 + ti, c = c0 + ci;
                 float w = 0.f;
                 if (t < T && c < C) {

@@ -22,9 +22,11 @@
 //   - backward: the contraction runs across packed columns, so a fragment register needs two columns for one feature.
 //     Each lane builds pairs of features of its own column and the 8 x 8 tile is transposed across the warp with
 //     movmatrix: the register form of the transposition of the packed matrix (Section 3.1, "Implementation Details");
-//   - the contraction is split over a cluster of up to 8 CTAs; the partial tiles are added in rank order through
-//     distributed shared memory (CTA i owns a slice of the columns), so no workspace and no counters are needed and the
-//     result is the same on every run;
+//   - the contraction is split over a cluster of up to 8 CTAs, and inside a CTA over up to four sets of warps (sixteen
+//     warps per SM keep the schedulers busy).  CTA i of a cluster finishes a slice of the columns: every CTA stores its
+//     partial sums for that slice straight into i's shared memory (distributed shared memory; nothing waits on a remote
+//     store), one cluster barrier later i adds them in a fixed order.  No workspace, no counters, and the result is the
+//     same on every run;
 //   - the LoRA down-projection (H = X A^T, G = dY B) over the CTA's part of the contraction comes from a few MMAs fed
 //     straight from global memory (ranks up to 16), reduced with the partial tiles; the update s P L is added in the
 //     epilogue in fp32 before the one rounding to bf16.
@@ -49,7 +51,7 @@ struct Fmt {
     static constexpr int KB = BITS == 2 ? 64 : 32;
     static constexpr int ROWS = KB * BITS / 32;              // packed rows per stage: 4, 3, 4, 8
     static constexpr int SLOT = ROWS * 128 + 128;
-    static constexpr int NS = BITS == 8 ? 7 : (BITS == 3 ? 16 : 12);
+    static constexpr int NS = BITS == 8 ? 5 : 8;            // ring stages per warp: 4 - 5.6 KB in flight per warp
     static constexpr int STEPS = KB / 16;                    // k16 MMA steps per stage
     static constexpr int NPAIR = 2 * STEPS;                  // bf16 pairs per column and lane
     static constexpr int NLD = (BITS == 3 || BITS == 8) ? 2 : 1;
@@ -59,7 +61,7 @@ struct Fmt {
     static constexpr int BROWS = FW * BITS / 32;             // 1, 3, 4, 8
     static constexpr int SU = BITS == 2 ? 4 : 1;
     static constexpr int BSLOT = BROWS * 128 * SU;
-    static constexpr int BNS = BITS == 8 ? 8 : 16;
+    static constexpr int BNS = BITS == 8 ? 4 : 8;
     static constexpr int BPAIR = BITS == 2 ? 2 : 4;          // pairs per column and lane
 };
 
@@ -67,6 +69,9 @@ struct StreamParams {
     int M, K, N, g, r;
     int C;                       // output columns (N forward, K backward)
     int ks;                      // CTAs per cluster = ways the contraction is split
+    int wc;                      // warps side by side in a CTA (32 columns forward, FW features backward each)
+    int khs;                     // log2 of the parts the warps of a CTA split each staged slice of the contraction into
+    int sls;                     // log2 of the columns a CTA of the cluster finishes (32 wc / ks or FW wc / ks)
     int xc;                      // contraction elements of the activation slice staged per pass
     int copies;                  // backward: groups a CTA's features span (1 or 2)
     int fused;                   // H / G is computed here (ranks up to 16) and written to P; else P is an input
@@ -101,11 +106,6 @@ __device__ __forceinline__ uint32_t st_map(uint32_t addr, uint32_t rank) {
     uint32_t r;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
-}
-__device__ __forceinline__ float st_ld_cluster(uint32_t addr) {
-    float v;
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
-    return v;
 }
 __device__ __forceinline__ void st_cluster_sync() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -181,32 +181,56 @@ __device__ __forceinline__ float st_sum8(const uint4& v) {
     return ((bf16_lo(v.x) + bf16_hi(v.x)) + (bf16_lo(v.y) + bf16_hi(v.y))) + ((bf16_lo(v.z) + bf16_hi(v.z)) + (bf16_lo(v.w) + bf16_hi(v.w)));
 }
 
-// Epilogue shared by both directions.  part: [TOKS][tile_c + 4] fp32 partial tile of this CTA; hs: [16][16] partial H / G.
-// CTA `rank` adds the cluster's partial tiles in rank order for its slice of tile_c / ks columns, adds s P L and stores bf16.
+// ---- reduction across the cluster: push, barrier, add locally -------------------------------------------------------
+// The CTAs of a cluster hold partial tiles of the same output columns.  CTA `o` finishes the slice of tile_c / ks columns
+// [o sl, o sl + sl): every CTA stores its partial sums for those columns straight into o's shared memory (remote stores,
+// nothing waits on them), one cluster barrier later o adds what it received in a fixed order.  recv layout in the owner:
+//   recv_part [ks][KH][sl][16 tokens] fp32      recv_h [ks][16 ranks][16 tokens] fp32
+// Nobody reads a peer's shared memory, so a CTA may leave as soon as it has stored its own outputs.
+struct RecvLayout {
+    uint32_t part_addr, h_addr;   // shared-space addresses (the same in every CTA of the cluster)
+    int sls, khs;                 // log2 of the slice width and of the parts per CTA
+};
+
+__device__ __forceinline__ void st_push2(const RecvLayout& rl, int src_rank, int kh, int cl, int tok, float v0, float v1) {
+    const int owner = cl >> rl.sls, c = cl & ((1 << rl.sls) - 1);
+    const uint32_t off = (uint32_t)(((((src_rank << rl.khs) + kh) << rl.sls) + c) * 16 + tok) * 4u;
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(st_map(rl.part_addr + off, (uint32_t)owner)), "f"(v0), "f"(v1) : "memory");
+}
+
+// This CTA's part of H / G (hs [16][16]) goes to every CTA of the cluster.
+__device__ __forceinline__ void st_push_h(const RecvLayout& rl, const float* hs, int src_rank, int ks) {
+    for (int e = threadIdx.x; e < 256 * ks; e += blockDim.x) {
+        const int peer = e >> 8, i = e & 255;
+        asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(st_map(rl.h_addr + (uint32_t)(src_rank * 256 + i) * 4u, (uint32_t)peer)), "f"(hs[i]) : "memory");
+    }
+}
+
+__device__ __forceinline__ void st_cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
+__device__ __forceinline__ void st_cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
+// After the pushes: one cluster barrier, then the owner adds (source rank, part) in order, adds s P L, stores bf16.
 template <bool TRANSPOSED, int TOKS>
-__device__ __forceinline__ void st_epilogue(const StreamParams& p, float* part, float* hs, float* hfull, const __nv_bfloat16* lup,
-                                            int tile_c, int rank) {
+__device__ __forceinline__ void st_finish(const StreamParams& p, const float* recv_part, const float* recv_h, float* hfull,
+                                          const __nv_bfloat16* lup, int tile_c, int rank) {
     const int tid = threadIdx.x, nthr = blockDim.x;
-    const int pw = tile_c + 4;
-    const int sl = tile_c / p.ks;
-    st_cluster_sync();                                    // every CTA's partial tile (and partial H / G) is written
+    const int sl = tile_c / p.ks, KH = 1 << p.khs;
+    st_cluster_sync();                                    // every CTA's stores into this CTA's shared memory are visible
     if (p.r > 0 && p.fused) {
-        const uint32_t ha = s_u32(hs);
         for (int e = tid; e < 256; e += nthr) {
             float h = 0.f;
-            for (int rk = 0; rk < p.ks; ++rk) h += st_ld_cluster(st_map(ha + 4u * (uint32_t)e, (uint32_t)rk));
+            for (int rk = 0; rk < p.ks; ++rk) h += recv_h[rk * 256 + e];
             hfull[e] = h;
             const int j = e >> 4, tok = e & 15;
             if (blockIdx.y == 0 && rank == 0 && tok < p.M && j < p.r) p.P[(size_t)tok * p.r + j] = h;
         }
         __syncthreads();
     }
-    const uint32_t pa = s_u32(part);
-    for (int e = tid; e < TOKS * sl; e += nthr) {
-        const int tok = e / sl, c = e % sl;
-        const int cl = rank * sl + c, col = blockIdx.y * tile_c + cl;
+    for (int e = tid; e < sl * TOKS; e += nthr) {
+        const int tok = e % TOKS, c = e / TOKS;           // TOKS is a power of two
+        const int col = blockIdx.y * tile_c + rank * sl + c;
         float v = 0.f;
-        for (int rk = 0; rk < p.ks; ++rk) v += st_ld_cluster(st_map(pa + 4u * (uint32_t)(tok * pw + cl), (uint32_t)rk));
+        for (int i = 0; i < p.ks * KH; ++i) v += recv_part[(i * sl + c) * 16 + tok];
         if (tok >= p.M || col >= p.C) continue;
         if (p.r > 0) {
             float lo = 0.f;
@@ -220,7 +244,6 @@ __device__ __forceinline__ void st_epilogue(const StreamParams& p, float* part, 
         }
         p.Out[(size_t)tok * p.C + col] = __float2bfloat16_rn(v);
     }
-    st_cluster_sync();                                    // nobody leaves while a peer may still read its shared memory
 }
 
 // After griddepcontrol.wait: this CTA's slice of the second adapter (the columns it will finish) and, when H / G is an
@@ -248,97 +271,148 @@ __device__ __forceinline__ void st_stage_lup(const StreamParams& p, __nv_bfloat1
     }
 }
 
+// Before griddepcontrol.wait nothing but the frozen weights may be READ, but lines can be asked into L2 (the point of
+// coherence: a line the predecessor rewrites afterwards is simply updated there).  `rows` rows of `bytes` bytes each.
+__device__ __forceinline__ void st_prefetch_l2(const void* base, size_t row_pitch_bytes, int rows, int bytes, int first, int nthr) {
+    const int per_row = (bytes + 127) / 128;
+    for (int e = first; e < rows * per_row; e += nthr) {
+        const int rr = e / per_row, i = e - rr * per_row;
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(static_cast<const char*>(base) + (size_t)rr * row_pitch_bytes + (size_t)i * 128));
+    }
+}
+
+// A warp's partial H / G tile ([16 ranks][16 tokens], MMA accumulator layout) -> its slot of hp.
+template <int NT>
+__device__ __forceinline__ void st_store_hp(float (&ah)[NT][4], float* hp, int warp, int g, int q) {
+    float* mine = hp + warp * 256;
+#pragma unroll
+    for (int tt = 0; tt < 2; ++tt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            mine[(g + ((e & 2) ? 8 : 0)) * 16 + 8 * tt + 2 * q + (e & 1)] = tt < NT ? ah[tt < NT ? tt : 0][e] : 0.f;
+}
+
+// Part `kh` of `n` consecutive items split KH = 2^khs ways.
+__device__ __forceinline__ int st_part(int n, int kh, int khs) { return (n * kh) >> khs; }
+
 // ------------------------------------------------------------------------------------------------------------
-// Forward: Y = X W^T + s H B^T.  CTA (rank, tile): columns [32 W tile, +32 W) (warp w: 32 of them), contraction blocks
-// [kb0, kb1) of KB elements, all of them taken by every warp for its own columns.
+// Forward: Y = X W^T + s H B^T.  CTA (rank, tile): columns [32 wc tile, + 32 wc), contraction blocks [kb0, kb1) of KB
+// elements.  Warp (cg, kh): 32 columns, and part kh of the blocks of every staged activation slice.
 // ------------------------------------------------------------------------------------------------------------
+constexpr int ST_HSTEPS = 4;   // k16 steps of the fused down-projection whose operands a warp loads in one go
+
 template <int BITS, int NT>
-__global__ void __launch_bounds__(256, 2) stream_fwd_kernel(const StreamParams p) {
+__global__ void __launch_bounds__(512, 1) stream_fwd_kernel(const StreamParams p) {
     using F = Fmt<BITS>;
     constexpr int TOKS = 8 * NT;
     pdl_launch_dependents();
+    st_cluster_arrive_relaxed();                           // waited for before the first store into a peer's shared memory
     extern __shared__ __align__(128) uint8_t smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, q = lane & 3;
-    const int W = blockDim.x >> 5, tile_c = 32 * W;
+    const int nw = blockDim.x >> 5, tile_c = 32 * p.wc, KH = 1 << p.khs;
+    const int cg = warp % p.wc, kh = warp / p.wc;
     const int rank = (int)st_cluster_rank();
-    const int col0 = blockIdx.y * tile_c + 32 * warp;
+    const int col0 = blockIdx.y * tile_c + 32 * cg;
     const int nblk = (p.K + F::KB - 1) / F::KB;
     const int kb0 = nblk * rank / p.ks, kb1 = nblk * (rank + 1) / p.ks;
-    const int nit = kb1 - kb0;
     const int total_rows = p.K * BITS / 32;
     const int xp = p.xc * 2 + F::XPAD;
     const int xcb = p.xc / F::KB;                          // blocks per staged slice
+    const int bpg = p.g / F::KB;                           // blocks per group
+    const int sl = tile_c / p.ks;
     uint8_t* ring = smem + warp * (F::NS * F::SLOT);
-    uint8_t* xs = smem + W * (F::NS * F::SLOT);            // [TOKS][xp] permuted activation slice
+    uint8_t* xs = smem + nw * (F::NS * F::SLOT);           // [TOKS][xp] permuted activation slice
     float* sxc = reinterpret_cast<float*>(xs + TOKS * xp); // [TOKS][xc / 8] sums of 8 activations
-    float* sxs = sxc + TOKS * (p.xc / 8);                  // [xcb + 1][TOKS] sums per group segment of the slice
-    float* hs = sxs + (xcb + 1) * TOKS;                    // [16][16] this CTA's part of H
+    float* sxs = sxc + TOKS * (p.xc / 8);                  // [KH][xcb + 1][TOKS] sums per (part, group) segment of the slice
+    float* hs = sxs + KH * (xcb + 1) * TOKS;               // [16][16] this CTA's part of H
     float* hfull = hs + 256;                               // [r <= 64][16] the whole of H
     __nv_bfloat16* lup = reinterpret_cast<__nv_bfloat16*>(hfull + 1024);
-    float* part = reinterpret_cast<float*>(smem);          // reuses the rings after the main loop
-    float* hp = reinterpret_cast<float*>(xs);              // [W][16][16], before the first slice is staged
+    float* hp = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(lup) + ST_LUP_BYTES);   // [nw][16][16]
+    float* recv_h = hp + nw * 256;                         // [ks][16][16]
+    float* recv_part = recv_h + p.ks * 256;                // [ks][KH][sl][16]
+    RecvLayout rl;
+    rl.part_addr = s_u32(recv_part); rl.h_addr = s_u32(recv_h); rl.sls = p.sls; rl.khs = p.khs;
 
-    auto issue = [&](int it) {
-        if (it < nit) {
-            const int blk = kb0 + it;
-            const uint32_t dst = s_u32(ring + (it % F::NS) * F::SLOT);
+    // the copy engine's view of this warp's block sequence (it runs NS blocks ahead of the arithmetic)
+    int i_cb = kb0, i_blk = 0, i_end = 0, i_gpos = 0, i_slot = 0;
+    bool i_first = true, i_done = kb0 >= kb1;
+    auto i_enter = [&]() {                                 // position on this warp's part of slice i_cb (skipping empty parts)
+        while (!i_done) {
+            const int n = min(i_cb + xcb, kb1) - i_cb;
+            i_blk = i_cb + st_part(n, kh, p.khs);
+            i_end = i_cb + st_part(n, kh + 1, p.khs);
+            if (i_blk < i_end) { i_gpos = i_blk % bpg; i_first = true; return; }
+            i_cb += xcb;
+            if (i_cb >= kb1) i_done = true;
+        }
+    };
+    i_enter();
+    auto issue = [&]() {
+        if (!i_done) {
+            const uint32_t dst = s_u32(ring + i_slot * F::SLOT);
 #pragma unroll
             for (int h = 0; h < (F::ROWS + 3) / 4; ++h) {
                 const int row = 4 * h + (lane >> 3), ch = lane & 7;
                 if (row < F::ROWS) {
-                    const int grow = blk * F::ROWS + row, col = col0 + 4 * ch;
+                    const int grow = i_blk * F::ROWS + row, col = col0 + 4 * ch;
                     const bool ok = grow < total_rows && col < p.N;
                     cp16(dst + st_swz(row, ch), ok ? p.Q + (size_t)grow * p.N + col : p.Q, ok ? 16 : 0);
                 }
             }
-            const int k0 = blk * F::KB;
-            if ((k0 % p.g == 0 || it == 0) && lane < 8) {  // first block of a group in this CTA's range: its scales and zeros
+            if ((i_gpos == 0 || i_first) && lane < 8) {    // first block of a group in this part: its scales and zeros
                 const __half* base = lane < 4 ? p.scales : p.zeros;
                 const int col = col0 + 8 * (lane & 3);
                 const bool ok = col < p.N;
-                cp16(dst + F::ROWS * 128 + lane * 16, ok ? base + (size_t)(k0 / p.g) * p.N + col : base, ok ? 16 : 0);
+                cp16(dst + F::ROWS * 128 + lane * 16, ok ? base + (size_t)(i_blk / bpg) * p.N + col : base, ok ? 16 : 0);
+            }
+            i_first = false;
+            if (++i_gpos == bpg) i_gpos = 0;
+            if (++i_blk >= i_end) {
+                i_cb += xcb;
+                if (i_cb >= kb1) i_done = true; else i_enter();
             }
         }
+        if (++i_slot == F::NS) i_slot = 0;
         cp_commit();
     };
-    for (int it = 0; it < F::NS; ++it) issue(it);          // frozen weights only: in flight while the predecessor finishes
+#pragma unroll 1
+    for (int it = 0; it < F::NS; ++it) issue();            // frozen weights only: in flight while the predecessor finishes
+    {   // ask the lines this CTA will read right after the wait into L2: its slices of X, A and B
+        const int k_lo = kb0 * F::KB, kbytes = (min(kb1 * F::KB, p.K) - k_lo) * 2;
+        if (kbytes > 0) {
+            st_prefetch_l2(p.In + k_lo, (size_t)p.K * 2, p.M, kbytes, threadIdx.x, blockDim.x);
+            if (p.r > 0 && p.fused) st_prefetch_l2(p.Ldown + k_lo, (size_t)p.K * 2, p.r, kbytes, threadIdx.x, blockDim.x);
+        }
+        const int c_lo = blockIdx.y * tile_c + rank * sl;
+        if (p.r > 0 && c_lo < p.N) st_prefetch_l2(p.Lup + (size_t)c_lo * p.r, 0, 1, min(sl, p.N - c_lo) * p.r * 2, threadIdx.x, blockDim.x);
+    }
 
     pdl_wait();
 
-    // ---- LoRA: this CTA's part of H = X A^T (k16 steps dealt to the warps, operands straight from global memory) ----
-    st_stage_lup<false>(p, lup, hfull, tile_c, rank);
-    if (p.r > 0 && p.fused) {
-        float ah[NT][4];
+    // ---- LoRA: this CTA's part of H = X A^T (k16 steps dealt to the warps, operands straight from global memory); the
+    // loads of the first ST_HSTEPS steps are issued here and used once the activation slice is on its way too ----
+    const bool fused = p.r > 0 && p.fused;
+    const int h_k0 = kb0 * F::KB + 16 * warp, h_ke = min(kb1 * F::KB, p.K);
+    uint32_t ha[ST_HSTEPS][4], hb[ST_HSTEPS][NT][2];
+    auto h_load = [&](int kk) {
 #pragma unroll
-        for (int tt = 0; tt < NT; ++tt) ah[tt][0] = ah[tt][1] = ah[tt][2] = ah[tt][3] = 0.f;
-        const int ke = min(kb1 * F::KB, p.K);
-        for (int k0 = kb0 * F::KB + 16 * warp; k0 < ke; k0 += 16 * W) {
+        for (int h = 0; h < ST_HSTEPS; ++h) {
+            const int k0 = kk + 16 * nw * h;
+            const bool in = fused && k0 < h_ke;
             const __nv_bfloat16* a_lo = p.Ldown + (size_t)g * p.K + k0 + 2 * q;
             const __nv_bfloat16* a_hi = p.Ldown + (size_t)(g + 8) * p.K + k0 + 2 * q;
-            const uint32_t a0 = g < p.r ? ldg32(a_lo) : 0u, a2 = g < p.r ? ldg32(a_lo + 8) : 0u;
-            const uint32_t a1 = g + 8 < p.r ? ldg32(a_hi) : 0u, a3 = g + 8 < p.r ? ldg32(a_hi + 8) : 0u;
+            ha[h][0] = (in && g < p.r) ? ldg32(a_lo) : 0u; ha[h][2] = (in && g < p.r) ? ldg32(a_lo + 8) : 0u;
+            ha[h][1] = (in && g + 8 < p.r) ? ldg32(a_hi) : 0u; ha[h][3] = (in && g + 8 < p.r) ? ldg32(a_hi + 8) : 0u;
 #pragma unroll
             for (int tt = 0; tt < NT; ++tt) {
                 const int tok = g + 8 * tt;
                 const __nv_bfloat16* x = p.In + (size_t)tok * p.K + k0 + 2 * q;
-                const uint32_t b0 = tok < p.M ? ldg32(x) : 0u, b1 = tok < p.M ? ldg32(x + 8) : 0u;
-                st_mma(ah[tt], a0, a1, a2, a3, b0, b1);
+                hb[h][tt][0] = (in && tok < p.M) ? ldg32(x) : 0u; hb[h][tt][1] = (in && tok < p.M) ? ldg32(x + 8) : 0u;
             }
         }
-        float* mine = hp + warp * 256;
-#pragma unroll
-        for (int tt = 0; tt < 2; ++tt)
-#pragma unroll
-            for (int e = 0; e < 4; ++e)
-                mine[(g + ((e & 2) ? 8 : 0)) * 16 + 8 * tt + 2 * q + (e & 1)] = tt < NT ? ah[tt < NT ? tt : 0][e] : 0.f;
-        __syncthreads();
-        for (int e = threadIdx.x; e < 256; e += blockDim.x) {
-            float h = 0.f;
-            for (int w = 0; w < W; ++w) h += hp[w * 256 + e];
-            hs[e] = h;
-        }
-        __syncthreads();
-    }
+    };
+    if (fused) h_load(h_k0);
+    st_stage_lup<false>(p, lup, hfull, tile_c, rank);
 
     // ---- main loop ----
     float acc[2][NT][4], grp[2][NT][4];
@@ -349,52 +423,95 @@ __global__ void __launch_bounds__(256, 2) stream_fwd_kernel(const StreamParams p
 #pragma unroll
             for (int e = 0; e < 4; ++e) acc[u][tt][e] = grp[u][tt][e] = 0.f;
     float sc[4] = {0.f, 0.f, 0.f, 0.f}, cz[4] = {0.f, 0.f, 0.f, 0.f};   // this lane's four columns: scale, -scale (OFF + zero)
-    int it = 0;
+    int c_slot = 0;
+    if (kb0 >= kb1) st_cluster_wait();                     // (an empty range: the wait below is never reached)
     for (int cb = kb0; cb < kb1; cb += xcb) {
         const int ce = min(cb + xcb, kb1);
         const int k_lo = cb * F::KB, k_hi = min(ce * F::KB, p.K);
+        const int g_first = k_lo / p.g;
         // stage the activation slice [k_lo, k_hi): permuted for the fragment loads, plus the sums the zero-points need
         {
             constexpr int KP = BITS == 2 ? 16 : 8;
-            const int per_tok = (ce - cb) * F::KB / KP;
-            for (int e = threadIdx.x; e < TOKS * per_tok; e += blockDim.x) {
-                const int tok = e / per_tok, ci = e % per_tok;
-                const int k = k_lo + ci * KP;
-                uint4 v0 = make_uint4(0, 0, 0, 0), v1 = make_uint4(0, 0, 0, 0);
-                if (tok < p.M && k < p.K) {
-                    v0 = *reinterpret_cast<const uint4*>(p.In + (size_t)tok * p.K + k);
-                    if (KP == 16 && k + 8 < p.K) v1 = *reinterpret_cast<const uint4*>(p.In + (size_t)tok * p.K + k + 8);
+            constexpr int NB = BITS == 2 ? 2 : 4;          // items per round, their loads issued together
+            const int per_tok = (ce - cb) * F::KB / KP, n_items = TOKS * per_tok;
+            for (int e0 = threadIdx.x; e0 < n_items; e0 += NB * blockDim.x) {
+                uint4 v0[NB], v1[NB];
+                int tk[NB], ci[NB];
+#pragma unroll
+                for (int h = 0; h < NB; ++h) {
+                    const int e = e0 + h * blockDim.x;
+                    tk[h] = e / per_tok; ci[h] = e - tk[h] * per_tok;
+                    const int k = k_lo + ci[h] * KP;
+                    v0[h] = make_uint4(0, 0, 0, 0); v1[h] = make_uint4(0, 0, 0, 0);
+                    if (e < n_items && tk[h] < p.M && k < p.K) {
+                        v0[h] = *reinterpret_cast<const uint4*>(p.In + (size_t)tk[h] * p.K + k);
+                        if (KP == 16 && k + 8 < p.K) v1[h] = *reinterpret_cast<const uint4*>(p.In + (size_t)tk[h] * p.K + k + 8);
+                    }
                 }
-                uint8_t* dst = xs + tok * xp + ci * (2 * KP);
-                if constexpr (BITS == 2) {                 // (x0,x8) (x1,x9) ... (x7,x15)
-                    *reinterpret_cast<uint4*>(dst) = make_uint4(__byte_perm(v0.x, v1.x, 0x5410), __byte_perm(v0.x, v1.x, 0x7632),
-                                                                __byte_perm(v0.y, v1.y, 0x5410), __byte_perm(v0.y, v1.y, 0x7632));
-                    *reinterpret_cast<uint4*>(dst + 16) = make_uint4(__byte_perm(v0.z, v1.z, 0x5410), __byte_perm(v0.z, v1.z, 0x7632),
-                                                                     __byte_perm(v0.w, v1.w, 0x5410), __byte_perm(v0.w, v1.w, 0x7632));
-                    sxc[tok * (p.xc / 8) + 2 * ci] = st_sum8(v0);
-                    sxc[tok * (p.xc / 8) + 2 * ci + 1] = st_sum8(v1);
-                } else {
-                    *reinterpret_cast<uint4*>(dst) = BITS == 8 ? v0 : st_permute8(v0);
-                    sxc[tok * (p.xc / 8) + ci] = st_sum8(v0);
+#pragma unroll
+                for (int h = 0; h < NB; ++h) {
+                    if (e0 + h * blockDim.x >= n_items) break;
+                    uint8_t* dst = xs + tk[h] * xp + ci[h] * (2 * KP);
+                    if constexpr (BITS == 2) {             // (x0,x8) (x1,x9) ... (x7,x15)
+                        *reinterpret_cast<uint4*>(dst) = make_uint4(__byte_perm(v0[h].x, v1[h].x, 0x5410), __byte_perm(v0[h].x, v1[h].x, 0x7632),
+                                                                    __byte_perm(v0[h].y, v1[h].y, 0x5410), __byte_perm(v0[h].y, v1[h].y, 0x7632));
+                        *reinterpret_cast<uint4*>(dst + 16) = make_uint4(__byte_perm(v0[h].z, v1[h].z, 0x5410), __byte_perm(v0[h].z, v1[h].z, 0x7632),
+                                                                         __byte_perm(v0[h].w, v1[h].w, 0x5410), __byte_perm(v0[h].w, v1[h].w, 0x7632));
+                        sxc[tk[h] * (p.xc / 8) + 2 * ci[h]] = st_sum8(v0[h]);
+                        sxc[tk[h] * (p.xc / 8) + 2 * ci[h] + 1] = st_sum8(v1[h]);
+                    } else {
+                        *reinterpret_cast<uint4*>(dst) = BITS == 8 ? v0[h] : st_permute8(v0[h]);
+                        sxc[tk[h] * (p.xc / 8) + ci[h]] = st_sum8(v0[h]);
+                    }
                 }
             }
+            if (cb == kb0 && fused) {                      // the down-projection's MMAs, with the slice's loads behind them
+                float ah[NT][4];
+#pragma unroll
+                for (int tt = 0; tt < NT; ++tt) ah[tt][0] = ah[tt][1] = ah[tt][2] = ah[tt][3] = 0.f;
+                for (int kk = h_k0;;) {
+#pragma unroll
+                    for (int h = 0; h < ST_HSTEPS; ++h)
+#pragma unroll
+                        for (int tt = 0; tt < NT; ++tt) st_mma(ah[tt], ha[h][0], ha[h][1], ha[h][2], ha[h][3], hb[h][tt][0], hb[h][tt][1]);
+                    kk += 16 * nw * ST_HSTEPS;
+                    if (kk >= h_ke) break;
+                    h_load(kk);
+                }
+                st_store_hp<NT>(ah, hp, warp, g, q);
+            }
             __syncthreads();
-            const int g_first = k_lo / p.g, nseg = (k_hi - 1) / p.g - g_first + 1;
-            for (int e = threadIdx.x; e < nseg * TOKS; e += blockDim.x) {
-                const int seg = e / TOKS, tok = e % TOKS;
-                const int a = max(k_lo, (g_first + seg) * p.g), b = min(k_hi, (g_first + seg + 1) * p.g);
+            const int nseg = (k_hi - 1) / p.g - g_first + 1;
+            for (int e = threadIdx.x; e < KH * nseg * TOKS; e += blockDim.x) {
+                const int tok = e % TOKS, sg = (e / TOKS) % nseg, h = e / (TOKS * nseg);
+                const int n = ce - cb;
+                const int p_lo = (cb + st_part(n, h, p.khs)) * F::KB, p_hi = min((cb + st_part(n, h + 1, p.khs)) * F::KB, p.K);
+                const int a = max(p_lo, (g_first + sg) * p.g), b = min(p_hi, (g_first + sg + 1) * p.g);
                 float sum = 0.f;
                 for (int c8 = (a - k_lo) / 8; c8 < (b - k_lo) / 8; ++c8) sum += sxc[tok * (p.xc / 8) + c8];
-                sxs[seg * TOKS + tok] = sum;
+                sxs[(h * (xcb + 1) + sg) * TOKS + tok] = sum;
+            }
+            if (cb == kb0 && fused) {
+                for (int e = threadIdx.x; e < 256; e += blockDim.x) {
+                    float h = 0.f;
+                    for (int w = 0; w < nw; ++w) h += hp[w * 256 + e];
+                    hs[e] = h;
+                }
             }
             __syncthreads();
+            if (cb == kb0) {
+                st_cluster_wait();                         // every CTA of the cluster is running: its shared memory may be written
+                if (fused) st_push_h(rl, hs, rank, p.ks);
+            }
         }
-        for (int blk = cb; blk < ce; ++blk, ++it) {
+        const int b0 = cb + st_part(ce - cb, kh, p.khs), b1 = cb + st_part(ce - cb, kh + 1, p.khs);
+        int gpos = b0 < b1 ? b0 % bpg : 0, grpi = b0 < b1 ? b0 / bpg : 0;
+#pragma unroll 1
+        for (int blk = b0; blk < b1; ++blk) {
             cp_wait<F::NS - 1>();
             __syncwarp();
-            const uint8_t* slot = ring + (it % F::NS) * F::SLOT;
-            const int k0 = blk * F::KB;
-            if (k0 % p.g == 0 || it == 0) {                // a new group: this lane's scales and zero-points
+            const uint8_t* slot = ring + c_slot * F::SLOT;
+            if (gpos == 0 || blk == b0) {                  // a new group: this lane's scales and zero-points
                 const uint2 s2 = *reinterpret_cast<const uint2*>(slot + F::ROWS * 128 + 8 * g);
                 const uint2 z2 = *reinterpret_cast<const uint2*>(slot + F::ROWS * 128 + 64 + 8 * g);
                 const float2 sa = __half22float2(*reinterpret_cast<const __half2*>(&s2.x)), sb = __half22float2(*reinterpret_cast<const __half2*>(&s2.y));
@@ -436,11 +553,11 @@ __global__ void __launch_bounds__(256, 2) stream_fwd_kernel(const StreamParams p
                     for (int tt = 0; tt < NT; ++tt)
                         st_mma(grp[u][tt], pa[2 * s], pb[2 * s], pa[2 * s + 1], pb[2 * s + 1], xf[tt][2 * s], xf[tt][2 * s + 1]);
             }
-            if ((k0 + F::KB) % p.g == 0 || blk + 1 == ce) {   // end of a group segment: scale, correct, start afresh
-                const int seg = k0 / p.g - k_lo / p.g;
+            if (gpos == bpg - 1 || blk + 1 == b1) {        // end of a group segment: scale, correct, start afresh
+                const float* sxr = sxs + (kh * (xcb + 1) + grpi - g_first) * TOKS;
 #pragma unroll
                 for (int tt = 0; tt < NT; ++tt) {
-                    const float2 sx = *reinterpret_cast<const float2*>(sxs + seg * TOKS + 8 * tt + 2 * q);
+                    const float2 sx = *reinterpret_cast<const float2*>(sxr + 8 * tt + 2 * q);
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
                         acc[u][tt][0] += sc[2 * u] * grp[u][tt][0] + cz[2 * u] * sx.x;
@@ -451,64 +568,81 @@ __global__ void __launch_bounds__(256, 2) stream_fwd_kernel(const StreamParams p
                     }
                 }
             }
+            if (++gpos == bpg) { gpos = 0; ++grpi; }
+            if (++c_slot == F::NS) c_slot = 0;
             __syncwarp();
-            issue(it + F::NS);
+            issue();
         }
-        __syncthreads();                                   // the slice (and, at the end, the rings) may be overwritten
+        if (cb + xcb < kb1) __syncthreads();               // the slice may be overwritten
     }
-    cp_wait<0>();
-    // accumulator element (u, tt, e): column 4g + 2u + (e >> 1) of this warp's 32, token 2q + (e & 1) + 8 tt
-    {
-        const int pw = tile_c + 4;
+    // accumulator element (u, tt, e): column 4g + 2u + (e >> 1) of this warp's 32, token 2q + (e & 1) + 8 tt; sent to the
+    // CTA that finishes that column
 #pragma unroll
-        for (int u = 0; u < 2; ++u)
+    for (int u = 0; u < 2; ++u)
 #pragma unroll
-            for (int tt = 0; tt < NT; ++tt)
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    part[(2 * q + (e & 1) + 8 * tt) * pw + 32 * warp + 4 * g + 2 * u + (e >> 1)] = acc[u][tt][e];
-    }
-    st_epilogue<false, TOKS>(p, part, hs, hfull, lup, tile_c, rank);
+        for (int tt = 0; tt < NT; ++tt) {
+            st_push2(rl, rank, kh, 32 * cg + 4 * g + 2 * u, 2 * q + 8 * tt, acc[u][tt][0], acc[u][tt][1]);
+            st_push2(rl, rank, kh, 32 * cg + 4 * g + 2 * u + 1, 2 * q + 8 * tt, acc[u][tt][2], acc[u][tt][3]);
+        }
+    st_finish<false, TOKS>(p, recv_part, recv_h, hfull, lup, tile_c, rank);
 }
 
 // ------------------------------------------------------------------------------------------------------------
-// Backward: dX = dY W + s G A.  CTA (rank, tile): output features [FW W tile, + FW W) (warp w: FW of them, all inside
-// one group), contraction stages [st0, st1) of 32 SU packed columns.
+// Backward: dX = dY W + s G A.  CTA (rank, tile): output features [FW wc tile, + FW wc), contraction stages [st0, st1)
+// of 32 SU packed columns.  Warp (fw, kh): FW features (all inside one group) and part kh of the stages of every staged
+// slice of dY.
 // ------------------------------------------------------------------------------------------------------------
 template <int BITS, int NT>
-__global__ void __launch_bounds__(256, 2) stream_bwd_kernel(const StreamParams p) {
+__global__ void __launch_bounds__(512, 1) stream_bwd_kernel(const StreamParams p) {
     using F = Fmt<BITS>;
     constexpr int TOKS = 8 * NT;
     constexpr int NTILE = F::BPAIR / 2;                    // 16-feature MMA tiles per warp
     pdl_launch_dependents();
+    st_cluster_arrive_relaxed();                           // waited for before the first store into a peer's shared memory
     extern __shared__ __align__(128) uint8_t smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, q = lane & 3;
-    const int W = blockDim.x >> 5, tile_c = F::FW * W;
+    const int nw = blockDim.x >> 5, tile_c = F::FW * p.wc, sl = tile_c / p.ks;
+    const int fw = warp % p.wc, kh = warp / p.wc;
     const int rank = (int)st_cluster_rank();
-    const int tile_f0 = blockIdx.y * tile_c, f0 = tile_f0 + F::FW * warp;
+    const int tile_f0 = blockIdx.y * tile_c, f0 = tile_f0 + F::FW * fw;
     const bool live = f0 < p.K;                            // a warp beyond the last feature only keeps the barriers company
     const int row0 = f0 * BITS / 32;
     const int sw = 32 * F::SU;                             // packed columns per stage
     const int nst = (p.N + sw - 1) / sw;
     const int st0 = nst * rank / p.ks, st1 = nst * (rank + 1) / p.ks;
-    const int nit = st1 - st0;
     const int xp = p.xc * 2 + 64;
     const int xcs = p.xc / sw;                             // stages per staged slice
     const int copy = p.copies > 1 ? (f0 - tile_f0) / p.g : 0;
     uint8_t* ring = smem + warp * (F::BNS * F::BSLOT);
-    uint8_t* ys = smem + W * (F::BNS * F::BSLOT);          // [copies][TOKS][xp] scaled, permuted slices of dY
-    float* zp = reinterpret_cast<float*>(ys + p.copies * TOKS * xp);   // [W][2][16] zero-point sums, per warp
-    float* zc = zp + W * 32;                               // [2][16] their total
+    uint8_t* ys = smem + nw * (F::BNS * F::BSLOT);         // [copies][TOKS][xp] scaled, permuted slices of dY
+    float* zp = reinterpret_cast<float*>(ys + p.copies * TOKS * xp);   // [nw][2][16] zero-point sums, per warp
+    float* zc = zp + nw * 32;                              // [2][16] their total
     float* hs = zc + 32;
     float* hfull = hs + 256;
     __nv_bfloat16* lup = reinterpret_cast<__nv_bfloat16*>(hfull + 1024);
-    float* part = reinterpret_cast<float*>(smem);
-    float* hp = reinterpret_cast<float*>(ys);
+    float* hp = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(lup) + ST_LUP_BYTES);   // [nw][16][16]
+    float* recv_h = hp + nw * 256;                         // [ks][16][16]
+    float* recv_part = recv_h + p.ks * 256;                // [ks][KH][sl][16]
+    RecvLayout rl;
+    rl.part_addr = s_u32(recv_part); rl.h_addr = s_u32(recv_h); rl.sls = p.sls; rl.khs = p.khs;
 
-    auto issue = [&](int it) {
-        if (it < nit && live) {
-            const int cbase = (st0 + it) * sw;
-            const uint32_t dst = s_u32(ring + (it % F::BNS) * F::BSLOT);
+    int i_cs = st0, i_stg = 0, i_end = 0, i_slot = 0;
+    bool i_done = st0 >= st1 || !live;
+    auto i_enter = [&]() {
+        while (!i_done) {
+            const int n = min(i_cs + xcs, st1) - i_cs;
+            i_stg = i_cs + st_part(n, kh, p.khs);
+            i_end = i_cs + st_part(n, kh + 1, p.khs);
+            if (i_stg < i_end) return;
+            i_cs += xcs;
+            if (i_cs >= st1) i_done = true;
+        }
+    };
+    i_enter();
+    auto issue = [&]() {
+        if (!i_done) {
+            const int cbase = i_stg * sw;
+            const uint32_t dst = s_u32(ring + i_slot * F::BSLOT);
             if constexpr (BITS == 2) {
                 const int col = cbase + 32 * (lane >> 3) + 4 * (lane & 7);
                 const bool ok = col < p.N;
@@ -524,59 +658,74 @@ __global__ void __launch_bounds__(256, 2) stream_bwd_kernel(const StreamParams p
                     }
                 }
             }
+            if (++i_stg >= i_end) {
+                i_cs += xcs;
+                if (i_cs >= st1) i_done = true; else i_enter();
+            }
         }
+        if (++i_slot == F::BNS) i_slot = 0;
         cp_commit();
     };
-    for (int it = 0; it < F::BNS; ++it) issue(it);
+#pragma unroll 1
+    for (int it = 0; it < F::BNS; ++it) issue();
+
+    const int n_lo_cta = st0 * sw, n_hi_cta = min(st1 * sw, p.N);
+    const int ngroups = p.K / p.g;
+    {   // ask the lines this CTA will read right after the wait into L2: its slices of dY, B, A and of the group parameters
+        const int nbytes = (n_hi_cta - n_lo_cta) * 2;
+        if (nbytes > 0) {
+            st_prefetch_l2(p.In + n_lo_cta, (size_t)p.N * 2, p.M, nbytes, threadIdx.x, blockDim.x);
+            if (p.r > 0 && p.fused) st_prefetch_l2(p.Ldown + (size_t)n_lo_cta * p.r, 0, 1, nbytes * p.r, threadIdx.x, blockDim.x);
+            for (int c = 0; c < p.copies; ++c) {
+                const int gk = tile_f0 / p.g + c;
+                if (gk < ngroups) {
+                    st_prefetch_l2(p.scales + (size_t)gk * p.N + n_lo_cta, 0, 1, nbytes, threadIdx.x, blockDim.x);
+                    st_prefetch_l2(p.zeros + (size_t)gk * p.N + n_lo_cta, 0, 1, nbytes, threadIdx.x, blockDim.x);
+                }
+            }
+        }
+        const int c_lo = tile_f0 + rank * sl;
+        if (p.r > 0 && c_lo < p.K) st_prefetch_l2(p.Lup + c_lo, (size_t)p.K * 2, p.r, min(sl, p.K - c_lo) * 2, threadIdx.x, blockDim.x);
+    }
 
     pdl_wait();
 
-    const int n_lo_cta = st0 * sw, n_hi_cta = min(st1 * sw, p.N);
-    st_stage_lup<true>(p, lup, hfull, tile_c, rank);
-    for (int e = threadIdx.x; e < W * 32; e += blockDim.x) zp[e] = 0.f;
     // ---- LoRA: this CTA's part of G = dY B.  B [N, r] has the ranks contiguous, so a lane loads two ranks of its own
-    // contraction column and movmatrix turns them into two columns of one rank ----
-    if (p.r > 0 && p.fused) {
-        float ag[NT][4];
+    // contraction column and movmatrix turns them into two columns of one rank.  The loads of the first ST_HSTEPS steps are
+    // issued here and used once the slice of dY is on its way too ----
+    const bool fused = p.r > 0 && p.fused;
+    const int h_n0 = n_lo_cta + 16 * warp;
+    uint32_t ha[ST_HSTEPS][4], hb[ST_HSTEPS][NT][2];
+    auto h_load = [&](int nn) {
 #pragma unroll
-        for (int tt = 0; tt < NT; ++tt) ag[tt][0] = ag[tt][1] = ag[tt][2] = ag[tt][3] = 0.f;
-        for (int nb = n_lo_cta + 16 * warp; nb < n_hi_cta; nb += 16 * W) {
-            const bool v0 = nb + g < p.N, v1 = nb + 8 + g < p.N;
+        for (int h = 0; h < ST_HSTEPS; ++h) {
+            const int nb = nn + 16 * nw * h;
+            const bool in = fused && nb < n_hi_cta;
+            const bool v0 = in && nb + g < p.N, v1 = in && nb + 8 + g < p.N;
             const __nv_bfloat16* b_lo = p.Ldown + (size_t)(nb + g) * p.r + 2 * q;
             const __nv_bfloat16* b_hi = p.Ldown + (size_t)(nb + 8 + g) * p.r + 2 * q;
-            const uint32_t a0 = st_movm(v0 ? ldg32(b_lo) : 0u), a2 = st_movm(v1 ? ldg32(b_hi) : 0u);
-            const uint32_t a1 = st_movm(v0 && p.r > 8 ? ldg32(b_lo + 8) : 0u), a3 = st_movm(v1 && p.r > 8 ? ldg32(b_hi + 8) : 0u);
+            ha[h][0] = v0 ? ldg32(b_lo) : 0u; ha[h][2] = v1 ? ldg32(b_hi) : 0u;
+            ha[h][1] = (v0 && p.r > 8) ? ldg32(b_lo + 8) : 0u; ha[h][3] = (v1 && p.r > 8) ? ldg32(b_hi + 8) : 0u;
 #pragma unroll
             for (int tt = 0; tt < NT; ++tt) {
                 const int tok = g + 8 * tt;
                 const __nv_bfloat16* y = p.In + (size_t)tok * p.N + nb + 2 * q;
-                const uint32_t b0 = (tok < p.M && nb + 2 * q < p.N) ? ldg32(y) : 0u;
-                const uint32_t b1 = (tok < p.M && nb + 8 + 2 * q < p.N) ? ldg32(y + 8) : 0u;
-                st_mma(ag[tt], a0, a1, a2, a3, b0, b1);
+                hb[h][tt][0] = (in && tok < p.M && nb + 2 * q < p.N) ? ldg32(y) : 0u;
+                hb[h][tt][1] = (in && tok < p.M && nb + 8 + 2 * q < p.N) ? ldg32(y + 8) : 0u;
             }
         }
-        float* mine = hp + warp * 256;
-#pragma unroll
-        for (int tt = 0; tt < 2; ++tt)
-#pragma unroll
-            for (int e = 0; e < 4; ++e)
-                mine[(g + ((e & 2) ? 8 : 0)) * 16 + 8 * tt + 2 * q + (e & 1)] = tt < NT ? ag[tt < NT ? tt : 0][e] : 0.f;
-        __syncthreads();
-        for (int e = threadIdx.x; e < 256; e += blockDim.x) {
-            float h = 0.f;
-            for (int w = 0; w < W; ++w) h += hp[w * 256 + e];
-            hs[e] = h;
-        }
-    }
-    __syncthreads();
+    };
+    if (fused) h_load(h_n0);
+    st_stage_lup<true>(p, lup, hfull, tile_c, rank);
+    for (int e = threadIdx.x; e < nw * 32; e += blockDim.x) zp[e] = 0.f;
 
     float acc[NTILE][NT][4];
 #pragma unroll
     for (int t = 0; t < NTILE; ++t)
 #pragma unroll
         for (int tt = 0; tt < NT; ++tt) acc[t][tt][0] = acc[t][tt][1] = acc[t][tt][2] = acc[t][tt][3] = 0.f;
-    const int ngroups = p.K / p.g;
-    int it = 0;
+    int c_slot = 0;
+    if (st0 >= st1) st_cluster_wait();                     // (an empty range: the wait below is never reached)
     for (int cs = st0; cs < st1; cs += xcs) {
         const int ce = min(cs + xcs, st1);
         const int n_lo = cs * sw, n_hi = min(ce * sw, p.N);
@@ -584,36 +733,65 @@ __global__ void __launch_bounds__(256, 2) stream_bwd_kernel(const StreamParams p
         {
             const int per_tok = (ce - cs) * sw / 8;
             for (int e = threadIdx.x; e < TOKS * per_tok; e += blockDim.x) {
-                const int tok = e / per_tok, ci = e % per_tok;
+                const int tok = e / per_tok, ci = e - tok * per_tok;
                 const int n = n_lo + ci * 8;
                 const bool ok = tok < p.M && n < p.N;
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (ok) v = *reinterpret_cast<const uint4*>(p.In + (size_t)tok * p.N + n);
-                for (int c = 0; c < p.copies; ++c) {
-                    const int gk = tile_f0 / p.g + c;
-                    uint4 o = make_uint4(0, 0, 0, 0);
-                    if (ok && gk < ngroups) {
-                        const uint4 s8 = *reinterpret_cast<const uint4*>(p.scales + (size_t)gk * p.N + n);
-                        const float2 s0 = __half22float2(*reinterpret_cast<const __half2*>(&s8.x)), s1 = __half22float2(*reinterpret_cast<const __half2*>(&s8.y));
-                        const float2 s2 = __half22float2(*reinterpret_cast<const __half2*>(&s8.z)), s3 = __half22float2(*reinterpret_cast<const __half2*>(&s8.w));
-                        const __nv_bfloat162 o0 = __floats2bfloat162_rn(bf16_lo(v.x) * s0.x, bf16_hi(v.x) * s0.y);
-                        const __nv_bfloat162 o1 = __floats2bfloat162_rn(bf16_lo(v.y) * s1.x, bf16_hi(v.y) * s1.y);
-                        const __nv_bfloat162 o2 = __floats2bfloat162_rn(bf16_lo(v.z) * s2.x, bf16_hi(v.z) * s2.y);
-                        const __nv_bfloat162 o3 = __floats2bfloat162_rn(bf16_lo(v.w) * s3.x, bf16_hi(v.w) * s3.y);
-                        o = make_uint4(*reinterpret_cast<const uint32_t*>(&o0), *reinterpret_cast<const uint32_t*>(&o1),
-                                       *reinterpret_cast<const uint32_t*>(&o2), *reinterpret_cast<const uint32_t*>(&o3));
+                uint4 v = make_uint4(0, 0, 0, 0), s8[2];
+                s8[0] = s8[1] = make_uint4(0, 0, 0, 0);
+                if (ok) {
+                    v = *reinterpret_cast<const uint4*>(p.In + (size_t)tok * p.N + n);
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        const int gk = tile_f0 / p.g + c;
+                        if (c < p.copies && gk < ngroups) s8[c] = *reinterpret_cast<const uint4*>(p.scales + (size_t)gk * p.N + n);
                     }
+                }
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    if (c >= p.copies) break;
+                    const float2 s0 = __half22float2(*reinterpret_cast<const __half2*>(&s8[c].x)), s1 = __half22float2(*reinterpret_cast<const __half2*>(&s8[c].y));
+                    const float2 s2 = __half22float2(*reinterpret_cast<const __half2*>(&s8[c].z)), s3 = __half22float2(*reinterpret_cast<const __half2*>(&s8[c].w));
+                    const __nv_bfloat162 o0 = __floats2bfloat162_rn(bf16_lo(v.x) * s0.x, bf16_hi(v.x) * s0.y);
+                    const __nv_bfloat162 o1 = __floats2bfloat162_rn(bf16_lo(v.y) * s1.x, bf16_hi(v.y) * s1.y);
+                    const __nv_bfloat162 o2 = __floats2bfloat162_rn(bf16_lo(v.z) * s2.x, bf16_hi(v.z) * s2.y);
+                    const __nv_bfloat162 o3 = __floats2bfloat162_rn(bf16_lo(v.w) * s3.x, bf16_hi(v.w) * s3.y);
+                    const uint4 o = make_uint4(*reinterpret_cast<const uint32_t*>(&o0), *reinterpret_cast<const uint32_t*>(&o1),
+                                               *reinterpret_cast<const uint32_t*>(&o2), *reinterpret_cast<const uint32_t*>(&o3));
                     *reinterpret_cast<uint4*>(ys + (c * TOKS + tok) * xp + ci * 16) = st_permute8(o);
                 }
             }
+            if (cs == st0 && fused) {                      // the down-projection's MMAs, with the slice's loads behind them
+                float ag[NT][4];
+#pragma unroll
+                for (int tt = 0; tt < NT; ++tt) ag[tt][0] = ag[tt][1] = ag[tt][2] = ag[tt][3] = 0.f;
+                for (int nn = h_n0;;) {
+#pragma unroll
+                    for (int h = 0; h < ST_HSTEPS; ++h) {
+                        const uint32_t a0 = st_movm(ha[h][0]), a1 = st_movm(ha[h][1]), a2 = st_movm(ha[h][2]), a3 = st_movm(ha[h][3]);
+#pragma unroll
+                        for (int tt = 0; tt < NT; ++tt) st_mma(ag[tt], a0, a1, a2, a3, hb[h][tt][0], hb[h][tt][1]);
+                    }
+                    nn += 16 * nw * ST_HSTEPS;
+                    if (nn >= n_hi_cta) break;
+                    h_load(nn);
+                }
+                st_store_hp<NT>(ag, hp, warp, g, q);
+            }
             __syncthreads();
+            if (cs == st0 && fused) {
+                for (int e = threadIdx.x; e < 256; e += blockDim.x) {
+                    float h = 0.f;
+                    for (int w = 0; w < nw; ++w) h += hp[w * 256 + e];
+                    hs[e] = h;
+                }
+            }
             // zero-point term: sum_n dYs[m, n] (OFF + z[G, n]) as one MMA row; 32-column units dealt to the warps
             for (int c = 0; c < p.copies; ++c) {
                 const int gk = tile_f0 / p.g + c;
                 float za[NT][4];
 #pragma unroll
                 for (int tt = 0; tt < NT; ++tt) za[tt][0] = za[tt][1] = za[tt][2] = za[tt][3] = 0.f;
-                for (int un = warp; un < (n_hi - n_lo + 31) / 32; un += W) {
+                for (int un = warp; un < (n_hi - n_lo + 31) / 32; un += nw) {
                     const int n = n_lo + 32 * un + 8 * q;
                     uint32_t zr[4] = {0u, 0u, 0u, 0u};     // (z0,z4) (z1,z5) (z2,z6) (z3,z7) as bf16 of OFF + z
                     if (g == 0 && n < p.N && gk < ngroups) {
@@ -641,11 +819,20 @@ __global__ void __launch_bounds__(256, 2) stream_bwd_kernel(const StreamParams p
                 }
             }
         }
+        if (cs == st0) {
+            st_cluster_wait();                             // every CTA of the cluster is running: its shared memory may be written
+            if (fused) {
+                __syncthreads();                           // hs is complete
+                st_push_h(rl, hs, rank, p.ks);
+            }
+        }
         if (live) {
-            for (int stg = cs; stg < ce; ++stg, ++it) {
+            const int s0 = cs + st_part(ce - cs, kh, p.khs), s1 = cs + st_part(ce - cs, kh + 1, p.khs);
+#pragma unroll 1
+            for (int stg = s0; stg < s1; ++stg) {
                 cp_wait<F::BNS - 1>();
                 __syncwarp();
-                const uint8_t* slot = ring + (it % F::BNS) * F::BSLOT;
+                const uint8_t* slot = ring + c_slot * F::BSLOT;
 #pragma unroll
                 for (int su = 0; su < F::SU; ++su) {
                     const int ul = (stg - cs) * F::SU + su;    // 32-column unit inside the staged slice
@@ -678,38 +865,38 @@ __global__ void __launch_bounds__(256, 2) stream_bwd_kernel(const StreamParams p
                         }
                     }
                 }
+                if (++c_slot == F::BNS) c_slot = 0;
                 __syncwarp();
-                issue(it + F::BNS);
+                issue();
             }
         }
         __syncthreads();
     }
-    cp_wait<0>();
     for (int e = threadIdx.x; e < 32; e += blockDim.x) {   // zero-point sums of the whole range, warps added in order
         float z = 0.f;
-        for (int w = 0; w < W; ++w) z += zp[w * 32 + e];
+        for (int w = 0; w < nw; ++w) z += zp[w * 32 + e];
         zc[e] = z;
     }
     __syncthreads();
-    // accumulator element (t, tt, e): MMA row g + 8 (e >> 1) of tile t = matrix 2t + (e >> 1), column g of it; token 2q + (e & 1) + 8 tt
-    {
-        const int pw = tile_c + 4;
+    // accumulator element (t, tt, e): MMA row g + 8 (e >> 1) of tile t = matrix 2t + (e >> 1), column g of it; token
+    // 2q + (e & 1) + 8 tt.  The zero-point sum covers the CTA's whole range, so part 0 alone subtracts it.  Each pair of
+    // tokens goes to the CTA that finishes that feature.
 #pragma unroll
-        for (int t = 0; t < NTILE; ++t)
+    for (int t = 0; t < NTILE; ++t)
 #pragma unroll
-            for (int tt = 0; tt < NT; ++tt)
+        for (int tt = 0; tt < NT; ++tt)
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int m = 2 * t + (e >> 1);        // pair index of the matrix
-                    int f;                                 // feature of matrix m, column g (lane q' = g >> 1 supplied half g & 1)
-                    if constexpr (BITS == 2) f = 2 * (g >> 1) + m + 8 * (g & 1);
-                    else if constexpr (BITS == 8) f = 16 * (m >> 1) + 4 * (g >> 1) + 2 * (m & 1) + (g & 1);
-                    else f = 8 * (g >> 1) + m + 4 * (g & 1);
-                    const int tok = 2 * q + (e & 1) + 8 * tt;
-                    part[tok * pw + F::FW * warp + f] = acc[t][tt][e] - zc[copy * 16 + tok];
-                }
-    }
-    st_epilogue<true, TOKS>(p, part, hs, hfull, lup, tile_c, rank);
+            for (int hh = 0; hh < 2; ++hh) {
+                const int m = 2 * t + hh;                  // pair index of the matrix
+                int f;                                     // feature of matrix m, column g (lane q' = g >> 1 supplied half g & 1)
+                if constexpr (BITS == 2) f = 2 * (g >> 1) + m + 8 * (g & 1);
+                else if constexpr (BITS == 8) f = 16 * (m >> 1) + 4 * (g >> 1) + 2 * (m & 1) + (g & 1);
+                else f = 8 * (g >> 1) + m + 4 * (g & 1);
+                const int tok = 2 * q + 8 * tt;
+                const float z0 = kh == 0 ? zc[copy * 16 + tok] : 0.f, z1 = kh == 0 ? zc[copy * 16 + tok + 1] : 0.f;
+                st_push2(rl, rank, kh, F::FW * fw + f, tok, acc[t][tt][2 * hh] - z0, acc[t][tt][2 * hh + 1] - z1);
+            }
+    st_finish<true, TOKS>(p, recv_part, recv_h, hfull, lup, tile_c, rank);
 }
 
 // Raising a kernel's dynamic shared-memory limit is a per-function AND per-device setting: `done` belongs to one kernel
@@ -743,15 +930,63 @@ int st_launch(const StreamParams& p, int W, int tiles, size_t smem_bytes, cudaSt
     return err == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
 }
 
+// Dynamic shared memory of a launch: the carve-up at the top of the two kernels, in the same order.
+template <int BITS>
+size_t st_smem_bytes(bool transposed, int nw, int toks, int xc, int copies, int KH, int ks, int tile_c) {
+    using F = Fmt<BITS>;
+    const size_t tail = (size_t)(256 + 1024) * 4 + ST_LUP_BYTES + (size_t)nw * 1024 + (size_t)ks * 1024 + (size_t)KH * tile_c * 64;
+    if (transposed)
+        return (size_t)nw * F::BNS * F::BSLOT + (size_t)copies * toks * (xc * 2 + 64) + (size_t)(nw * 32 + 32) * 4 + tail;
+    return (size_t)nw * F::NS * F::SLOT + (size_t)toks * (xc * 2 + F::XPAD) + (size_t)(toks * (xc / 8) + KH * (xc / F::KB + 1) * toks) * 4 + tail;
+}
+
 // Warps per CTA of the backward kernel: the features of a CTA must lie in one group or span exactly two.
 int bwd_warps(int bits, int g) {
     const int fw = bits == 2 ? 16 : 32;
-    for (int W = 8; W >= 1; W /= 2)
-        if (g % (W * fw) == 0 || W * fw == 2 * g) return W;
+    const int order[4] = {4, 8, 2, 1};                     // four side by side leave room for four parts of the contraction
+    for (int i = 0; i < 4; ++i)
+        if (g % (order[i] * fw) == 0 || order[i] * fw == 2 * g) return order[i];
     return 0;
 }
 
 int fwd_kb(int bits) { return bits == 2 ? 64 : 32; }
+
+__global__ void __launch_bounds__(512, 1) st_probe_kernel() {}
+
+struct DeviceFacts { int sms = 0; int clusters[9] = {}; };
+
+// SM count and how many clusters of 2 / 4 / 8 CTAs that own an SM each can run at once, per device ordinal.
+const DeviceFacts& device_facts() {
+    static std::mutex mu;
+    static DeviceFacts facts[ST_MAX_DEVICES];
+    static DeviceFacts fallback;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= ST_MAX_DEVICES) { fallback.sms = 148; fallback.clusters[2] = 74; fallback.clusters[4] = 32; fallback.clusters[8] = 14; return fallback; }
+    std::lock_guard<std::mutex> lock(mu);
+    DeviceFacts& f = facts[dev];
+    if (f.sms == 0) {
+        int v = 0;
+        f.sms = (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) ? v : 148;
+        (void)cudaFuncSetAttribute(st_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        for (int cs = 2; cs <= 8; cs *= 2) {
+            cudaLaunchConfig_t cfg{};
+            cfg.gridDim = dim3((unsigned)cs, (unsigned)f.sms);
+            cfg.blockDim = dim3(512);
+            cfg.dynamicSmemBytes = 200 * 1024;         // one CTA per SM, as the streaming kernels are
+            cudaLaunchAttribute attr;
+            attr.id = cudaLaunchAttributeClusterDimension;
+            attr.val.clusterDim.x = (unsigned)cs; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+            cfg.attrs = &attr;
+            cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, st_probe_kernel, &cfg) != cudaSuccess || n <= 0) { (void)cudaGetLastError(); n = f.sms / cs * 3 / 4; }
+            f.clusters[cs] = n;
+        }
+    }
+    return f;
+}
+int max_clusters(int cs) { return cs <= 1 ? device_facts().sms : device_facts().clusters[cs > 8 ? 8 : cs]; }
+int sm_count_here() { return device_facts().sms; }
 
 }  // namespace
 
@@ -774,43 +1009,55 @@ int launch_stream_gemm(const qlora_desc& d, int M, bool transposed, const void* 
     p.fused = (d.r > 0 && !p_is_input) ? 1 : 0;
     if (p.fused && d.r > 16) return QLORA_ERR_INVALID_ARG;
     const int nt = M > 8 ? 2 : 1, toks = 8 * nt;
-    int W, tile_c, units;                                  // warps per CTA, output columns per CTA, contraction stages
+    int wc, tile_c, units;                                 // warps side by side, output columns per CTA, contraction stages
     if (transposed) {
-        W = bwd_warps(d.bits, d.group_size);
-        if (W == 0) return QLORA_ERR_UNSUPPORTED;
-        tile_c = W * (d.bits == 2 ? 16 : 32);
+        wc = bwd_warps(d.bits, d.group_size);
+        if (wc == 0) return QLORA_ERR_UNSUPPORTED;
+        tile_c = wc * (d.bits == 2 ? 16 : 32);
         p.copies = tile_c > d.group_size ? 2 : 1;
         units = (d.N + (d.bits == 2 ? 128 : 32) - 1) / (d.bits == 2 ? 128 : 32);
     } else {
         if (d.group_size % fwd_kb(d.bits) != 0) return QLORA_ERR_UNSUPPORTED;
-        W = d.N >= 256 ? 8 : (d.N >= 128 ? 4 : (d.N >= 64 ? 2 : 1));
-        tile_c = 32 * W;
+        wc = d.N >= 128 ? 4 : (d.N >= 64 ? 2 : 1);
+        tile_c = 32 * wc;
         p.copies = 1;
         units = (d.K + fwd_kb(d.bits) - 1) / fwd_kb(d.bits);
     }
+    p.wc = wc;
     const int tiles = (p.C + tile_c - 1) / tile_c;
-    // split the contraction until the grid covers the GPU (about one CTA per SM), keeping a few stages per CTA
+    // split the contraction over a cluster until the grid covers the GPU: one CTA per SM, and no more clusters than can
+    // run at once (the clusters of a launch that come later would wait for whole earlier ones to finish)
     int ks = 1;
-    while (ks < 8 && tiles * ks < 120 && units / (2 * ks) >= 4 && tile_c / (2 * ks) >= 1) ks *= 2;
+    while (ks < 8 && tiles * 2 * ks <= max_clusters(2 * ks) * 2 * ks && tiles * 2 * ks <= sm_count_here() && units / (2 * ks) >= 4 &&
+           tile_c / (2 * ks) >= 1)
+        ks *= 2;
     p.ks = ks;
-    p.xc = (transposed && p.copies * toks > 16) ? 256 : 512;
+    // ... and inside a CTA until it has sixteen warps, while a warp keeps at least two stages
+    p.khs = 0;
+    while ((wc << (p.khs + 1)) <= 16 && p.khs < 2 && units / (ks << (p.khs + 1)) >= 2) ++p.khs;
+    const int nw = wc << p.khs, KH = 1 << p.khs;
     const int sl = tile_c / ks;
-    p.lup_staged = (sl * d.r * 2 <= ST_LUP_BYTES) ? 1 : 0;
-    size_t smem;
-    if (transposed) {
-        const int bslot = (d.bits == 2 ? 1 : d.bits) * 128 * (d.bits == 2 ? 4 : 1), bns = d.bits == 8 ? 8 : 16;
-        smem = (size_t)W * bns * bslot + (size_t)p.copies * toks * (p.xc * 2 + 64) + (size_t)(W * 32 + 32 + 256 + 1024) * 4 + ST_LUP_BYTES;
-    } else {
-        const int kb = fwd_kb(d.bits), rows = kb * d.bits / 32, slot = rows * 128 + 128;
-        const int ns = d.bits == 8 ? 7 : (d.bits == 3 ? 16 : 12);
-        const int xpad = d.bits == 2 ? 16 : (d.bits == 8 ? 32 : 64);
-        smem = (size_t)W * ns * slot + (size_t)toks * (p.xc * 2 + xpad) + (size_t)(toks * (p.xc / 8) + (p.xc / kb + 1) * toks + 256 + 1024) * 4 + ST_LUP_BYTES;
+    p.sls = 0;
+    while ((1 << p.sls) < sl) ++p.sls;
+    // the activation slice staged per pass: the CTA's whole range when that fits (one pass, two barriers), else 512 at a time
+    {
+        const int unit = transposed ? (d.bits == 2 ? 128 : 32) : fwd_kb(d.bits);
+        const int range = ((units + ks - 1) / ks) * unit;
+        const int cap = transposed ? ((p.copies * toks > 16) ? 512 : 1024) : 1024;
+        p.xc = range <= cap ? ((range + 127) / 128) * 128 : 512;
+        if (p.xc < 128) p.xc = 128;
     }
-    // the partial tile [toks][tile_c + 4] fp32 reuses the rings
-    const size_t part = (size_t)16 * (tile_c + 4) * 4;
-    if (smem < part + 4096) smem = part + 4096;
+    p.lup_staged = (sl * d.r * 2 <= ST_LUP_BYTES) ? 1 : 0;
+    size_t smem = 0;
+    switch (d.bits) {
+        case 2: smem = st_smem_bytes<2>(transposed, nw, toks, p.xc, p.copies, KH, ks, tile_c); break;
+        case 3: smem = st_smem_bytes<3>(transposed, nw, toks, p.xc, p.copies, KH, ks, tile_c); break;
+        case 4: smem = st_smem_bytes<4>(transposed, nw, toks, p.xc, p.copies, KH, ks, tile_c); break;
+        case 8: smem = st_smem_bytes<8>(transposed, nw, toks, p.xc, p.copies, KH, ks, tile_c); break;
+    }
+    if (smem > 227 * 1024) return QLORA_ERR_UNSUPPORTED;
 #define QLORA_ST(B, NT)                                                                                   \
-    return transposed ? st_launch<B, NT, true>(p, W, tiles, smem, st) : st_launch<B, NT, false>(p, W, tiles, smem, st)
+    return transposed ? st_launch<B, NT, true>(p, nw, tiles, smem, st) : st_launch<B, NT, false>(p, nw, tiles, smem, st)
 #define QLORA_ST_BITS(NT)           \
     switch (d.bits) {               \
         case 2: QLORA_ST(2, NT);    \
