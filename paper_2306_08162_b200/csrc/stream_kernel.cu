@@ -72,7 +72,8 @@ struct StreamParams {
     int wc;                      // warps side by side in a CTA (32 columns forward, FW features backward each)
     int khs;                     // log2 of the parts the warps of a CTA split each staged slice of the contraction into
     int sls;                     // log2 of the columns a CTA of the cluster finishes (32 wc / ks or FW wc / ks)
-    int xc;                      // contraction elements of the activation slice staged per pass
+    int lwc, lks;                // log2 of wc and of ks
+    int xc;                      // contraction elements of the activations staged per pass (a power of two, all parts together)
     int copies;                  // backward: groups a CTA's features span (1 or 2)
     int fused;                   // H / G is computed here (ranks up to 16) and written to P; else P is an input
     int lup_staged;              // the epilogue's slice of the second adapter fits its shared-memory area
@@ -272,14 +273,8 @@ __device__ __forceinline__ void st_stage_lup(const StreamParams& p, __nv_bfloat1
 }
 
 // Before griddepcontrol.wait nothing but the frozen weights may be READ, but lines can be asked into L2 (the point of
-// coherence: a line the predecessor rewrites afterwards is simply updated there).  `rows` rows of `bytes` bytes each.
-__device__ __forceinline__ void st_prefetch_l2(const void* base, size_t row_pitch_bytes, int rows, int bytes, int first, int nthr) {
-    const int per_row = (bytes + 127) / 128;
-    for (int e = first; e < rows * per_row; e += nthr) {
-        const int rr = e / per_row, i = e - rr * per_row;
-        asm volatile("prefetch.global.L2 [%0];" ::"l"(static_cast<const char*>(base) + (size_t)rr * row_pitch_bytes + (size_t)i * 128));
-    }
-}
+// coherence: a line the predecessor rewrites afterwards is simply updated there); the kernels do that for the slices of
+// the activations and adapters they load right after the wait.
 
 // A warp's partial H / G tile ([16 ranks][16 tokens], MMA accumulator layout) -> its slot of hp.
 template <int NT>
@@ -292,39 +287,42 @@ __device__ __forceinline__ void st_store_hp(float (&ah)[NT][4], float* hp, int w
             mine[(g + ((e & 2) ? 8 : 0)) * 16 + 8 * tt + 2 * q + (e & 1)] = tt < NT ? ah[tt < NT ? tt : 0][e] : 0.f;
 }
 
-// Part `kh` of `n` consecutive items split KH = 2^khs ways.
-__device__ __forceinline__ int st_part(int n, int kh, int khs) { return (n * kh) >> khs; }
-
 // ------------------------------------------------------------------------------------------------------------
 // Forward: Y = X W^T + s H B^T.  CTA (rank, tile): columns [32 wc tile, + 32 wc), contraction blocks [kb0, kb1) of KB
-// elements.  Warp (cg, kh): 32 columns, and part kh of the blocks of every staged activation slice.
+// elements.  Warp (cg, kh): 32 columns and the kh-th of KH consecutive parts of [kb0, kb1).  The activations of the
+// parts are staged side by side, xpb blocks of every part per pass (one pass when the CTA's range fits the buffer).
 // ------------------------------------------------------------------------------------------------------------
 constexpr int ST_HSTEPS = 4;   // k16 steps of the fused down-projection whose operands a warp loads in one go
+
+struct PartInfo { int k0, k1, gf, nseg; };   // a part's share of the current pass: contraction range, first group, segments
 
 template <int BITS, int NT>
 __global__ void __launch_bounds__(512, 1) stream_fwd_kernel(const StreamParams p) {
     using F = Fmt<BITS>;
-    constexpr int TOKS = 8 * NT;
+    constexpr int TOKS = 8 * NT, LTOKS = NT == 1 ? 3 : 4;
+    constexpr int KP = BITS == 2 ? 16 : 8;                 // contraction elements per staged item
+    constexpr int LKB = BITS == 2 ? 6 : 5;
     pdl_launch_dependents();
     st_cluster_arrive_relaxed();                           // waited for before the first store into a peer's shared memory
     extern __shared__ __align__(128) uint8_t smem[];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, q = lane & 3;
-    const int nw = blockDim.x >> 5, tile_c = 32 * p.wc, KH = 1 << p.khs;
-    const int cg = warp % p.wc, kh = warp / p.wc;
+    __shared__ PartInfo tab[4];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, q = lane & 3;
+    const int nthr = blockDim.x, nw = nthr >> 5, tile_c = 32 * p.wc, KH = 1 << p.khs;
+    const int cg = warp & (p.wc - 1), kh = warp >> p.lwc;
     const int rank = (int)st_cluster_rank();
     const int col0 = blockIdx.y * tile_c + 32 * cg;
-    const int nblk = (p.K + F::KB - 1) / F::KB;
-    const int kb0 = nblk * rank / p.ks, kb1 = nblk * (rank + 1) / p.ks;
-    const int total_rows = p.K * BITS / 32;
+    const int nblk = (p.K + F::KB - 1) >> LKB;
+    const int kb0 = (nblk * rank) >> p.lks, kb1 = (nblk * (rank + 1)) >> p.lks, nb = kb1 - kb0;
+    const int wb0 = kb0 + ((nb * kh) >> p.khs), wb1 = kb0 + ((nb * (kh + 1)) >> p.khs);
     const int xp = p.xc * 2 + F::XPAD;
-    const int xcb = p.xc / F::KB;                          // blocks per staged slice
-    const int bpg = p.g / F::KB;                           // blocks per group
-    const int sl = tile_c / p.ks;
+    const int xpb = (p.xc >> LKB) >> p.khs;                // blocks of a part staged per pass
+    const int bpg = p.g >> LKB;                            // blocks per group
+    const int sl = tile_c >> p.lks;
     uint8_t* ring = smem + warp * (F::NS * F::SLOT);
-    uint8_t* xs = smem + nw * (F::NS * F::SLOT);           // [TOKS][xp] permuted activation slice
+    uint8_t* xs = smem + nw * (F::NS * F::SLOT);           // [TOKS][xp] permuted activations: KH parts side by side
     float* sxc = reinterpret_cast<float*>(xs + TOKS * xp); // [TOKS][xc / 8] sums of 8 activations
-    float* sxs = sxc + TOKS * (p.xc / 8);                  // [KH][xcb + 1][TOKS] sums per (part, group) segment of the slice
-    float* hs = sxs + KH * (xcb + 1) * TOKS;               // [16][16] this CTA's part of H
+    float* sxs = sxc + TOKS * (p.xc >> 3);                 // [KH][xpb + 1][TOKS] sums per (part, group) segment of the pass
+    float* hs = sxs + KH * (xpb + 1) * TOKS;               // [16][16] this CTA's part of H
     float* hfull = hs + 256;                               // [r <= 64][16] the whole of H
     __nv_bfloat16* lup = reinterpret_cast<__nv_bfloat16*>(hfull + 1024);
     float* hp = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(lup) + ST_LUP_BYTES);   // [nw][16][16]
@@ -333,44 +331,31 @@ __global__ void __launch_bounds__(512, 1) stream_fwd_kernel(const StreamParams p
     RecvLayout rl;
     rl.part_addr = s_u32(recv_part); rl.h_addr = s_u32(recv_h); rl.sls = p.sls; rl.khs = p.khs;
 
-    // the copy engine's view of this warp's block sequence (it runs NS blocks ahead of the arithmetic)
-    int i_cb = kb0, i_blk = 0, i_end = 0, i_gpos = 0, i_slot = 0;
-    bool i_first = true, i_done = kb0 >= kb1;
-    auto i_enter = [&]() {                                 // position on this warp's part of slice i_cb (skipping empty parts)
-        while (!i_done) {
-            const int n = min(i_cb + xcb, kb1) - i_cb;
-            i_blk = i_cb + st_part(n, kh, p.khs);
-            i_end = i_cb + st_part(n, kh + 1, p.khs);
-            if (i_blk < i_end) { i_gpos = i_blk % bpg; i_first = true; return; }
-            i_cb += xcb;
-            if (i_cb >= kb1) i_done = true;
-        }
-    };
-    i_enter();
+    // ---- the copy side of this warp: blocks wb0 .. wb1 - 1 in order, NS ahead of the arithmetic ----
+    const int i_row = lane >> 3, i_ch = lane & 7;
+    const bool i_col_ok = col0 + 4 * i_ch < p.N;
+    const uint32_t* i_src = p.Q + (size_t)(wb0 * F::ROWS + i_row) * p.N + col0 + 4 * i_ch;   // row i_row of block wb0
+    const size_t i_stride = (size_t)F::ROWS * p.N;
+    const uint32_t i_dst = s_u32(ring) + st_swz(i_row, i_ch);
+    const bool i_sz_lane = lane < 8 && col0 + 8 * (lane & 3) < p.N;
+    const __half* i_sz = (lane < 4 ? p.scales : p.zeros) + col0 + 8 * (lane & 3);
+    int i_blk = wb0, i_gpos = wb0 % bpg, i_slot = 0;
+    bool i_first = true;
     auto issue = [&]() {
-        if (!i_done) {
-            const uint32_t dst = s_u32(ring + i_slot * F::SLOT);
-#pragma unroll
-            for (int h = 0; h < (F::ROWS + 3) / 4; ++h) {
-                const int row = 4 * h + (lane >> 3), ch = lane & 7;
-                if (row < F::ROWS) {
-                    const int grow = i_blk * F::ROWS + row, col = col0 + 4 * ch;
-                    const bool ok = grow < total_rows && col < p.N;
-                    cp16(dst + st_swz(row, ch), ok ? p.Q + (size_t)grow * p.N + col : p.Q, ok ? 16 : 0);
-                }
+        if (i_blk < wb1) {
+            const uint32_t dst = i_dst + i_slot * F::SLOT;
+            if (BITS != 3 || i_row < 3) {
+                const bool ok = i_col_ok && (BITS != 2 || i_blk * F::ROWS + i_row < (p.K >> 4));
+                cp16(dst, ok ? i_src : p.Q, ok ? 16 : 0);
+                if (BITS == 8) cp16(dst + 512, i_col_ok ? i_src + 4 * (size_t)p.N : p.Q, i_col_ok ? 16 : 0);
             }
-            if ((i_gpos == 0 || i_first) && lane < 8) {    // first block of a group in this part: its scales and zeros
-                const __half* base = lane < 4 ? p.scales : p.zeros;
-                const int col = col0 + 8 * (lane & 3);
-                const bool ok = col < p.N;
-                cp16(dst + F::ROWS * 128 + lane * 16, ok ? base + (size_t)(i_blk / bpg) * p.N + col : base, ok ? 16 : 0);
-            }
+            if ((i_gpos == 0 || i_first) && lane < 8)      // first block of a group in this part: its scales and zeros
+                cp16(s_u32(ring) + i_slot * F::SLOT + F::ROWS * 128 + lane * 16, i_sz_lane ? i_sz + (size_t)(i_blk / bpg) * p.N : p.scales,
+                     i_sz_lane ? 16 : 0);
             i_first = false;
+            i_src += i_stride;
+            ++i_blk;
             if (++i_gpos == bpg) i_gpos = 0;
-            if (++i_blk >= i_end) {
-                i_cb += xcb;
-                if (i_cb >= kb1) i_done = true; else i_enter();
-            }
         }
         if (++i_slot == F::NS) i_slot = 0;
         cp_commit();
@@ -378,13 +363,16 @@ __global__ void __launch_bounds__(512, 1) stream_fwd_kernel(const StreamParams p
 #pragma unroll 1
     for (int it = 0; it < F::NS; ++it) issue();            // frozen weights only: in flight while the predecessor finishes
     {   // ask the lines this CTA will read right after the wait into L2: its slices of X, A and B
-        const int k_lo = kb0 * F::KB, kbytes = (min(kb1 * F::KB, p.K) - k_lo) * 2;
-        if (kbytes > 0) {
-            st_prefetch_l2(p.In + k_lo, (size_t)p.K * 2, p.M, kbytes, threadIdx.x, blockDim.x);
-            if (p.r > 0 && p.fused) st_prefetch_l2(p.Ldown + k_lo, (size_t)p.K * 2, p.r, kbytes, threadIdx.x, blockDim.x);
+        const int k_lo = kb0 << LKB, kbytes = (min(kb1 << LKB, p.K) - k_lo) * 2;
+        const int lines = (kbytes + 127) >> 7, rows = p.M + ((p.r > 0 && p.fused) ? p.r : 0);
+        for (int e = tid; e < rows * lines; e += nthr) {
+            const int rr = e / lines, i = e - rr * lines;
+            const __nv_bfloat16* base = rr < p.M ? p.In + (size_t)rr * p.K : p.Ldown + (size_t)(rr - p.M) * p.K;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(base + k_lo) + (size_t)i * 128));
         }
         const int c_lo = blockIdx.y * tile_c + rank * sl;
-        if (p.r > 0 && c_lo < p.N) st_prefetch_l2(p.Lup + (size_t)c_lo * p.r, 0, 1, min(sl, p.N - c_lo) * p.r * 2, threadIdx.x, blockDim.x);
+        if (p.r > 0 && c_lo < p.N && tid * 64 < min(sl, p.N - c_lo) * p.r)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(p.Lup + (size_t)c_lo * p.r + tid * 64));
     }
 
     pdl_wait();
@@ -392,22 +380,23 @@ __global__ void __launch_bounds__(512, 1) stream_fwd_kernel(const StreamParams p
     // ---- LoRA: this CTA's part of H = X A^T (k16 steps dealt to the warps, operands straight from global memory); the
     // loads of the first ST_HSTEPS steps are issued here and used once the activation slice is on its way too ----
     const bool fused = p.r > 0 && p.fused;
-    const int h_k0 = kb0 * F::KB + 16 * warp, h_ke = min(kb1 * F::KB, p.K);
+    const int h_k0 = (kb0 << LKB) + 16 * warp, h_ke = min(kb1 << LKB, p.K);
     uint32_t ha[ST_HSTEPS][4], hb[ST_HSTEPS][NT][2];
     auto h_load = [&](int kk) {
+        const __nv_bfloat16* a_lo = p.Ldown + (size_t)g * p.K + 2 * q;
+        const __nv_bfloat16* a_hi = a_lo + 8 * (size_t)p.K;
+        const __nv_bfloat16* x_lo = p.In + (size_t)g * p.K + 2 * q;
 #pragma unroll
         for (int h = 0; h < ST_HSTEPS; ++h) {
             const int k0 = kk + 16 * nw * h;
-            const bool in = fused && k0 < h_ke;
-            const __nv_bfloat16* a_lo = p.Ldown + (size_t)g * p.K + k0 + 2 * q;
-            const __nv_bfloat16* a_hi = p.Ldown + (size_t)(g + 8) * p.K + k0 + 2 * q;
-            ha[h][0] = (in && g < p.r) ? ldg32(a_lo) : 0u; ha[h][2] = (in && g < p.r) ? ldg32(a_lo + 8) : 0u;
-            ha[h][1] = (in && g + 8 < p.r) ? ldg32(a_hi) : 0u; ha[h][3] = (in && g + 8 < p.r) ? ldg32(a_hi + 8) : 0u;
+            const bool in = k0 < h_ke;
+            ha[h][0] = (in && g < p.r) ? ldg32(a_lo + k0) : 0u; ha[h][2] = (in && g < p.r) ? ldg32(a_lo + k0 + 8) : 0u;
+            ha[h][1] = (in && g + 8 < p.r) ? ldg32(a_hi + k0) : 0u; ha[h][3] = (in && g + 8 < p.r) ? ldg32(a_hi + k0 + 8) : 0u;
 #pragma unroll
             for (int tt = 0; tt < NT; ++tt) {
-                const int tok = g + 8 * tt;
-                const __nv_bfloat16* x = p.In + (size_t)tok * p.K + k0 + 2 * q;
-                hb[h][tt][0] = (in && tok < p.M) ? ldg32(x) : 0u; hb[h][tt][1] = (in && tok < p.M) ? ldg32(x + 8) : 0u;
+                const bool tin = in && g + 8 * tt < p.M;
+                hb[h][tt][0] = tin ? ldg32(x_lo + 8 * tt * (size_t)p.K + k0) : 0u;
+                hb[h][tt][1] = tin ? ldg32(x_lo + 8 * tt * (size_t)p.K + k0 + 8) : 0u;
             }
         }
     };
@@ -424,48 +413,53 @@ __global__ void __launch_bounds__(512, 1) stream_fwd_kernel(const StreamParams p
             for (int e = 0; e < 4; ++e) acc[u][tt][e] = grp[u][tt][e] = 0.f;
     float sc[4] = {0.f, 0.f, 0.f, 0.f}, cz[4] = {0.f, 0.f, 0.f, 0.f};   // this lane's four columns: scale, -scale (OFF + zero)
     int c_slot = 0;
-    if (kb0 >= kb1) st_cluster_wait();                     // (an empty range: the wait below is never reached)
-    for (int cb = kb0; cb < kb1; cb += xcb) {
-        const int ce = min(cb + xcb, kb1);
-        const int k_lo = cb * F::KB, k_hi = min(ce * F::KB, p.K);
-        const int g_first = k_lo / p.g;
-        // stage the activation slice [k_lo, k_hi): permuted for the fragment loads, plus the sums the zero-points need
+    const int lcpt = 31 - __clz(p.xc / KP), lcpp = lcpt - p.khs;          // log2: items per token row, per part of it
+    const int npass = (((nb + KH - 1) >> p.khs) + xpb - 1) / xpb;
+    if (npass == 0) st_cluster_wait();                     // (an empty range: the wait below is never reached)
+    for (int ps = 0; ps < npass; ++ps) {
+        // this warp's blocks of the pass, and what the staging needs to know about every part
+        const int pb0 = min(wb0 + ps * xpb, wb1), pb1 = min(wb1, pb0 + xpb);
+        const int wk0 = pb0 << LKB, wk1 = min(pb1 << LKB, p.K);
+        const int gf = wk0 / p.g;
+        if (cg == 0 && lane == 0) { tab[kh].k0 = wk0; tab[kh].k1 = wk1; tab[kh].gf = gf; tab[kh].nseg = wk1 > wk0 ? (wk1 - 1) / p.g - gf + 1 : 0; }
+        // stage the activations: permuted for the fragment loads, plus the sums the zero-points need
         {
-            constexpr int KP = BITS == 2 ? 16 : 8;
             constexpr int NB = BITS == 2 ? 2 : 4;          // items per round, their loads issued together
-            const int per_tok = (ce - cb) * F::KB / KP, n_items = TOKS * per_tok;
-            for (int e0 = threadIdx.x; e0 < n_items; e0 += NB * blockDim.x) {
+            const int n_items = TOKS << lcpt;
+            for (int e0 = tid; e0 < n_items; e0 += NB * nthr) {
                 uint4 v0[NB], v1[NB];
                 int tk[NB], ci[NB];
 #pragma unroll
-                for (int h = 0; h < NB; ++h) {
-                    const int e = e0 + h * blockDim.x;
-                    tk[h] = e / per_tok; ci[h] = e - tk[h] * per_tok;
-                    const int k = k_lo + ci[h] * KP;
-                    v0[h] = make_uint4(0, 0, 0, 0); v1[h] = make_uint4(0, 0, 0, 0);
-                    if (e < n_items && tk[h] < p.M && k < p.K) {
-                        v0[h] = *reinterpret_cast<const uint4*>(p.In + (size_t)tk[h] * p.K + k);
-                        if (KP == 16 && k + 8 < p.K) v1[h] = *reinterpret_cast<const uint4*>(p.In + (size_t)tk[h] * p.K + k + 8);
+                for (int j = 0; j < NB; ++j) {
+                    const int e = e0 + j * nthr;
+                    tk[j] = e >> lcpt; ci[j] = e & ((1 << lcpt) - 1);
+                    const int h = ci[j] >> lcpp, cl = ci[j] & ((1 << lcpp) - 1);
+                    const int hb0 = kb0 + ((nb * h) >> p.khs), hb1 = kb0 + ((nb * (h + 1)) >> p.khs);
+                    const int k = (min(hb0 + ps * xpb, hb1) << LKB) + cl * KP, kend = min(min(hb1, hb0 + (ps + 1) * xpb) << LKB, p.K);
+                    v0[j] = make_uint4(0, 0, 0, 0); v1[j] = make_uint4(0, 0, 0, 0);
+                    if (e < n_items && tk[j] < p.M && k < kend) {
+                        v0[j] = *reinterpret_cast<const uint4*>(p.In + (size_t)tk[j] * p.K + k);
+                        if (KP == 16 && k + 8 < kend) v1[j] = *reinterpret_cast<const uint4*>(p.In + (size_t)tk[j] * p.K + k + 8);
                     }
                 }
 #pragma unroll
-                for (int h = 0; h < NB; ++h) {
-                    if (e0 + h * blockDim.x >= n_items) break;
-                    uint8_t* dst = xs + tk[h] * xp + ci[h] * (2 * KP);
+                for (int j = 0; j < NB; ++j) {
+                    if (e0 + j * nthr >= n_items) break;
+                    uint8_t* dst = xs + tk[j] * xp + ci[j] * (2 * KP);
                     if constexpr (BITS == 2) {             // (x0,x8) (x1,x9) ... (x7,x15)
-                        *reinterpret_cast<uint4*>(dst) = make_uint4(__byte_perm(v0[h].x, v1[h].x, 0x5410), __byte_perm(v0[h].x, v1[h].x, 0x7632),
-                                                                    __byte_perm(v0[h].y, v1[h].y, 0x5410), __byte_perm(v0[h].y, v1[h].y, 0x7632));
-                        *reinterpret_cast<uint4*>(dst + 16) = make_uint4(__byte_perm(v0[h].z, v1[h].z, 0x5410), __byte_perm(v0[h].z, v1[h].z, 0x7632),
-                                                                         __byte_perm(v0[h].w, v1[h].w, 0x5410), __byte_perm(v0[h].w, v1[h].w, 0x7632));
-                        sxc[tk[h] * (p.xc / 8) + 2 * ci[h]] = st_sum8(v0[h]);
-                        sxc[tk[h] * (p.xc / 8) + 2 * ci[h] + 1] = st_sum8(v1[h]);
+                        *reinterpret_cast<uint4*>(dst) = make_uint4(__byte_perm(v0[j].x, v1[j].x, 0x5410), __byte_perm(v0[j].x, v1[j].x, 0x7632),
+                                                                    __byte_perm(v0[j].y, v1[j].y, 0x5410), __byte_perm(v0[j].y, v1[j].y, 0x7632));
+                        *reinterpret_cast<uint4*>(dst + 16) = make_uint4(__byte_perm(v0[j].z, v1[j].z, 0x5410), __byte_perm(v0[j].z, v1[j].z, 0x7632),
+                                                                         __byte_perm(v0[j].w, v1[j].w, 0x5410), __byte_perm(v0[j].w, v1[j].w, 0x7632));
+                        sxc[tk[j] * (p.xc >> 3) + 2 * ci[j]] = st_sum8(v0[j]);
+                        sxc[tk[j] * (p.xc >> 3) + 2 * ci[j] + 1] = st_sum8(v1[j]);
                     } else {
-                        *reinterpret_cast<uint4*>(dst) = BITS == 8 ? v0[h] : st_permute8(v0[h]);
-                        sxc[tk[h] * (p.xc / 8) + ci[h]] = st_sum8(v0[h]);
+                        *reinterpret_cast<uint4*>(dst) = BITS == 8 ? v0[j] : st_permute8(v0[j]);
+                        sxc[tk[j] * (p.xc >> 3) + ci[j]] = st_sum8(v0[j]);
                     }
                 }
             }
-            if (cb == kb0 && fused) {                      // the down-projection's MMAs, with the slice's loads behind them
+            if (ps == 0 && fused) {                        // the down-projection's MMAs, with the activations' loads behind them
                 float ah[NT][4];
 #pragma unroll
                 for (int tt = 0; tt < NT; ++tt) ah[tt][0] = ah[tt][1] = ah[tt][2] = ah[tt][3] = 0.f;
@@ -481,37 +475,48 @@ __global__ void __launch_bounds__(512, 1) stream_fwd_kernel(const StreamParams p
                 st_store_hp<NT>(ah, hp, warp, g, q);
             }
             __syncthreads();
-            const int nseg = (k_hi - 1) / p.g - g_first + 1;
-            for (int e = threadIdx.x; e < KH * nseg * TOKS; e += blockDim.x) {
-                const int tok = e % TOKS, sg = (e / TOKS) % nseg, h = e / (TOKS * nseg);
-                const int n = ce - cb;
-                const int p_lo = (cb + st_part(n, h, p.khs)) * F::KB, p_hi = min((cb + st_part(n, h + 1, p.khs)) * F::KB, p.K);
-                const int a = max(p_lo, (g_first + sg) * p.g), b = min(p_hi, (g_first + sg + 1) * p.g);
-                float sum = 0.f;
-                for (int c8 = (a - k_lo) / 8; c8 < (b - k_lo) / 8; ++c8) sum += sxc[tok * (p.xc / 8) + c8];
-                sxs[(h * (xcb + 1) + sg) * TOKS + tok] = sum;
+            {   // sums per (part, group segment): four lanes per (token, segment), segments numbered through the parts
+                int n_all = 0;
+                for (int h = 0; h < KH; ++h) n_all += tab[h].nseg;
+                const int total = n_all << LTOKS;
+                for (int base = 0; base < total; base += nthr >> 2) {      // the same trip count for every thread
+                    const int task = base + (tid >> 2), sub = tid & 3;
+                    const bool on = task < total;
+                    const int tok = task & (TOKS - 1);
+                    int h = 0, sg = on ? task >> LTOKS : 0;
+                    while (on && sg >= tab[h].nseg) { sg -= tab[h].nseg; ++h; }
+                    const PartInfo pi = tab[h];
+                    const int a = max(pi.k0, (pi.gf + sg) * p.g), b = min(pi.k1, (pi.gf + sg + 1) * p.g);
+                    const float* src = sxc + tok * (p.xc >> 3) + ((h << lcpp) * KP + (a - pi.k0)) / 8;
+                    float sum = 0.f;
+                    if (on)
+                        for (int c8 = sub; c8 < (b - a) >> 3; c8 += 4) sum += src[c8];
+                    sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+                    sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+                    if (on && sub == 0) sxs[(h * (xpb + 1) + sg) * TOKS + tok] = sum;
+                }
             }
-            if (cb == kb0 && fused) {
-                for (int e = threadIdx.x; e < 256; e += blockDim.x) {
+            if (ps == 0 && fused) {
+                for (int e = tid; e < 256; e += nthr) {
                     float h = 0.f;
                     for (int w = 0; w < nw; ++w) h += hp[w * 256 + e];
                     hs[e] = h;
                 }
             }
             __syncthreads();
-            if (cb == kb0) {
+            if (ps == 0) {
                 st_cluster_wait();                         // every CTA of the cluster is running: its shared memory may be written
                 if (fused) st_push_h(rl, hs, rank, p.ks);
             }
         }
-        const int b0 = cb + st_part(ce - cb, kh, p.khs), b1 = cb + st_part(ce - cb, kh + 1, p.khs);
-        int gpos = b0 < b1 ? b0 % bpg : 0, grpi = b0 < b1 ? b0 / bpg : 0;
-#pragma unroll 1
-        for (int blk = b0; blk < b1; ++blk) {
+        int gpos = pb0 - gf * bpg, grpi = gf;
+        const uint8_t* xw = xs + (kh * xpb << (LKB + 1)) + (BITS == 2 ? 32 * q : (BITS == 8 ? 8 * q : 16 * q)) + g * xp;
+#pragma unroll 2
+        for (int blk = pb0; blk < pb1; ++blk) {
             cp_wait<F::NS - 1>();
             __syncwarp();
             const uint8_t* slot = ring + c_slot * F::SLOT;
-            if (gpos == 0 || blk == b0) {                  // a new group: this lane's scales and zero-points
+            if (gpos == 0 || blk == wb0) {                 // a new group: this lane's scales and zero-points
                 const uint2 s2 = *reinterpret_cast<const uint2*>(slot + F::ROWS * 128 + 8 * g);
                 const uint2 z2 = *reinterpret_cast<const uint2*>(slot + F::ROWS * 128 + 64 + 8 * g);
                 const float2 sa = __half22float2(*reinterpret_cast<const __half2*>(&s2.x)), sb = __half22float2(*reinterpret_cast<const __half2*>(&s2.y));
@@ -523,41 +528,40 @@ __global__ void __launch_bounds__(512, 1) stream_fwd_kernel(const StreamParams p
             st_load_words<BITS>(slot, g, q, w);
             // activation fragments: token g (+ 8), this lane's quarter of the block
             uint32_t xf[NT][F::NPAIR];
-            const int bl = blk - cb;
+            const uint8_t* xb = xw + ((blk - pb0) << (LKB + 1));
 #pragma unroll
             for (int tt = 0; tt < NT; ++tt) {
-                const uint8_t* xr = xs + (g + 8 * tt) * xp;
+                const uint8_t* xr = xb + 8 * tt * xp;
                 if constexpr (BITS == 2) {
-                    const uint4 v0 = *reinterpret_cast<const uint4*>(xr + bl * 128 + 32 * q);
-                    const uint4 v1 = *reinterpret_cast<const uint4*>(xr + bl * 128 + 32 * q + 16);
+                    const uint4 v0 = *reinterpret_cast<const uint4*>(xr);
+                    const uint4 v1 = *reinterpret_cast<const uint4*>(xr + 16);
                     xf[tt][0] = v0.x; xf[tt][1] = v0.y; xf[tt][2] = v0.z; xf[tt][3] = v0.w;
                     xf[tt][4] = v1.x; xf[tt][5] = v1.y; xf[tt][6] = v1.z; xf[tt][7] = v1.w;
                 } else if constexpr (BITS == 8) {
-                    const uint2 v0 = *reinterpret_cast<const uint2*>(xr + bl * 64 + 8 * q);
-                    const uint2 v1 = *reinterpret_cast<const uint2*>(xr + bl * 64 + 32 + 8 * q);
+                    const uint2 v0 = *reinterpret_cast<const uint2*>(xr);
+                    const uint2 v1 = *reinterpret_cast<const uint2*>(xr + 32);
                     xf[tt][0] = v0.x; xf[tt][1] = v0.y; xf[tt][2] = v1.x; xf[tt][3] = v1.y;
                 } else {
-                    const uint4 v0 = *reinterpret_cast<const uint4*>(xr + bl * 64 + 16 * q);
+                    const uint4 v0 = *reinterpret_cast<const uint4*>(xr);
                     xf[tt][0] = v0.x; xf[tt][1] = v0.y; xf[tt][2] = v0.z; xf[tt][3] = v0.w;
                 }
             }
             // two tiles of 16 columns: rows g / g + 8 of tile u are columns 4g + 2u / 4g + 2u + 1
+            uint32_t pc[4][F::NPAIR];                      // [column i of the lane's four][pair]
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                uint32_t pa[F::NPAIR], pb[F::NPAIR];
-                st_unpack<BITS>(st_comp(w[0], 2 * u), F::NLD > 1 ? st_comp(w[F::NLD - 1], 2 * u) : 0u, q, pa);
-                st_unpack<BITS>(st_comp(w[0], 2 * u + 1), F::NLD > 1 ? st_comp(w[F::NLD - 1], 2 * u + 1) : 0u, q, pb);
+            for (int i = 0; i < 4; ++i) st_unpack<BITS>(st_comp(w[0], i), F::NLD > 1 ? st_comp(w[F::NLD - 1], i) : 0u, q, pc[i]);
 #pragma unroll
-                for (int s = 0; s < F::STEPS; ++s)
+            for (int s = 0; s < F::STEPS; ++s)             // MMAs into the same accumulator are 2 NT instructions apart
+#pragma unroll
+                for (int u = 0; u < 2; ++u)
 #pragma unroll
                     for (int tt = 0; tt < NT; ++tt)
-                        st_mma(grp[u][tt], pa[2 * s], pb[2 * s], pa[2 * s + 1], pb[2 * s + 1], xf[tt][2 * s], xf[tt][2 * s + 1]);
-            }
-            if (gpos == bpg - 1 || blk + 1 == b1) {        // end of a group segment: scale, correct, start afresh
-                const float* sxr = sxs + (kh * (xcb + 1) + grpi - g_first) * TOKS;
+                        st_mma(grp[u][tt], pc[2 * u][2 * s], pc[2 * u + 1][2 * s], pc[2 * u][2 * s + 1], pc[2 * u + 1][2 * s + 1], xf[tt][2 * s], xf[tt][2 * s + 1]);
+            if (gpos == bpg - 1 || blk + 1 == pb1) {       // end of a group segment: scale, correct, start afresh
+                const float* sxr = sxs + (kh * (xpb + 1) + grpi - gf) * TOKS + 2 * q;
 #pragma unroll
                 for (int tt = 0; tt < NT; ++tt) {
-                    const float2 sx = *reinterpret_cast<const float2*>(sxr + 8 * tt + 2 * q);
+                    const float2 sx = *reinterpret_cast<const float2*>(sxr + 8 * tt);
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
                         acc[u][tt][0] += sc[2 * u] * grp[u][tt][0] + cz[2 * u] * sx.x;
@@ -573,7 +577,7 @@ __global__ void __launch_bounds__(512, 1) stream_fwd_kernel(const StreamParams p
             __syncwarp();
             issue();
         }
-        if (cb + xcb < kb1) __syncthreads();               // the slice may be overwritten
+        if (ps + 1 < npass) __syncthreads();               // the staged activations may be overwritten
     }
     // accumulator element (u, tt, e): column 4g + 2u + (e >> 1) of this warp's 32, token 2q + (e & 1) + 8 tt; sent to the
     // CTA that finishes that column
@@ -589,29 +593,32 @@ __global__ void __launch_bounds__(512, 1) stream_fwd_kernel(const StreamParams p
 
 // ------------------------------------------------------------------------------------------------------------
 // Backward: dX = dY W + s G A.  CTA (rank, tile): output features [FW wc tile, + FW wc), contraction stages [st0, st1)
-// of 32 SU packed columns.  Warp (fw, kh): FW features (all inside one group) and part kh of the stages of every staged
-// slice of dY.
+// of 32 SU packed columns.  Warp (fw, kh): FW features (all inside one group) and the kh-th of KH consecutive parts of
+// [st0, st1).  The slices of dY of the parts are staged side by side, xps stages of every part per pass.
 // ------------------------------------------------------------------------------------------------------------
 template <int BITS, int NT>
 __global__ void __launch_bounds__(512, 1) stream_bwd_kernel(const StreamParams p) {
     using F = Fmt<BITS>;
     constexpr int TOKS = 8 * NT;
     constexpr int NTILE = F::BPAIR / 2;                    // 16-feature MMA tiles per warp
+    constexpr int LSW = BITS == 2 ? 7 : 5;                 // log2 of the packed columns per stage
     pdl_launch_dependents();
     st_cluster_arrive_relaxed();                           // waited for before the first store into a peer's shared memory
     extern __shared__ __align__(128) uint8_t smem[];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, q = lane & 3;
-    const int nw = blockDim.x >> 5, tile_c = F::FW * p.wc, sl = tile_c / p.ks;
-    const int fw = warp % p.wc, kh = warp / p.wc;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, q = lane & 3;
+    const int nthr = blockDim.x, nw = nthr >> 5, tile_c = F::FW * p.wc, sl = tile_c >> p.lks, KH = 1 << p.khs;
+    const int fw = warp & (p.wc - 1), kh = warp >> p.lwc;
     const int rank = (int)st_cluster_rank();
     const int tile_f0 = blockIdx.y * tile_c, f0 = tile_f0 + F::FW * fw;
     const bool live = f0 < p.K;                            // a warp beyond the last feature only keeps the barriers company
     const int row0 = f0 * BITS / 32;
-    const int sw = 32 * F::SU;                             // packed columns per stage
-    const int nst = (p.N + sw - 1) / sw;
-    const int st0 = nst * rank / p.ks, st1 = nst * (rank + 1) / p.ks;
+    const int nst = (p.N + (1 << LSW) - 1) >> LSW;
+    const int st0 = (nst * rank) >> p.lks, st1 = (nst * (rank + 1)) >> p.lks, ns = st1 - st0;
+    const int ws0 = st0 + ((ns * kh) >> p.khs), ws1 = st0 + ((ns * (kh + 1)) >> p.khs);
     const int xp = p.xc * 2 + 64;
-    const int xcs = p.xc / sw;                             // stages per staged slice
+    const int xps = (p.xc >> LSW) >> p.khs;                // stages of a part staged per pass
+    const int gk0 = tile_f0 / p.g;                         // group of the CTA's first feature
+    const int ngroups = p.K / p.g;
     const int copy = p.copies > 1 ? (f0 - tile_f0) / p.g : 0;
     uint8_t* ring = smem + warp * (F::BNS * F::BSLOT);
     uint8_t* ys = smem + nw * (F::BNS * F::BSLOT);         // [copies][TOKS][xp] scaled, permuted slices of dY
@@ -626,42 +633,22 @@ __global__ void __launch_bounds__(512, 1) stream_bwd_kernel(const StreamParams p
     RecvLayout rl;
     rl.part_addr = s_u32(recv_part); rl.h_addr = s_u32(recv_h); rl.sls = p.sls; rl.khs = p.khs;
 
-    int i_cs = st0, i_stg = 0, i_end = 0, i_slot = 0;
-    bool i_done = st0 >= st1 || !live;
-    auto i_enter = [&]() {
-        while (!i_done) {
-            const int n = min(i_cs + xcs, st1) - i_cs;
-            i_stg = i_cs + st_part(n, kh, p.khs);
-            i_end = i_cs + st_part(n, kh + 1, p.khs);
-            if (i_stg < i_end) return;
-            i_cs += xcs;
-            if (i_cs >= st1) i_done = true;
-        }
-    };
-    i_enter();
+    // ---- the copy side of this warp: stages ws0 .. ws1 - 1 in order, BNS ahead of the arithmetic ----
+    const int i_row = BITS == 2 ? 0 : lane >> 3;
+    const int i_coff = BITS == 2 ? 32 * (lane >> 3) + 4 * (lane & 7) : 4 * (lane & 7);   // column inside the stage
+    const uint32_t* i_src = p.Q + (size_t)(row0 + i_row) * p.N;
+    const uint32_t i_dst = s_u32(ring) + (BITS == 2 ? lane * 16 : st_swz(i_row, lane & 7));
+    int i_stg = ws0, i_slot = 0;
     auto issue = [&]() {
-        if (!i_done) {
-            const int cbase = i_stg * sw;
-            const uint32_t dst = s_u32(ring + i_slot * F::BSLOT);
-            if constexpr (BITS == 2) {
-                const int col = cbase + 32 * (lane >> 3) + 4 * (lane & 7);
-                const bool ok = col < p.N;
-                cp16(dst + lane * 16, ok ? p.Q + (size_t)row0 * p.N + col : p.Q, ok ? 16 : 0);
-            } else {
-#pragma unroll
-                for (int h = 0; h < (F::BROWS + 3) / 4; ++h) {
-                    const int row = 4 * h + (lane >> 3), ch = lane & 7;
-                    if (row < F::BROWS) {
-                        const int col = cbase + 4 * ch;
-                        const bool ok = col < p.N;
-                        cp16(dst + st_swz(row, ch), ok ? p.Q + (size_t)(row0 + row) * p.N + col : p.Q, ok ? 16 : 0);
-                    }
-                }
+        if (i_stg < ws1 && live) {
+            const uint32_t dst = i_dst + i_slot * F::BSLOT;
+            const int col = (i_stg << LSW) + i_coff;
+            const bool ok = col < p.N;
+            if (BITS != 3 || i_row < 3) {
+                cp16(dst, ok ? i_src + col : p.Q, ok ? 16 : 0);
+                if (BITS == 8) cp16(dst + 512, ok ? i_src + 4 * (size_t)p.N + col : p.Q, ok ? 16 : 0);
             }
-            if (++i_stg >= i_end) {
-                i_cs += xcs;
-                if (i_cs >= st1) i_done = true; else i_enter();
-            }
+            ++i_stg;
         }
         if (++i_slot == F::BNS) i_slot = 0;
         cp_commit();
@@ -669,23 +656,25 @@ __global__ void __launch_bounds__(512, 1) stream_bwd_kernel(const StreamParams p
 #pragma unroll 1
     for (int it = 0; it < F::BNS; ++it) issue();
 
-    const int n_lo_cta = st0 * sw, n_hi_cta = min(st1 * sw, p.N);
-    const int ngroups = p.K / p.g;
+    const int n_lo_cta = st0 << LSW, n_hi_cta = min(st1 << LSW, p.N);
     {   // ask the lines this CTA will read right after the wait into L2: its slices of dY, B, A and of the group parameters
-        const int nbytes = (n_hi_cta - n_lo_cta) * 2;
-        if (nbytes > 0) {
-            st_prefetch_l2(p.In + n_lo_cta, (size_t)p.N * 2, p.M, nbytes, threadIdx.x, blockDim.x);
-            if (p.r > 0 && p.fused) st_prefetch_l2(p.Ldown + (size_t)n_lo_cta * p.r, 0, 1, nbytes * p.r, threadIdx.x, blockDim.x);
-            for (int c = 0; c < p.copies; ++c) {
-                const int gk = tile_f0 / p.g + c;
-                if (gk < ngroups) {
-                    st_prefetch_l2(p.scales + (size_t)gk * p.N + n_lo_cta, 0, 1, nbytes, threadIdx.x, blockDim.x);
-                    st_prefetch_l2(p.zeros + (size_t)gk * p.N + n_lo_cta, 0, 1, nbytes, threadIdx.x, blockDim.x);
-                }
+        const int nbytes = (n_hi_cta - n_lo_cta) * 2, lines = (nbytes + 127) >> 7;
+        const int rows = p.M + 2 * p.copies;
+        for (int e = tid; e < rows * lines; e += nthr) {
+            const int rr = e / lines, i = e - rr * lines;
+            const char* base;
+            if (rr < p.M) base = reinterpret_cast<const char*>(p.In + (size_t)rr * p.N + n_lo_cta);
+            else {
+                const int c = (rr - p.M) >> 1, gk = min(gk0 + c, ngroups - 1);
+                base = reinterpret_cast<const char*>(((rr - p.M) & 1 ? p.zeros : p.scales) + (size_t)gk * p.N + n_lo_cta);
             }
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(base + (size_t)i * 128));
         }
+        if (p.r > 0 && p.fused)
+            for (int e = tid; e * 64 < (n_hi_cta - n_lo_cta) * p.r; e += nthr)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(p.Ldown + (size_t)n_lo_cta * p.r + (size_t)e * 64));
         const int c_lo = tile_f0 + rank * sl;
-        if (p.r > 0 && c_lo < p.K) st_prefetch_l2(p.Lup + c_lo, (size_t)p.K * 2, p.r, min(sl, p.K - c_lo) * 2, threadIdx.x, blockDim.x);
+        if (p.r > 0 && c_lo < p.K && tid < p.r) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.Lup + (size_t)tid * p.K + c_lo));
     }
 
     pdl_wait();
@@ -700,10 +689,10 @@ __global__ void __launch_bounds__(512, 1) stream_bwd_kernel(const StreamParams p
 #pragma unroll
         for (int h = 0; h < ST_HSTEPS; ++h) {
             const int nb = nn + 16 * nw * h;
-            const bool in = fused && nb < n_hi_cta;
+            const bool in = nb < n_hi_cta;
             const bool v0 = in && nb + g < p.N, v1 = in && nb + 8 + g < p.N;
             const __nv_bfloat16* b_lo = p.Ldown + (size_t)(nb + g) * p.r + 2 * q;
-            const __nv_bfloat16* b_hi = p.Ldown + (size_t)(nb + 8 + g) * p.r + 2 * q;
+            const __nv_bfloat16* b_hi = b_lo + 8 * p.r;
             ha[h][0] = v0 ? ldg32(b_lo) : 0u; ha[h][2] = v1 ? ldg32(b_hi) : 0u;
             ha[h][1] = (v0 && p.r > 8) ? ldg32(b_lo + 8) : 0u; ha[h][3] = (v1 && p.r > 8) ? ldg32(b_hi + 8) : 0u;
 #pragma unroll
@@ -717,7 +706,7 @@ __global__ void __launch_bounds__(512, 1) stream_bwd_kernel(const StreamParams p
     };
     if (fused) h_load(h_n0);
     st_stage_lup<true>(p, lup, hfull, tile_c, rank);
-    for (int e = threadIdx.x; e < nw * 32; e += blockDim.x) zp[e] = 0.f;
+    for (int e = tid; e < nw * 32; e += nthr) zp[e] = 0.f;
 
     float acc[NTILE][NT][4];
 #pragma unroll
@@ -725,42 +714,51 @@ __global__ void __launch_bounds__(512, 1) stream_bwd_kernel(const StreamParams p
 #pragma unroll
         for (int tt = 0; tt < NT; ++tt) acc[t][tt][0] = acc[t][tt][1] = acc[t][tt][2] = acc[t][tt][3] = 0.f;
     int c_slot = 0;
-    if (st0 >= st1) st_cluster_wait();                     // (an empty range: the wait below is never reached)
-    for (int cs = st0; cs < st1; cs += xcs) {
-        const int ce = min(cs + xcs, st1);
-        const int n_lo = cs * sw, n_hi = min(ce * sw, p.N);
-        // stage the slice of dY, once per group the CTA's features span, scaled by that group's scales (one rounding)
+    const int lcpt = 31 - __clz(p.xc >> 3), lcpp = lcpt - p.khs;          // log2: 8-column items per token row, per part of it
+    const int npass = (((ns + KH - 1) >> p.khs) + xps - 1) / xps;
+    if (npass == 0) st_cluster_wait();                     // (an empty range: the wait below is never reached)
+    for (int ps = 0; ps < npass; ++ps) {
+        const int pb0 = min(ws0 + ps * xps, ws1), pb1 = min(ws1, pb0 + xps);     // this warp's stages of the pass
+        // stage the slices of dY, once per group the CTA's features span, scaled by that group's scales (one rounding)
         {
-            const int per_tok = (ce - cs) * sw / 8;
-            for (int e = threadIdx.x; e < TOKS * per_tok; e += blockDim.x) {
-                const int tok = e / per_tok, ci = e - tok * per_tok;
-                const int n = n_lo + ci * 8;
-                const bool ok = tok < p.M && n < p.N;
-                uint4 v = make_uint4(0, 0, 0, 0), s8[2];
-                s8[0] = s8[1] = make_uint4(0, 0, 0, 0);
-                if (ok) {
-                    v = *reinterpret_cast<const uint4*>(p.In + (size_t)tok * p.N + n);
+            const int n_items = TOKS << lcpt;
+            for (int e0 = tid; e0 < n_items; e0 += 2 * nthr) {                   // two items per round, loads first
+                uint4 v[2], s8[2][2];
+                int tk[2], ci[2];
 #pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        const int gk = tile_f0 / p.g + c;
-                        if (c < p.copies && gk < ngroups) s8[c] = *reinterpret_cast<const uint4*>(p.scales + (size_t)gk * p.N + n);
+                for (int j = 0; j < 2; ++j) {
+                    const int e = e0 + j * nthr;
+                    tk[j] = e >> lcpt; ci[j] = e & ((1 << lcpt) - 1);
+                    const int h = ci[j] >> lcpp, cl = ci[j] & ((1 << lcpp) - 1);
+                    const int hs0 = st0 + ((ns * h) >> p.khs), hs1 = st0 + ((ns * (h + 1)) >> p.khs);
+                    const int n = (min(hs0 + ps * xps, hs1) << LSW) + cl * 8, nend = min(min(hs1, hs0 + (ps + 1) * xps) << LSW, p.N);
+                    v[j] = s8[j][0] = s8[j][1] = make_uint4(0, 0, 0, 0);
+                    if (e < n_items && tk[j] < p.M && n < nend) {
+                        v[j] = *reinterpret_cast<const uint4*>(p.In + (size_t)tk[j] * p.N + n);
+#pragma unroll
+                        for (int c = 0; c < 2; ++c)
+                            if (c < p.copies && gk0 + c < ngroups) s8[j][c] = *reinterpret_cast<const uint4*>(p.scales + (size_t)(gk0 + c) * p.N + n);
                     }
                 }
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    if (c >= p.copies) break;
-                    const float2 s0 = __half22float2(*reinterpret_cast<const __half2*>(&s8[c].x)), s1 = __half22float2(*reinterpret_cast<const __half2*>(&s8[c].y));
-                    const float2 s2 = __half22float2(*reinterpret_cast<const __half2*>(&s8[c].z)), s3 = __half22float2(*reinterpret_cast<const __half2*>(&s8[c].w));
-                    const __nv_bfloat162 o0 = __floats2bfloat162_rn(bf16_lo(v.x) * s0.x, bf16_hi(v.x) * s0.y);
-                    const __nv_bfloat162 o1 = __floats2bfloat162_rn(bf16_lo(v.y) * s1.x, bf16_hi(v.y) * s1.y);
-                    const __nv_bfloat162 o2 = __floats2bfloat162_rn(bf16_lo(v.z) * s2.x, bf16_hi(v.z) * s2.y);
-                    const __nv_bfloat162 o3 = __floats2bfloat162_rn(bf16_lo(v.w) * s3.x, bf16_hi(v.w) * s3.y);
-                    const uint4 o = make_uint4(*reinterpret_cast<const uint32_t*>(&o0), *reinterpret_cast<const uint32_t*>(&o1),
-                                               *reinterpret_cast<const uint32_t*>(&o2), *reinterpret_cast<const uint32_t*>(&o3));
-                    *reinterpret_cast<uint4*>(ys + (c * TOKS + tok) * xp + ci * 16) = st_permute8(o);
+                for (int j = 0; j < 2; ++j) {
+                    if (e0 + j * nthr >= n_items) break;
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        if (c >= p.copies) break;
+                        const float2 s0 = __half22float2(*reinterpret_cast<const __half2*>(&s8[j][c].x)), s1 = __half22float2(*reinterpret_cast<const __half2*>(&s8[j][c].y));
+                        const float2 s2 = __half22float2(*reinterpret_cast<const __half2*>(&s8[j][c].z)), s3 = __half22float2(*reinterpret_cast<const __half2*>(&s8[j][c].w));
+                        const __nv_bfloat162 o0 = __floats2bfloat162_rn(bf16_lo(v[j].x) * s0.x, bf16_hi(v[j].x) * s0.y);
+                        const __nv_bfloat162 o1 = __floats2bfloat162_rn(bf16_lo(v[j].y) * s1.x, bf16_hi(v[j].y) * s1.y);
+                        const __nv_bfloat162 o2 = __floats2bfloat162_rn(bf16_lo(v[j].z) * s2.x, bf16_hi(v[j].z) * s2.y);
+                        const __nv_bfloat162 o3 = __floats2bfloat162_rn(bf16_lo(v[j].w) * s3.x, bf16_hi(v[j].w) * s3.y);
+                        const uint4 o = make_uint4(*reinterpret_cast<const uint32_t*>(&o0), *reinterpret_cast<const uint32_t*>(&o1),
+                                                   *reinterpret_cast<const uint32_t*>(&o2), *reinterpret_cast<const uint32_t*>(&o3));
+                        *reinterpret_cast<uint4*>(ys + (c * TOKS + tk[j]) * xp + ci[j] * 16) = st_permute8(o);
+                    }
                 }
             }
-            if (cs == st0 && fused) {                      // the down-projection's MMAs, with the slice's loads behind them
+            if (ps == 0 && fused) {                        // the down-projection's MMAs, with the slice's loads behind them
                 float ag[NT][4];
 #pragma unroll
                 for (int tt = 0; tt < NT; ++tt) ag[tt][0] = ag[tt][1] = ag[tt][2] = ag[tt][3] = 0.f;
@@ -778,21 +776,22 @@ __global__ void __launch_bounds__(512, 1) stream_bwd_kernel(const StreamParams p
                 st_store_hp<NT>(ag, hp, warp, g, q);
             }
             __syncthreads();
-            if (cs == st0 && fused) {
-                for (int e = threadIdx.x; e < 256; e += blockDim.x) {
+            if (ps == 0 && fused) {
+                for (int e = tid; e < 256; e += nthr) {
                     float h = 0.f;
                     for (int w = 0; w < nw; ++w) h += hp[w * 256 + e];
                     hs[e] = h;
                 }
             }
-            // zero-point term: sum_n dYs[m, n] (OFF + z[G, n]) as one MMA row; 32-column units dealt to the warps
+            // zero-point term: sum_n dYs[m, n] (OFF + z[G, n]) as one MMA row; the warps of a part share its 32-column units
+            const int un_end = ((min(pb1 << LSW, p.N) - (pb0 << LSW)) + 31) >> 5;
             for (int c = 0; c < p.copies; ++c) {
-                const int gk = tile_f0 / p.g + c;
+                const int gk = gk0 + c;
                 float za[NT][4];
 #pragma unroll
                 for (int tt = 0; tt < NT; ++tt) za[tt][0] = za[tt][1] = za[tt][2] = za[tt][3] = 0.f;
-                for (int un = warp; un < (n_hi - n_lo + 31) / 32; un += nw) {
-                    const int n = n_lo + 32 * un + 8 * q;
+                for (int un = fw; un < un_end; un += p.wc) {
+                    const int n = (pb0 << LSW) + 32 * un + 8 * q;
                     uint32_t zr[4] = {0u, 0u, 0u, 0u};     // (z0,z4) (z1,z5) (z2,z6) (z3,z7) as bf16 of OFF + z
                     if (g == 0 && n < p.N && gk < ngroups) {
                         const uint4 z8 = *reinterpret_cast<const uint4*>(p.zeros + (size_t)gk * p.N + n);
@@ -805,7 +804,7 @@ __global__ void __launch_bounds__(512, 1) stream_bwd_kernel(const StreamParams p
                     }
 #pragma unroll
                     for (int tt = 0; tt < NT; ++tt) {
-                        const uint4 xv = *reinterpret_cast<const uint4*>(ys + (c * TOKS + g + 8 * tt) * xp + (un * 4 + q) * 16);
+                        const uint4 xv = *reinterpret_cast<const uint4*>(ys + (c * TOKS + g + 8 * tt) * xp + (((kh << lcpp) + un * 4 + q) << 4));
                         st_mma(za[tt], zr[0], 0u, zr[1], 0u, xv.x, xv.y);
                         st_mma(za[tt], zr[2], 0u, zr[3], 0u, xv.z, xv.w);
                     }
@@ -818,24 +817,24 @@ __global__ void __launch_bounds__(512, 1) stream_bwd_kernel(const StreamParams p
                     }
                 }
             }
-        }
-        if (cs == st0) {
-            st_cluster_wait();                             // every CTA of the cluster is running: its shared memory may be written
-            if (fused) {
-                __syncthreads();                           // hs is complete
-                st_push_h(rl, hs, rank, p.ks);
+            if (ps == 0) {
+                st_cluster_wait();                         // every CTA of the cluster is running: its shared memory may be written
+                if (fused) {
+                    __syncthreads();                       // hs is complete
+                    st_push_h(rl, hs, rank, p.ks);
+                }
             }
         }
         if (live) {
-            const int s0 = cs + st_part(ce - cs, kh, p.khs), s1 = cs + st_part(ce - cs, kh + 1, p.khs);
-#pragma unroll 1
-            for (int stg = s0; stg < s1; ++stg) {
+            const uint8_t* yw = ys + (copy * TOKS + g) * xp + (((kh << lcpp) + q) << 4);
+#pragma unroll 2
+            for (int stg = pb0; stg < pb1; ++stg) {
                 cp_wait<F::BNS - 1>();
                 __syncwarp();
                 const uint8_t* slot = ring + c_slot * F::BSLOT;
 #pragma unroll
                 for (int su = 0; su < F::SU; ++su) {
-                    const int ul = (stg - cs) * F::SU + su;    // 32-column unit inside the staged slice
+                    const int ul = (stg - pb0) * F::SU + su;   // 32-column unit inside this part's staged slice
                     uint32_t mx[4][F::BPAIR];                  // [column i of the lane's four][pair], transposed
                     if constexpr (BITS == 2) {
                         const uint4 w = *reinterpret_cast<const uint4*>(slot + su * 128 + g * 16);
@@ -857,7 +856,7 @@ __global__ void __launch_bounds__(512, 1) stream_bwd_kernel(const StreamParams p
                     }
 #pragma unroll
                     for (int tt = 0; tt < NT; ++tt) {
-                        const uint4 xv = *reinterpret_cast<const uint4*>(ys + (copy * TOKS + g + 8 * tt) * xp + (ul * 4 + q) * 16);
+                        const uint4 xv = *reinterpret_cast<const uint4*>(yw + 8 * tt * xp + (ul << 6));
 #pragma unroll
                         for (int t = 0; t < NTILE; ++t) {
                             st_mma(acc[t][tt], mx[0][2 * t], mx[0][2 * t + 1], mx[1][2 * t], mx[1][2 * t + 1], xv.x, xv.y);
@@ -872,10 +871,10 @@ __global__ void __launch_bounds__(512, 1) stream_bwd_kernel(const StreamParams p
         }
         __syncthreads();
     }
-    for (int e = threadIdx.x; e < 32; e += blockDim.x) {   // zero-point sums of the whole range, warps added in order
+    if (tid < 32) {                                        // zero-point sums of the whole range, warps added in order
         float z = 0.f;
-        for (int w = 0; w < nw; ++w) z += zp[w * 32 + e];
-        zc[e] = z;
+        for (int w = 0; w < nw; ++w) z += zp[w * 32 + tid];
+        zc[tid] = z;
     }
     __syncthreads();
     // accumulator element (t, tt, e): MMA row g + 8 (e >> 1) of tile t = matrix 2t + (e >> 1), column g of it; token
@@ -897,6 +896,33 @@ __global__ void __launch_bounds__(512, 1) stream_bwd_kernel(const StreamParams p
                 st_push2(rl, rank, kh, F::FW * fw + f, tok, acc[t][tt][2 * hh] - z0, acc[t][tt][2 * hh + 1] - z1);
             }
     st_finish<true, TOKS>(p, recv_part, recv_h, hfull, lup, tile_c, rank);
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// Weight prefetch.  A streaming kernel owns its SM (sixteen warps, most of the registers and shared memory), so the CTAs
+// of the next call cannot move in beside it and start their copies early.  This small kernel goes in front of every
+// streaming kernel instead: its CTAs need almost nothing, so they run while the preceding call is still computing
+// (programmatic dependent launch), ask the call's packed words, scales and zeros into L2 with bulk prefetches, and then
+// wait for the preceding grid -- the streaming kernel behind it waits for THIS grid, hence for everything before it.
+// Only the frozen tensors are touched.
+// ------------------------------------------------------------------------------------------------------------
+constexpr int ST_PF_CHUNK = 8192;   // bytes per bulk prefetch
+
+__device__ __forceinline__ void st_bulk_prefetch(const char* base, size_t bytes, size_t first, size_t stride) {
+    for (size_t off = first * ST_PF_CHUNK; off < bytes; off += stride * ST_PF_CHUNK) {
+        const size_t left = bytes - off;
+        const uint32_t n = (uint32_t)(left < ST_PF_CHUNK ? left : ST_PF_CHUNK) & ~15u;
+        if (n) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + off), "r"(n) : "memory");
+    }
+}
+
+__global__ void __launch_bounds__(128) stream_prefetch_kernel(const char* Q, size_t q_bytes, const char* scales, const char* zeros, size_t sz_bytes) {
+    pdl_launch_dependents();
+    const size_t me = (size_t)blockIdx.x * blockDim.x + threadIdx.x, all = (size_t)gridDim.x * blockDim.x;
+    st_bulk_prefetch(Q, q_bytes, me, all);
+    st_bulk_prefetch(scales, sz_bytes, me, all);
+    st_bulk_prefetch(zeros, sz_bytes, me, all);
+    pdl_wait();
 }
 
 // Raising a kernel's dynamic shared-memory limit is a per-function AND per-device setting: `done` belongs to one kernel
@@ -937,7 +963,7 @@ size_t st_smem_bytes(bool transposed, int nw, int toks, int xc, int copies, int 
     const size_t tail = (size_t)(256 + 1024) * 4 + ST_LUP_BYTES + (size_t)nw * 1024 + (size_t)ks * 1024 + (size_t)KH * tile_c * 64;
     if (transposed)
         return (size_t)nw * F::BNS * F::BSLOT + (size_t)copies * toks * (xc * 2 + 64) + (size_t)(nw * 32 + 32) * 4 + tail;
-    return (size_t)nw * F::NS * F::SLOT + (size_t)toks * (xc * 2 + F::XPAD) + (size_t)(toks * (xc / 8) + KH * (xc / F::KB + 1) * toks) * 4 + tail;
+    return (size_t)nw * F::NS * F::SLOT + (size_t)toks * (xc * 2 + F::XPAD) + (size_t)(toks * (xc / 8) + KH * (xc / F::KB / KH + 1) * toks) * 4 + tail;
 }
 
 // Warps per CTA of the backward kernel: the features of a CTA must lie in one group or span exactly two.
@@ -1024,6 +1050,8 @@ int launch_stream_gemm(const qlora_desc& d, int M, bool transposed, const void* 
         units = (d.K + fwd_kb(d.bits) - 1) / fwd_kb(d.bits);
     }
     p.wc = wc;
+    p.lwc = 0;
+    while ((1 << p.lwc) < wc) ++p.lwc;
     const int tiles = (p.C + tile_c - 1) / tile_c;
     // split the contraction over a cluster until the grid covers the GPU: one CTA per SM, and no more clusters than can
     // run at once (the clusters of a launch that come later would wait for whole earlier ones to finish)
@@ -1032,6 +1060,8 @@ int launch_stream_gemm(const qlora_desc& d, int M, bool transposed, const void* 
            tile_c / (2 * ks) >= 1)
         ks *= 2;
     p.ks = ks;
+    p.lks = 0;
+    while ((1 << p.lks) < ks) ++p.lks;
     // ... and inside a CTA until it has sixteen warps, while a warp keeps at least two stages
     p.khs = 0;
     while ((wc << (p.khs + 1)) <= 16 && p.khs < 2 && units / (ks << (p.khs + 1)) >= 2) ++p.khs;
@@ -1039,13 +1069,15 @@ int launch_stream_gemm(const qlora_desc& d, int M, bool transposed, const void* 
     const int sl = tile_c / ks;
     p.sls = 0;
     while ((1 << p.sls) < sl) ++p.sls;
-    // the activation slice staged per pass: the CTA's whole range when that fits (one pass, two barriers), else 512 at a time
+    // the activations staged per pass (all parts of a CTA together): the CTA's whole range when that fits (one pass, two
+    // barriers), else 512 at a time; a power of two, and at least one stage per part
     {
         const int unit = transposed ? (d.bits == 2 ? 128 : 32) : fwd_kb(d.bits);
-        const int range = ((units + ks - 1) / ks) * unit;
-        const int cap = transposed ? ((p.copies * toks > 16) ? 512 : 1024) : 1024;
-        p.xc = range <= cap ? ((range + 127) / 128) * 128 : 512;
-        if (p.xc < 128) p.xc = 128;
+        const int range = ((units + ks - 1) / ks + KH - 1) / KH * KH * unit;
+        const int cap = (transposed && p.copies * toks > 16) ? 512 : 1024;
+        p.xc = 128;
+        while (p.xc < range && p.xc < cap) p.xc *= 2;
+        if (p.xc < unit * KH) p.xc = unit * KH;
     }
     p.lup_staged = (sl * d.r * 2 <= ST_LUP_BYTES) ? 1 : 0;
     size_t smem = 0;
@@ -1056,6 +1088,13 @@ int launch_stream_gemm(const qlora_desc& d, int M, bool transposed, const void* 
         case 8: smem = st_smem_bytes<8>(transposed, nw, toks, p.xc, p.copies, KH, ks, tile_c); break;
     }
     if (smem > 227 * 1024) return QLORA_ERR_UNSUPPORTED;
+    {   // the frozen tensors on their way into L2 while the preceding call computes
+        const size_t q_bytes = (size_t)d.K * d.bits / 8 * d.N, sz_bytes = (size_t)(d.K / d.group_size) * d.N * 2;
+        const unsigned blocks = (unsigned)((q_bytes / ST_PF_CHUNK + 127) / 128 + 1);
+        if (launch_pdl(stream_prefetch_kernel, dim3(blocks), dim3(128), 0, st, 1, (const char*)Q, q_bytes, (const char*)scales, (const char*)zeros,
+                       sz_bytes) != cudaSuccess)
+            return QLORA_ERR_CUDA;
+    }
 #define QLORA_ST(B, NT)                                                                                   \
     return transposed ? st_launch<B, NT, true>(p, nw, tiles, smem, st) : st_launch<B, NT, false>(p, nw, tiles, smem, st)
 #define QLORA_ST_BITS(NT)           \
