@@ -177,6 +177,17 @@ int qlora_gather_columns(int elem_bytes, int rows, int cols, const void* in, con
 int qlora_dequant(const qlora_desc* desc, const int32_t* Q, const void* scales, const void* zeros, void* W,
                   void* cuda_stream);
 
+/* Asymmetric min-max round-to-nearest quantizer: the "RTN" baseline of the paper's tables (Section 4.2) and the way the
+ * benchmark layers are produced.  W: fp32 [N, K] device pointer (the weight as the paper writes it, one row per output
+ * feature).  For every output feature n and every group of group_size consecutive k:
+ *     lo = min(0, min w), hi = max(0, max w), qmax = 2^bits - 1,
+ *     scale = fp16((hi - lo) / qmax), 1 when that is 0;  zero = clamp(rint(-lo / scale), 0, qmax);
+ *     q[k] = clamp(rint(w[k] / scale) + zero, 0, qmax)
+ * in float32 with the fp16-rounded scale, halves to even.  Outputs: Q int32 [K*bits/32, N] (packed as above), scales and
+ * zeros fp16 [K/g, N].  Integer results: the same bits as a plain CPU evaluation of these formulas.  Weights must be
+ * finite.  desc->r and desc->alpha are ignored. */
+int qlora_quantize_rtn(const qlora_desc* desc, const float* W, int32_t* Q, void* scales, void* zeros, void* cuda_stream);
+
 /* Health check of the kernels enqueued so far on the current device.  Every wait inside the tensor-core kernels (on a
  * TMA transfer, on another warp, on the tensor cores) is bounded; if one ever runs out, the kernel stops early, leaves
  * its outputs incomplete and sets a sticky per-device status word instead of hanging the GPU.  This call SYNCHRONISES

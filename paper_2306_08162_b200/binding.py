@@ -55,12 +55,13 @@ def library() -> ctypes.CDLL:
     lib.qlora_pack.argtypes = [i32, i32, i32, vp, vp, vp]
     lib.qlora_unpack.argtypes = [i32, i32, i32, vp, vp, vp]
     lib.qlora_dequant.argtypes = [dp, vp, vp, vp, vp, vp]
+    lib.qlora_quantize_rtn.argtypes = [dp, vp, vp, vp, vp, vp]
     lib.qlora_gather_columns.argtypes = [i32, i32, i32, vp, vp, vp, vp]
     lib.qlora_lrec_loss.argtypes = [i32, i32, vp, vp, vp, ctypes.c_float, ctypes.c_float, ctypes.c_float, vp, vp, vp]
     lib.qlora_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint), i32]
     for name in ("qlora_workspace_bytes", "qlora_fwd", "qlora_bwd_input", "qlora_bwd_lora", "qlora_bwd_lora_static", "qlora_fwd_dropout", "qlora_bwd_input_dropout",
                  "qlora_bwd_lora_dropout", "qlora_pack",
-                 "qlora_unpack", "qlora_dequant", "qlora_gather_columns", "qlora_lrec_loss", "qlora_device_status"):
+                 "qlora_unpack", "qlora_dequant", "qlora_quantize_rtn", "qlora_gather_columns", "qlora_lrec_loss", "qlora_device_status"):
         getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -185,6 +186,12 @@ def qlora_gather_columns(inp, perm, out, stream=None):
 def qlora_dequant(d, Q, scales, zeros, W, stream=None):
     _check(library().qlora_dequant(ctypes.byref(d), _ptr(Q), _ptr(scales), _ptr(zeros), _ptr(W), _stream(stream)),
            "qlora_dequant")
+
+
+def qlora_quantize_rtn(d, W, Q, scales, zeros, stream=None):
+    """Min-max round-to-nearest quantization of W fp32 [N, K] into packed Q, fp16 scales and zeros [K/g, N]."""
+    _check(library().qlora_quantize_rtn(ctypes.byref(d), _ptr(W), _ptr(Q), _ptr(scales), _ptr(zeros), _stream(stream)),
+           "qlora_quantize_rtn")
 
 
 def qlora_device_status(clear: bool = True) -> int:

@@ -141,6 +141,16 @@ int qlora_dequant(const qlora_desc* desc, const int32_t* Q, const void* scales, 
     return launch_dequant(*desc, Q, scales, zeros, W, (cudaStream_t)cuda_stream);
 }
 
+int qlora_quantize_rtn(const qlora_desc* desc, const float* W, int32_t* Q, void* scales, void* zeros, void* cuda_stream) {
+    const int rc = check_desc(desc, false);
+    if (rc != QLORA_OK) return rc;
+    if (desc->K == 0 || desc->N == 0) return QLORA_OK;
+    if (!W || !Q || !scales || !zeros) return QLORA_ERR_INVALID_ARG;
+    if (!aligned16(W) || !aligned16(Q) || !aligned16(scales) || !aligned16(zeros)) return QLORA_ERR_ALIGNMENT;
+    if ((long long)desc->K / desc->group_size > 65535) return QLORA_ERR_UNSUPPORTED;
+    return launch_quantize_rtn(*desc, W, Q, scales, zeros, (cudaStream_t)cuda_stream);
+}
+
 // mask == NULL: the plain layer.  Otherwise LoRA dropout: the branch sees keep_scale * mask (.) X.
 static int fwd_common(const qlora_desc* desc, int M, const void* X, const uint8_t* mask, float keep_scale, const int32_t* Q,
                       const void* scales, const void* zeros, const void* A, const void* B, void* Y, float* H_out,

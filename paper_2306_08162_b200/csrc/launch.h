@@ -14,6 +14,7 @@ int launch_unpack(int bits, int K, int N, const int32_t* Q, uint8_t* codes, cuda
 int launch_gather_columns(int elem_bytes, int rows, int cols, const void* in, const int32_t* perm, void* out, cudaStream_t st);
 int launch_dequant(const qlora_desc& d, const int32_t* Q, const void* scales, const void* zeros, void* W,
                    cudaStream_t st);
+int launch_quantize_rtn(const qlora_desc& d, const float* W, int32_t* Q, void* scales, void* zeros, cudaStream_t st);
 
 // loss_kernel.cu -- fused KL + cross-entropy loss and its gradient over [T, V] logits (V % 8 == 0, V <= 32768)
 int launch_lrec_loss(int T, int V, const void* Z, const void* Tt, const int32_t* labels, float lambda_kl, float lambda_ce,
