@@ -60,7 +60,6 @@ def layer_bytes(w):
 
 def weight_bytes(w):
     return w["N"] * w["K"] * w["bits"] / 8 + 4 * w["N"] * w["K"] / w["group_size"]
-KERNELS_PER_STEP = None           # filled from the library's dispatch (see launches_per_step)
 
 # DRAM traffic (read + write) per launch of the dominant kernel of the default workload, from one ncu capture of that
 # kernel (dram__bytes_read.sum + dram__bytes_write.sum).  Set back to None whenever that kernel changes.
@@ -228,6 +227,137 @@ def aggregate_value(flops_per_step, steps, world, total_ms):
     return flops_per_step * steps * world / (total_ms * 1e-3) / 1e12
 
 
+def count_kernel_launches(body):
+    """Kernel launches of one call of `body`, counted as the kernel nodes of a stream capture of it (so the number is
+    what the library really enqueues for this shape on this device).  None when the CUDA Python bindings are missing."""
+    import torch
+    try:
+        from cuda.bindings import runtime as rt
+    except Exception:
+        return None
+    st = torch.cuda.Stream()
+    st.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(st):
+        (err,) = rt.cudaStreamBeginCapture(st.cuda_stream, rt.cudaStreamCaptureMode.cudaStreamCaptureModeThreadLocal)
+        if err != rt.cudaError_t.cudaSuccess:
+            return None
+        try:
+            body()
+        finally:
+            err, graph = rt.cudaStreamEndCapture(st.cuda_stream)
+    if err != rt.cudaError_t.cudaSuccess:
+        return None
+    err, _, total = rt.cudaGraphGetNodes(graph, 0)
+    err, nodes, total = rt.cudaGraphGetNodes(graph, total)
+    n = sum(1 for nd in nodes[:total] if rt.cudaGraphNodeGetType(nd)[1] == rt.cudaGraphNodeType.cudaGraphNodeTypeKernel)
+    rt.cudaGraphDestroy(graph)
+    torch.cuda.current_stream().wait_stream(st)
+    return n
+
+
+class GraphTimer:
+    """A sequence of C-ABI calls captured once in a CUDA graph; timed by replaying it back to back inside one CUDA-event
+    pair until the region is at least `min_ms` long (the interpreter's per-call cost is not what is timed, and a region
+    of tens of milliseconds gives the clock sampler something to sample)."""
+
+    def __init__(self, body, barrier):
+        import torch
+        self.torch, self.barrier = torch, barrier
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            body()
+        self.graph.replay()
+        barrier()
+
+    def one(self):
+        t = self.torch
+        e0, e1 = t.cuda.Event(enable_timing=True), t.cuda.Event(enable_timing=True)
+        e0.record(); self.graph.replay(); e1.record()
+        self.barrier()
+        return e0.elapsed_time(e1)
+
+    def region(self, min_ms, device_index=None):
+        """(ms per replay, replays, total ms, clocks) over a region of >= min_ms."""
+        t = self.torch
+        probe = max(self.one(), 1e-3)
+        reps = max(1, int(np.ceil(min_ms / probe)))
+        sampler = ClockSampler(device_index, period_s=0.002) if device_index is not None else None
+        e0, e1 = t.cuda.Event(enable_timing=True), t.cuda.Event(enable_timing=True)
+        self.barrier()
+        if sampler:
+            sampler.start()
+        e0.record()
+        for _ in range(reps):
+            self.graph.replay()
+        e1.record()
+        self.barrier()
+        clocks = sampler.stop() if sampler else None
+        total = e0.elapsed_time(e1)
+        return total / reps, reps, total, clocks
+
+
+def measure_small_m(ql, dev, local, peaks, barrier):
+    """The few-token regime (configs[3]: INT3 at 16 tokens, INT8 at 1 token, K = N = 4096, group 128, r = 8): one call
+    streams the packed weights of a layer once, so the bound is HBM bandwidth.  96 calls of one kind over a rotation of
+    layer copies (> 300 MiB of frozen weights and adapters, so no call finds its layer in L2; the few activation rows
+    rotate over four buffers, as a network's would be warm) are captured in a graph and replayed for >= 50 ms."""
+    import torch
+    out = []
+    K = N = 4096
+    g, r = 128, 8
+    for bits, M in ((3, 16), (8, 1)):
+        d = ql.desc(bits, g, K, N, r, 16.0)
+        wb = N * K * bits / 8 + 4 * N * K / g
+        nl = max(4, int(np.ceil(300 * 2**20 / (wb + 4 * r * (K + N)))))
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(1234 + bits)
+        layers = []
+        for _ in range(nl):
+            layers.append(dict(
+                Q=torch.randint(-2**31, 2**31 - 1, (K * bits // 32, N), dtype=torch.int32, device=dev, generator=gen),
+                s=(torch.rand((K // g, N), device=dev, generator=gen) * 0.01 + 0.002).half(),
+                z=torch.randint(0, 1 << bits, (K // g, N), device=dev, generator=gen).half(),
+                A=(torch.randn((r, K), device=dev, generator=gen) * 0.02).bfloat16(),
+                B=(torch.randn((N, r), device=dev, generator=gen) * 0.01).bfloat16()))
+        acts = [dict(X=torch.randn((M, K), device=dev, generator=gen).bfloat16(), dY=torch.randn((M, N), device=dev, generator=gen).bfloat16(),
+                     Y=torch.empty((M, N), dtype=torch.bfloat16, device=dev), dX=torch.empty((M, K), dtype=torch.bfloat16, device=dev))
+                for _ in range(4)]
+        ws = torch.empty(ql.qlora_workspace_bytes(d, M), dtype=torch.uint8, device=dev)
+        calls = 96
+
+        def fwd():
+            for i in range(calls):
+                L, a = layers[i % nl], acts[i % 4]
+                ql.qlora_fwd(d, M, a["X"], L["Q"], L["s"], L["z"], L["A"], L["B"], a["Y"], None, ws)
+
+        def bwd():
+            for i in range(calls):
+                L, a = layers[i % nl], acts[i % 4]
+                ql.qlora_bwd_input(d, M, a["dY"], L["Q"], L["s"], L["z"], L["A"], L["B"], a["dX"], None, ws)
+
+        alg = wb + 2 * M * (K + N) + 2 * r * (K + N)
+        rec = {"workload": f"configs[3]: K=N=4096, INT{bits} group 128, LoRA r=8, M={M}", "algorithmic_bytes_per_call": alg,
+               "rotation": f"{nl} layer copies, {int(nl * (wb + 4 * r * (K + N))) >> 20} MiB", "calls": {}}
+        worst = None
+        for name, body in (("qlora_fwd", fwd), ("qlora_bwd_input", bwd)):
+            for _ in range(2):
+                body()
+            gt = GraphTimer(body, barrier)
+            ms, reps, total, clocks = gt.region(50.0, local)
+            us = ms / calls * 1e3
+            gbs = alg / (us * 1e-6) / 1e9
+            rec["calls"][name] = {"us_per_call": us, "achieved": gbs, "unit": "GB/s", "frac": gbs / peaks["hbm"],
+                                  "timed_region_ms": total, "clocks": clocks}
+            worst = gbs if worst is None else min(worst, gbs)
+            del gt
+        rec["achieved"], rec["unit"], rec["peak"], rec["frac"] = worst, "GB/s", peaks["hbm"], worst / peaks["hbm"]
+        rec["peak_kind"] = f"{peaks['source']} HBM copy bandwidth"
+        out.append(rec)
+        del layers, acts
+        torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -309,30 +439,34 @@ def run_ours(args):
     call_ms = [float(np.mean([ev[i][c].elapsed_time(ev[i][c + 1]) for i in range(args.steps)])) for c in range(3)]
 
     eager_ms_per_step = total_ms / args.steps
+    sustained = None
+    launches = count_kernel_launches(lambda: step(layers[0]))
     if args.graph:
-        # The same K steps (same C-ABI calls, same rotation) captured once in a CUDA graph and replayed, so that the
-        # Python interpreter's per-call cost (tens of microseconds, more than some of the kernels) is not what is timed.
-        def graph_ms(body, replays=1):
-            gr = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(gr):
+        # The same K steps (same C-ABI calls, same rotation) captured once in a CUDA graph and replayed back to back, so that
+        # the Python interpreter's per-call cost (tens of microseconds, more than some of the kernels) is not what is
+        # timed.  Two regions: >= 60 ms (the burst regime the burst peak was measured in) and >= 1 s (power-capped clocks,
+        # compared with the sustained peak); each with its own clock record.
+        def steps_body(call):
+            def body():
                 for i in range(args.steps):
-                    body(layers[i % ROTATION])
-            gr.replay()
-            barrier()
-            times = []
-            for _ in range(replays):
-                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                g0.record(); gr.replay(); g1.record()
-                barrier()
-                times.append(g0.elapsed_time(g1))
-            return float(np.median(times))
-        sampler = ClockSampler(local)
-        sampler.start()
-        total_ms = graph_ms(step)
-        clocks = sampler.stop()
-        call_ms = [graph_ms(lambda L: ql.qlora_fwd(d, M, L["X"], L["Q"], L["scales"], L["zeros"], L["A"], L["B"], L["Y"], L["H"], ws), 3) / args.steps,
-                   graph_ms(lambda L: ql.qlora_bwd_input(d, M, L["dY"], L["Q"], L["scales"], L["zeros"], L["A"], L["B"], L["dX"], L["G"], ws), 3) / args.steps,
-                   graph_ms(lambda L: ql.qlora_bwd_lora(d, M, L["X"], L["dY"], L["A"], L["B"], L["H"], L["G"], L["dA"], L["dB"], 0, ws), 3) / args.steps]   # (per-call split: median of three replays)
+                    call(layers[i % ROTATION])
+            return body
+        gt = GraphTimer(steps_body(step), barrier)
+        ms_replay, replays, region_ms, clocks = gt.region(60.0, local)
+        total_ms = ms_replay                                   # K steps
+        if not args.no_sustained:
+            s_ms, s_reps, s_region, s_clocks = gt.region(1000.0, local)
+            sustained = dict(ms_per_step=s_ms / args.steps, replays=s_reps, timed_region_ms=s_region, clocks=s_clocks)
+        del gt
+        call_ms = []
+        for call in (lambda L: ql.qlora_fwd(d, M, L["X"], L["Q"], L["scales"], L["zeros"], L["A"], L["B"], L["Y"], L["H"], ws),
+                     lambda L: ql.qlora_bwd_input(d, M, L["dY"], L["Q"], L["scales"], L["zeros"], L["A"], L["B"], L["dX"], L["G"], ws),
+                     lambda L: ql.qlora_bwd_lora(d, M, L["X"], L["dY"], L["A"], L["B"], L["H"], L["G"], L["dA"], L["dB"], 0, ws)):
+            gtc = GraphTimer(steps_body(call), barrier)
+            call_ms.append(gtc.region(20.0)[0] / args.steps)
+            del gtc
+    else:
+        replays, region_ms = 1, total_ms
 
     # ---- end to end: pinned host inputs copied in, results copied out, every step --------------------------
     e2e_steps = max(3, min(args.steps, 50))
@@ -388,7 +522,10 @@ def run_ours(args):
     h2d = 2 * M * (K + N)
     d2h = 2 * M * (K + N) + 4 * r * (K + N)
 
-    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], world, dev)
+    sus_ms = sustained["ms_per_step"] * args.steps if sustained else 0.0
+    total_ms, e2e_ms, sus_ms = max_over_ranks([total_ms, e2e_ms, sus_ms], world, dev)
+    small_m = measure_small_m(ql, dev, local, measured_peaks(), barrier) if (rank == 0 and world == 1 and args.workload == "config2"
+                                                                             and not args.no_small_m) else None
 
     if rank == 0:
         flops_step = layer_flops(M, K, N, r)
@@ -398,7 +535,7 @@ def run_ours(args):
         # dominant kernel: the dequant-GEMM of the forward or backward-input call, whichever takes longer
         dom = 0 if call_ms[0] >= call_ms[1] else 1
         dom_name = ("qlora_fwd", "qlora_bwd_input")[dom]
-        long_run = total_ms > 1000.0
+        long_run = False
         if M > 64:    # a dense contraction: tensor roofline
             bound, r_unit = "tensor", "TFLOP/s"
             achieved = fwd_flops(M, K, N, r) / (call_ms[dom] * 1e-3) / 1e12
@@ -417,25 +554,120 @@ def run_ours(args):
             "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD_NAME, "parallelism": "replicas only" if world > 1 else "single GPU",
-                       "launch": ("the K steps' C-ABI calls captured in one CUDA graph, replayed once inside the timed region"
+                       "launch": (f"the K steps' C-ABI calls captured in one CUDA graph, replayed {replays} times back to back inside "
+                                  f"one CUDA-event region of {region_ms:.1f} ms; ms_per_step = region / (replays x K)"
                                   if args.graph else "one C-ABI call at a time from Python"),
                        "eager_ms_per_step": eager_ms_per_step,
                        "l2": f"inputs larger than L2: steps rotate through {ROTATION} independent layer copies "
                              f"(~{ROTATION * layer_bytes(w) // 2**20} MiB)",
                        "calls_ms": {"qlora_fwd": call_ms[0], "qlora_bwd_input": call_ms[1], "qlora_bwd_lora": call_ms[2]}},
             "roofline": {"bound": bound, "kernel": dom_name, "achieved": achieved, "peak": peak, "unit": r_unit,
-                         "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if args.workload == "config2" else None,
+                         "frac": achieved / peak,
+                         "frac_sustained": ((achieved * total_ms / sus_ms) / peaks["bf16_sustained"]
+                                            if (sustained and bound == "tensor" and sus_ms > 0) else None),
+                         "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if args.workload == "config2" else None,
                          "peak_kind": peak_kind,
                          "step_frac_of_peak": (value / world / peak) if bound == "tensor" else None},
+            "sustained": (None if not sustained else {
+                "value": aggregate_value(flops_step, args.steps, world, sus_ms), "unit": UNIT,
+                "ms_per_step": sus_ms / args.steps, "timed_region_ms": sustained["timed_region_ms"], "replays": sustained["replays"],
+                "clocks": sustained["clocks"],
+                "peak": peaks["bf16_sustained"], "peak_kind": f"{peaks['source']} cuBLAS bf16 sustained",
+                "step_frac_of_peak": aggregate_value(flops_step, args.steps, world, sus_ms) / world / peaks["bf16_sustained"]}),
+            "small_m": small_m,
             "cpu_baseline": {"value": cpu["value"], "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": cpu["sample"]},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
-            "gpu_launches": launches_per_step(M, r, K, N, w["bits"]) * args.steps,
+            "gpu_launches": (launches if launches is not None else 4) * args.steps * (replays if args.graph else 1),
+            "gpu_launches_per_step": launches,
             "clocks": clocks,
         }
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+    return 0
+
+
+def run_chain(args):
+    """--workload config5: the projection set of configs[4] -- 32 decoder blocks x (q, k, v, o 4096x4096; gate, up
+    4096->11008; down 11008->4096), INT2 group 64, LoRA r = 8 on all 224 projections, M = 4096 tokens (8 x 512) -- run as
+    a chain: forward through every projection, then backward (qlora_bwd_input + qlora_bwd_lora) in reverse order.  One step
+    streams 2 GB of packed weights and 12 GB of saved activations, far more than the L2.  The codes are random (drawn on
+    the device: 6.5 G weights), the scales sized so that the activations keep their magnitude along the chain."""
+    import torch
+    import paper_2306_08162_b200 as ql
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    ql.library()
+    M, bits, g, r, alpha, blocks = 4096, 2, 64, 8, 16.0, 32
+    shapes = [("q", 4096, 4096), ("k", 4096, 4096), ("v", 4096, 4096), ("o", 4096, 4096), ("gate", 4096, 11008), ("up", 4096, 11008),
+              ("down", 11008, 4096)]
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(5)
+    projs, flops, ws_bytes = [], 0.0, 0
+    for blk in range(blocks):
+        row = {}
+        for name, K, N in shapes:
+            d = ql.desc(bits, g, K, N, r, alpha)
+            ws_bytes = max(ws_bytes, ql.qlora_workspace_bytes(d, M))
+            row[name] = dict(d=d, K=K, N=N,
+                             Q=torch.randint(-2**31, 2**31 - 1, (K * bits // 32, N), dtype=torch.int32, device=dev, generator=gen),
+                             s=torch.full((K // g, N), 0.85 / float(np.sqrt(1.25 * K)), dtype=torch.float16, device=dev),
+                             z=torch.randint(1, 3, (K // g, N), device=dev, generator=gen).half(),
+                             A=((torch.rand((r, K), device=dev, generator=gen) * 2 - 1) / float(np.sqrt(K))).bfloat16(),
+                             B=(torch.randn((N, r), device=dev, generator=gen) * 0.01).bfloat16(),
+                             Y=torch.empty((M, N), dtype=torch.bfloat16, device=dev), H=torch.empty((M, r), dtype=torch.float32, device=dev),
+                             dX=torch.empty((M, K), dtype=torch.bfloat16, device=dev), G=torch.empty((M, r), dtype=torch.float32, device=dev),
+                             dA=torch.empty((r, K), dtype=torch.float32, device=dev), dB=torch.empty((N, r), dtype=torch.float32, device=dev))
+            flops += layer_flops(M, K, N, r)
+        projs.append(row)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    x0 = torch.randn((M, 4096), device=dev, generator=gen).bfloat16()
+    seed_grad = {4096: torch.randn((M, 4096), device=dev, generator=gen).bfloat16(), 11008: torch.randn((M, 11008), device=dev, generator=gen).bfloat16()}
+
+    def step():
+        x = x0
+        for row in projs:
+            for name in ("q", "k", "v", "o", "gate", "up", "down"):
+                P = row[name]
+                P["X"] = {"q": x, "k": x, "v": x, "o": row["q"]["Y"], "gate": row["o"]["Y"], "up": row["o"]["Y"], "down": row["gate"]["Y"]}[name]
+                ql.qlora_fwd(P["d"], M, P["X"], P["Q"], P["s"], P["z"], P["A"], P["B"], P["Y"], P["H"], ws)
+            x = row["down"]["Y"]
+        grad = seed_grad[4096]
+        for row in reversed(projs):
+            for name in ("down", "up", "gate", "o", "v", "k", "q"):
+                P = row[name]
+                dY = {"down": grad, "up": seed_grad[11008], "v": seed_grad[4096], "k": seed_grad[4096]}.get(name)
+                if dY is None:
+                    dY = row[{"gate": "down", "o": "gate", "q": "o"}[name]]["dX"]
+                ql.qlora_bwd_input(P["d"], M, dY, P["Q"], P["s"], P["z"], P["A"], P["B"], P["dX"], P["G"], ws)
+                ql.qlora_bwd_lora(P["d"], M, P["X"], dY, P["A"], P["B"], P["H"], P["G"], P["dA"], P["dB"], 0, ws)
+            grad = row["q"]["dX"]
+
+    def barrier():
+        torch.cuda.synchronize()
+
+    for _ in range(max(1, min(args.warmup, 3))):
+        step()
+    barrier()
+    launches = count_kernel_launches(step)
+    gt = GraphTimer(step, barrier)
+    ms, reps, region, clocks = gt.region(1000.0, local)
+    peaks = measured_peaks()
+    value = flops / (ms * 1e-3) / 1e12
+    finite = bool(torch.isfinite(projs[-1]["down"]["Y"].float()).all().item())
+    print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": 1, "steps": reps, "warmup": args.warmup, "ms_per_step": ms,
+                      "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": "configs[4]: 32 blocks x (q,k,v,o 4096x4096; gate,up 4096->11008; down 11008->4096), INT2 group 64, "
+                                             "LoRA r=8 on all 224 projections, M=4096 (8x512), chained fwd then bwd",
+                                 "launch": f"one step (224 fwd + 224 bwd_input + 224 bwd_lora calls) captured in a CUDA graph, replayed {reps} times "
+                                           f"in a region of {region:.0f} ms", "flops_per_step": flops, "outputs_finite": finite,
+                                 "l2": "inputs larger than L2: 2 GB of packed weights and 12 GB of activations per step"},
+                      "roofline": {"bound": "tensor", "kernel": "whole step", "achieved": value, "peak": peaks["bf16_sustained"], "unit": UNIT,
+                                   "frac": value / peaks["bf16_sustained"], "traffic": None,
+                                   "peak_kind": f"{peaks['source']} cuBLAS bf16 sustained (the region is {region / 1e3:.1f} s long)"},
+                      "e2e": None, "cpu_baseline": None, "gpu_launches": (launches or 0) * reps, "gpu_launches_per_step": launches, "clocks": clocks}))
     return 0
 
 
@@ -481,64 +713,6 @@ def run_loss(args):
     return 0
 
 
-def prefer_pair_kernel(M: int, C: int, T: int, sms: int = 148) -> bool:
-    """Mirror of the library's choice between its two tensor-core kernels (the cost model in csrc/umma_kernel.cu)."""
-    if M <= 256:
-        return False
-    if M > 1024:
-        return True
-    steps = T // 64
-    tiles_mid = -(-M // 256) * -(-C // 128)
-    split = next((sp for sp in (4, 2) if tiles_mid * sp <= sms and steps % sp == 0 and steps // sp >= 4), 1)
-    waves_mid = 1 if split > 1 else -(-tiles_mid // sms)
-    mid_us = waves_mid * ((steps // split) * 0.29 + 15.0)
-    tiles_pair = -(-M // 512) * -(-C // 256)
-    pair_us = -(-tiles_pair // (sms // 2)) * (steps * 0.62 + 4.0)
-    return pair_us < mid_us
-
-
-def pair_kernel_computes_p(M: int, C: int, T: int, r: int, sms: int = 148) -> bool:
-    """Mirror of the library's dispatch: the CTA-pair kernel (where prefer_pair_kernel picks it) runs the LoRA down-projection on SM pairs
-    that have less to do than the rest -- no tile (512 tokens x 256 of the C output columns) at all, or one tile fewer
-    because the last wave is partly filled -- when there are enough of them."""
-    if not prefer_pair_kernel(M, C, T, sms) or r == 0 or r > 16:
-        return False
-    tiles, pairs = -(-M // 512) * -(-C // 256), sms // 2
-    idle = pairs - tiles if tiles < pairs else (pairs - tiles % pairs if tiles % pairs else 0)
-    blocks = -(-M // 16)
-    n_prod = min(idle, -(-blocks // 4))
-    return n_prod > 0 and n_prod * 16 >= blocks
-
-
-def mid_kernel_computes_p(M: int, C: int, T: int, r: int, sms: int = 148) -> bool:
-    """Mirror of the dispatch for the single-CTA tensor-core kernel (from 17 tokens, or one with 8-bit weights, up to
-    where prefer_pair_kernel picks the other): tiles of 128 output columns, the contraction split over clusters of 4 or
-    2 CTAs when that still fits the GPU; producer clusters are added while the GPU can hold more clusters of that width
-    (33 of width 4, 74 of width 2) and two row blocks of 16 tokens per producer CTA cover the batch."""
-    if prefer_pair_kernel(M, C, T, sms) or r == 0 or r > 16:
-        return False
-    tiles, steps, bt = -(-C // 128) * max(1, -(-M // 256)), T // 64, (256 if M > 128 else 128 if M > 64 else 64 if M > 32 else 32)
-    split = next((sp for sp in (4, 2) if tiles * sp <= sms and steps % sp == 0 and steps // sp >= 4 and bt % sp == 0), 1)
-    clusters = tiles if split > 1 else min(tiles, sms)
-    idle = {1: sms, 2: sms // 2, 4: 33}[split] - clusters
-    blocks = -(-M // 16)
-    n_prod = min(idle, -(-blocks // split))
-    return n_prod > 0 and n_prod * split * 2 >= blocks
-
-
-def launches_per_step(M: int, r: int, K: int, N: int, bits: int = 4) -> int:
-    """Kernels the library launches for one fwd + bwd_input + bwd_lora (H, G saved).  Each of fwd and bwd_input is a
-    down-projection launch plus the dequant-GEMM, or the dequant-GEMM alone where it computes H / G itself (the streaming
-    kernels with r <= 16; above that where the tiles leave SMs idle).  The gradients are one launch up to 256 tokens (the row
-    slices of a column block form a cluster and reduce through distributed shared memory), else two."""
-    if r == 0:
-        return 2
-    streaming = M <= 16 and bits != 8          # (shapes the tensor-core kernels tile; the bench's all are)
-    fwd = 1 if (streaming and r <= 16) or pair_kernel_computes_p(M, N, K, r) or (not streaming and mid_kernel_computes_p(M, N, K, r)) else 2
-    bwd = 1 if (streaming and r <= 16) or pair_kernel_computes_p(M, K, N, r) or (not streaming and mid_kernel_computes_p(M, K, N, r)) else 2
-    return fwd + bwd + (1 if M <= 256 else 2)       # gradients: one clustered launch up to 256 tokens
-
-
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -547,11 +721,13 @@ def main():
                          "runs longer than 1 s are compared with the sustained peak)")
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=sorted(WORKLOADS) + ["lrec_loss"], default="config2",
+    ap.add_argument("--workload", choices=sorted(WORKLOADS) + ["config5", "lrec_loss"], default="config2",
                     help="layer shape to run (default: configs[1], the headline workload)")
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="time the K steps as issued call by call from Python instead of as one CUDA-graph replay "
                          "(the default; the interpreter's per-call cost is otherwise part of every step)")
+    ap.add_argument("--no-sustained", action="store_true", help="leave out the second, >= 1 s timed region")
+    ap.add_argument("--no-small-m", action="store_true", help="leave out the few-token (HBM-bound) record of the default run")
     ap.add_argument("--skip-cpu-baseline", action="store_true",
                     help="leave out the CPU-oracle timing leg (for profiler runs, where only the GPU launches matter)")
     args = ap.parse_args()
@@ -559,6 +735,10 @@ def main():
         args.warmup = 3
     if args.workload == "lrec_loss":
         return run_loss(args)
+    if args.workload == "config5" and args.impl == "ours":
+        return run_chain(args)
+    if args.workload == "config5":
+        raise SystemExit("--impl reference times the default workloads only")
     global WORKLOAD, WORKLOAD_NAME, ROTATION
     WORKLOAD, WORKLOAD_NAME = WORKLOADS[args.workload]
     ROTATION = max(4, -(-300 * 2**20 // layer_bytes(WORKLOAD)))     # > 126 MB of L2 with margin
