@@ -27,18 +27,24 @@
  *
  * General rules for every entry point below.
  *   - All tensor pointers are DEVICE pointers owned by the caller, dense row-major, 16-byte aligned.  The
- *     descriptor is a HOST pointer.  The library allocates no device memory, keeps no per-call state and never
- *     frees anything.  Q, scales, zeros, A, B are read-only (theta_q is frozen and there is no gradient for it;
- *     Section 3.1).
- *     Because they are read-only for every call of the library, a call may start loading Q, scales, zeros, A and B
- *     while the library's own preceding call in the stream is still finishing (programmatic dependent launch); it waits
- *     for that call before it touches activations, H / G or outputs.  Work of other origin in the stream (a kernel
- *     that repacks Q or updates A / B) is always complete before a call starts.
+ *     descriptor is a HOST pointer.  The library allocates no device memory and never frees anything.  What it keeps
+ *     between calls is host-side and per device ordinal: which of its kernels have had their shared-memory limit
+ *     raised there, the SM count and cluster occupancy it queried, one sticky health word on the device
+ *     (qlora_device_status) and the fixed array of qlora_bwd_lora_static.  Nothing is keyed by a caller's pointer and no
+ *     result depends on the history of calls.
+ *   - Q, scales, zeros, A, B are read-only for the library.  Q, scales and zeros are FROZEN (theta_q has no gradient;
+ *     Section 3.1): the layer calls are launched with programmatic stream serialization and may read these three -- and
+ *     only these -- while the preceding kernel in the stream is still finishing.  A and B are theta_l, which an optimizer
+ *     rewrites every step (Section 3.2, Eq. 3): they, the activations, H / G, the workspace and the outputs are touched
+ *     only after the preceding kernel has completed and its writes are visible (griddepcontrol.wait).  A caller that
+ *     rewrites Q, scales or zeros in the same stream must synchronise that stream (or use another stream and an event)
+ *     before the next layer call on them.
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = the legacy default stream) of
  *     the current device.  No call synchronises the device; outputs are valid in stream order.
  *   - Calls given the same workspace must be ordered one after the other (same stream, or events): they share
- *     its contents, and the library keys the few words of device-side bookkeeping some kernels need (counters that
- *     a launch leaves zeroed) by the workspace address.  Calls with different workspaces may overlap freely.
+ *     its contents, which include two counters through which CTAs of one launch signal each other (set to zero in
+ *     stream order ahead of the launch, so the workspace needs no initialisation).  Calls with different workspaces may
+ *     overlap freely.
  *   - Return value: QLORA_OK or a negative QLORA_ERR_* code.  Arguments are validated before anything is
  *     launched; on error nothing has been enqueued.  Nothing is printed, nothing throws.
  *   - Same inputs give bitwise the same outputs on every run (fixed-order reductions, no floating-point atomics).
@@ -78,7 +84,7 @@ typedef struct {
 } qlora_desc;
 
 /* Bytes of scratch the three layer calls may need for M tokens (the maximum over the calls, so one buffer
- * serves all).  `out` is a host pointer.  The scratch holds H / G when the caller does not keep them, the
+ * serves all).  The paper has no counterpart: it is how a library that allocates nothing gets its scratch.  `out` is a host pointer.  The scratch holds H / G when the caller does not keep them, the
  * split partial sums of the LoRA gradients and of small-M products.  Contents are undefined between calls. */
 int qlora_workspace_bytes(const qlora_desc* desc, int M, size_t* out);
 
@@ -171,7 +177,8 @@ int qlora_lrec_loss(int T, int V, const void* student_logits, const void* teache
  * permutation (the same call). */
 int qlora_gather_columns(int elem_bytes, int rows, int cols, const void* in, const int32_t* perm, void* out, void* cuda_stream);
 
-/* Full dequantisation to the bf16 weight the tensor-core kernels stage:  W[n,k] = bf16_rne(fp32(scale) * (q - zero)),
+/* Full dequantisation (Section 3.1: the weights are unpacked to floating point before every matrix product; here as a
+ * stand-alone utility, for checks and for callers that want the dense weight) to the bf16 weight the tensor-core kernels stage:  W[n,k] = bf16_rne(fp32(scale) * (q - zero)),
  * bf16 [N, K].  The fp32 product is exact (an 11-bit significand times an integer of at most 9 bits), so the result
  * is a single rounding of the closed form.  desc->r and desc->alpha are ignored. */
 int qlora_dequant(const qlora_desc* desc, const int32_t* Q, const void* scales, const void* zeros, void* W,
@@ -195,7 +202,14 @@ int qlora_quantize_rtn(const qlora_desc* desc, const float* W, int32_t* Q, void*
  * returns QLORA_OK or QLORA_ERR_TIMEOUT.  The paper has no counterpart; it exists so that a synchronisation fault cannot hang a device. */
 int qlora_device_status(unsigned int* status_out, int clear);
 
-/* Human-readable name of a status code (static storage; never NULL). */
+/* Self-test of the give-up path behind qlora_device_status (the paper has no counterpart).  Enqueues a one-CTA kernel in
+ * which one thread waits, with the same bounded wait the tensor-core kernels use, on a shared-memory barrier that nobody
+ * arrives at.  After limit_us microseconds (1 .. 1000000) the wait gives up, the sticky status word is set and the kernel
+ * ends normally; the next qlora_device_status call reports QLORA_ERR_TIMEOUT (and clears the word if asked to).  No real
+ * kernel is stalled and nothing else on the device is touched. */
+int qlora_selftest_bounded_wait(int limit_us, void* cuda_stream);
+
+/* Human-readable name of a status code (static storage; never NULL).  The paper has no counterpart. */
 const char* qlora_status_string(int status);
 
 #ifdef __cplusplus

@@ -59,9 +59,10 @@ def library() -> ctypes.CDLL:
     lib.qlora_gather_columns.argtypes = [i32, i32, i32, vp, vp, vp, vp]
     lib.qlora_lrec_loss.argtypes = [i32, i32, vp, vp, vp, ctypes.c_float, ctypes.c_float, ctypes.c_float, vp, vp, vp]
     lib.qlora_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint), i32]
+    lib.qlora_selftest_bounded_wait.argtypes = [i32, vp]
     for name in ("qlora_workspace_bytes", "qlora_fwd", "qlora_bwd_input", "qlora_bwd_lora", "qlora_bwd_lora_static", "qlora_fwd_dropout", "qlora_bwd_input_dropout",
                  "qlora_bwd_lora_dropout", "qlora_pack",
-                 "qlora_unpack", "qlora_dequant", "qlora_quantize_rtn", "qlora_gather_columns", "qlora_lrec_loss", "qlora_device_status"):
+                 "qlora_unpack", "qlora_dequant", "qlora_quantize_rtn", "qlora_gather_columns", "qlora_lrec_loss", "qlora_device_status", "qlora_selftest_bounded_wait"):
         getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -192,6 +193,11 @@ def qlora_quantize_rtn(d, W, Q, scales, zeros, stream=None):
     """Min-max round-to-nearest quantization of W fp32 [N, K] into packed Q, fp16 scales and zeros [K/g, N]."""
     _check(library().qlora_quantize_rtn(ctypes.byref(d), _ptr(W), _ptr(Q), _ptr(scales), _ptr(zeros), _stream(stream)),
            "qlora_quantize_rtn")
+
+
+def qlora_selftest_bounded_wait(limit_us: int, stream=None):
+    """Enqueue a wait that is known to run out after limit_us microseconds (sets the device's sticky status word)."""
+    _check(library().qlora_selftest_bounded_wait(int(limit_us), _stream(stream)), "qlora_selftest_bounded_wait")
 
 
 def qlora_device_status(clear: bool = True) -> int:

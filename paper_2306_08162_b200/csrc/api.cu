@@ -34,15 +34,8 @@ int check_desc(const qlora_desc* d, bool need_lora) {
     return QLORA_OK;
 }
 
-// Up to 16 tokens (one 16-row MMA tile) the streaming kernels are the fastest form for 2-, 3- and 4-bit weights; from 17
-// to 32 tokens they would stream the weights twice, and with 8-bit weights their unpacking is the slower one (measured
-// 16.3 against 13.5 us at one token), so there the tensor-core kernel takes over wherever it tiles the shape.
-bool use_streaming(const qlora_desc& d, int M) {
-    return skinny_supported(d, M) && !((M > 16 || d.bits == 8) && umma_supported(d, M));
-}
-
 struct Workspace {
-    size_t p0_off, p1_off, grad_off, total;
+    size_t p0_off, p1_off, grad_off, sync_off, total;
 };
 
 Workspace carve(const qlora_desc& d, int M) {
@@ -51,8 +44,8 @@ Workspace carve(const qlora_desc& d, int M) {
     w.p0_off = 0;
     w.p1_off = p;
     w.grad_off = 2 * p;
-    w.total = w.grad_off + align_up(lora_grad_scratch_bytes(M, d.K, d.N, d.r), 256);
-    if (w.total == 0) w.total = 256;
+    w.sync_off = w.grad_off + align_up(lora_grad_scratch_bytes(M, d.K, d.N, d.r), 256);
+    w.total = w.sync_off + 256;          // two counters of the tensor-core kernels' producer clusters
     return w;
 }
 
@@ -80,6 +73,11 @@ int qlora_device_status(unsigned int* status_out, int clear) {
     const int rc = read_device_status(status_out, clear);
     if (rc != QLORA_OK) return rc;
     return *status_out == 0 ? QLORA_OK : QLORA_ERR_TIMEOUT;
+}
+
+int qlora_selftest_bounded_wait(int limit_us, void* cuda_stream) {
+    if (limit_us < 1 || limit_us > 1000000) return QLORA_ERR_INVALID_ARG;
+    return launch_wait_probe(limit_us, (cudaStream_t)cuda_stream);
 }
 
 int qlora_workspace_bytes(const qlora_desc* desc, int M, size_t* out) {
@@ -169,17 +167,17 @@ static int fwd_common(const qlora_desc* desc, int M, const void* X, const uint8_
     if (workspace == nullptr || workspace_bytes < w.total) return QLORA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     float* H = H_out ? H_out : reinterpret_cast<float*>(static_cast<char*>(workspace) + w.p0_off);
-    if (stream_supported(d, M, false) || use_streaming(d, M)) {
+    unsigned int* sync = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + w.sync_off);
+    if (stream_supported(d, M, false)) {                              // up to 16 tokens: the weight-streaming kernels
         const bool fused = d.r > 0 && d.r <= 16 && mask == nullptr;   // the down-projection rides along inside the kernel
         if (d.r > 0 && !fused) {
             rc = launch_lora_down(M, d.K, d.r, true, X, A, H, st, mask, keep_scale);
             if (rc != QLORA_OK) return rc;
         }
-        if (stream_supported(d, M, false)) return launch_stream_gemm(d, M, false, X, Q, scales, zeros, A, B, H, !fused, Y, st);
-        return launch_skinny_gemm(d, M, false, X, Q, scales, zeros, A, B, H, !fused, Y, st);
+        return launch_stream_gemm(d, M, false, X, Q, scales, zeros, A, B, H, !fused, Y, st);
     }
     // the tensor-core path computes H itself when given A (beside its tiles where SM pairs are idle, else ahead of them)
-    if (umma_supported(d, M) && mask == nullptr) return launch_umma_gemm(d, M, false, X, Q, scales, zeros, B, H, Y, st, A, workspace);
+    if (umma_supported(d, M) && mask == nullptr) return launch_umma_gemm(d, M, false, X, Q, scales, zeros, B, H, Y, st, A, sync);
     if (d.r > 0) {
         rc = launch_lora_down(M, d.K, d.r, true, X, A, H, st, mask, keep_scale);
         if (rc != QLORA_OK) return rc;
@@ -213,22 +211,21 @@ static int bwd_input_common(const qlora_desc* desc, int M, const void* dY, const
         qlora_desc d0 = d;
         d0.r = 0;
         if (stream_supported(d0, M, true)) rc = launch_stream_gemm(d0, M, true, dY, Q, scales, zeros, B, A, G, true, dX, st);
-        else if (use_streaming(d0, M)) rc = launch_skinny_gemm(d0, M, true, dY, Q, scales, zeros, B, A, G, true, dX, st);
         else if (umma_supported(d0, M)) rc = launch_umma_gemm(d0, M, true, dY, Q, scales, zeros, A, G, dX, st);
         else rc = launch_simt_gemm(d0, M, true, dY, Q, scales, zeros, A, G, dX, st);
         if (rc != QLORA_OK) return rc;
         return launch_lora_masked_update(M, d.K, d.r, keep_scale * d.alpha / (float)d.r, G, A, mask, dX, st);
     }
-    if (stream_supported(d, M, true) || use_streaming(d, M)) {
+    if (stream_supported(d, M, true)) {
         const bool fused = d.r > 0 && d.r <= 16;
         if (d.r > 0 && !fused) {
             rc = launch_lora_down(M, d.N, d.r, false, dY, B, G, st);
             if (rc != QLORA_OK) return rc;
         }
-        if (stream_supported(d, M, true)) return launch_stream_gemm(d, M, true, dY, Q, scales, zeros, B, A, G, !fused, dX, st);
-        return launch_skinny_gemm(d, M, true, dY, Q, scales, zeros, B, A, G, !fused, dX, st);
+        return launch_stream_gemm(d, M, true, dY, Q, scales, zeros, B, A, G, !fused, dX, st);
     }
-    if (umma_supported(d, M)) return launch_umma_gemm(d, M, true, dY, Q, scales, zeros, A, G, dX, st, B, workspace);   // computes G
+    unsigned int* sync = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + w.sync_off);
+    if (umma_supported(d, M)) return launch_umma_gemm(d, M, true, dY, Q, scales, zeros, A, G, dX, st, B, sync);   // computes G
     if (d.r > 0) {
         rc = launch_lora_down(M, d.N, d.r, false, dY, B, G, st);
         if (rc != QLORA_OK) return rc;

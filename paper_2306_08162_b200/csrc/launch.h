@@ -46,25 +46,20 @@ int launch_lora_masked_update(int M, int K, int r, float c, const float* G, cons
 // umma_kernel.cu -- tcgen05 tensor-core kernel (both directions); same contract as launch_simt_gemm
 // Ldown == NULL: P is an input.  Ldown != NULL (the adapter applied first: A forward, B backward): P is an output,
 // computed on the way -- by SM pairs the tiles of the CTA-pair kernel leave idle when there are some (they signal the
-// tiles through a pair of counters in device memory chosen by `sync_key`: calls that may overlap in time must pass
-// different keys; the layer calls pass their workspace), otherwise by a down-projection launch ahead of the kernel.
+// tiles through the two counters at `sync`, device memory the caller owns: the layer calls carve them out of their
+// workspace, so calls that may overlap in time have different ones), otherwise by a down-projection launch ahead of it.
 bool umma_supported(const qlora_desc& d, int M);
 int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q,
                      const void* scales, const void* zeros, const void* L, float* P, void* Out,
-                     cudaStream_t st, const void* Ldown = nullptr, const void* sync_key = nullptr);
-// Small token counts (M <= 32): TMA-fed mma.sync streaming kernels.  Ldown / Lup: the adapter applied first / second
-// (forward A, B; backward B, A).  P = H or G, fp32 [M, r]: read when p_is_input, otherwise computed inside the kernel
-// (ranks 8 and 16 only) and written out.
-bool skinny_supported(const qlora_desc& d, int M);
-int launch_skinny_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
-                       const void* zeros, const void* Ldown, const void* Lup, float* P, bool p_is_input, void* Out,
-                       cudaStream_t st);
+                     cudaStream_t st, const void* Ldown = nullptr, unsigned int* sync = nullptr);
 // stream_kernel.cu -- few tokens (M <= 16): cp.async-fed mma.sync kernels on raw codes, the contraction split over a
-// cluster; same arguments as launch_skinny_gemm (the down-projection is computed inside for ranks up to 16).
+// cluster.  Ldown / Lup: the adapter applied first / second (forward A, B; backward B, A).  P = H or G, fp32 [M, r]: read
+// when p_is_input, otherwise computed inside the kernel (ranks up to 16) and written out.
 bool stream_supported(const qlora_desc& d, int M, bool transposed);
 int launch_stream_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
                        const void* zeros, const void* Ldown, const void* Lup, float* P, bool p_is_input, void* Out,
                        cudaStream_t st);
 int read_device_status(unsigned int* out, int clear);
+int launch_wait_probe(int limit_us, cudaStream_t st);   // a wait that is known to run out after limit_us (self-test)
 
 }  // namespace qlora

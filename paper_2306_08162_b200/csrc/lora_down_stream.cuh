@@ -174,7 +174,7 @@ __device__ __forceinline__ void lora_down_stream(int M, int T, int r, const __nv
 }
 
 struct LdsParams {
-    int M, T, r, stages;
+    int M, T, r, stages, wait_limit_us;
     const __nv_bfloat16* In;
     const __nv_bfloat16* L;
     float* P;
@@ -183,15 +183,15 @@ struct LdsParams {
 template <bool L_IS_A>
 __global__ void __launch_bounds__(kThreads, 1) lora_down_stream_kernel(const LdsParams p) {
     extern __shared__ uint8_t lds_raw[];
-    __shared__ int abort_flag_s;
+    __shared__ int abort_flag_s[2];   // [0] set when a wait gave up, [1] the wait limit in microseconds
     pdl_launch_dependents();
     uint8_t* smem = lds_raw + ((128u - (smem_u32(lds_raw) & 127u)) & 127u);
-    if (threadIdx.x == 0) abort_flag_s = 0;
+    if (threadIdx.x == 0) { abort_flag_s[0] = 0; abort_flag_s[1] = p.wait_limit_us; }
     __syncthreads();
     pdl_wait();
-    if (p.r <= 8) lora_down_stream<L_IS_A, 1>(p.M, p.T, p.r, p.In, p.L, p.P, (int)blockIdx.x, (int)gridDim.x, smem, p.stages, &abort_flag_s);
-    else          lora_down_stream<L_IS_A, 2>(p.M, p.T, p.r, p.In, p.L, p.P, (int)blockIdx.x, (int)gridDim.x, smem, p.stages, &abort_flag_s);
-    if (abort_flag_s) {   // give copies that may still be in flight time to land before the CTA's memory is released
+    if (p.r <= 8) lora_down_stream<L_IS_A, 1>(p.M, p.T, p.r, p.In, p.L, p.P, (int)blockIdx.x, (int)gridDim.x, smem, p.stages, abort_flag_s);
+    else          lora_down_stream<L_IS_A, 2>(p.M, p.T, p.r, p.In, p.L, p.P, (int)blockIdx.x, (int)gridDim.x, smem, p.stages, abort_flag_s);
+    if (abort_flag_s[0]) {   // give copies that may still be in flight time to land before the CTA's memory is released
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
         __syncthreads();
     }
@@ -204,16 +204,11 @@ int launch_lora_down_stream_impl(int M, int T, int r, bool l_is_A, const void* I
     int grid = n_blocks < sm_count() ? n_blocks : sm_count();
     if ((n_blocks + grid - 1) / grid > LDS_MAXB) grid = (n_blocks + LDS_MAXB - 1) / LDS_MAXB;   // several waves of CTAs
     LdsParams p{};
-    p.M = M; p.T = T; p.r = r; p.stages = 6;
+    p.M = M; p.T = T; p.r = r; p.stages = 6; p.wait_limit_us = kWaitLimitUs;
     p.In = (const __nv_bfloat16*)In; p.L = (const __nv_bfloat16*)L; p.P = P;
     const size_t smem_bytes = lds_smem_bytes(p.stages) + 128;
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(lora_down_stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess ||
-            cudaFuncSetAttribute(lora_down_stream_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
-            return QLORA_ERR_CUDA;
-        configured = true;
-    }
+    static SmemLimit limit_a, limit_b;
+    if (!limit_a.raise(lora_down_stream_kernel<true>, smem_bytes) || !limit_b.raise(lora_down_stream_kernel<false>, smem_bytes)) return QLORA_ERR_CUDA;
     const cudaError_t err = l_is_A ? launch_pdl(lora_down_stream_kernel<true>, dim3((unsigned)grid), dim3(kThreads), smem_bytes, st, 1, p)
                                    : launch_pdl(lora_down_stream_kernel<false>, dim3((unsigned)grid), dim3(kThreads), smem_bytes, st, 1, p);
     return err == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;

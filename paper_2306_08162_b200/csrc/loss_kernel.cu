@@ -12,6 +12,7 @@
 // every thread prefetches ITS OWN chunks of the block's next row into shared memory with cp.async (thread-private slots:
 // no barrier is involved, the thread just waits for its own copies) and moves them to registers when the row's turn comes.
 #include "common.cuh"
+#include "device_state.h"
 #include "launch.h"
 
 namespace qlora {
@@ -160,18 +161,13 @@ int launch_lrec_loss(int T, int V, const void* Z, const void* Tt, const int32_t*
     if (T == 0) return QLORA_OK;
     const int chunks = V / 8;
     const int ch = (chunks + LL_THREADS - 1) / LL_THREADS;
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     const unsigned grid = (unsigned)(T < sms ? T : sms);   // one block per SM (registers), persistent over the rows
     cudaError_t err;
 #define QLORA_LL(CHV)                                                                                                  \
     {                                                                                                                  \
-        static bool configured = false;                                                                                \
-        if (!configured) {                                                                                             \
-            if (cudaFuncSetAttribute(lrec_loss_kernel<CHV>, cudaFuncAttributeMaxDynamicSharedMemorySize,                \
-                                     2 * CHV * LL_THREADS * 16) != cudaSuccess) return QLORA_ERR_CUDA;                  \
-            configured = true;                                                                                         \
-        }                                                                                                              \
+        static SmemLimit limit;                                                                                        \
+        if (!limit.raise(lrec_loss_kernel<CHV>, (size_t)2 * CHV * LL_THREADS * 16)) return QLORA_ERR_CUDA;             \
     }                                                                                                                  \
     err = launch_pdl(lrec_loss_kernel<CHV>, dim3(grid), dim3(LL_THREADS), (size_t)2 * CHV * LL_THREADS * 16, st, 1, T, V, (const __nv_bfloat16*)Z, \
                      (const __nv_bfloat16*)Tt, labels, lambda_kl, lambda_ce, grad_scale, loss_tokens, (__nv_bfloat16*)dZ)

@@ -2,6 +2,7 @@
 // and serve (a) shapes the tensor-core kernels do not tile, and (b) the skinny LoRA products, which are bound by
 // HBM traffic rather than by arithmetic (Figure 1 of the paper: the green "MM" blocks and their gradients).
 #include "common.cuh"
+#include "device_state.h"
 #include "launch.h"
 #include "lora_down.cuh"
 
@@ -393,12 +394,8 @@ int launch_lora_grads(int M, int K, int N, int r, float s, const void* X, const 
         const dim3 grid((unsigned)(col_blocks * cl), 1, 2);
 #define QLORA_LGC(RTV, CLV)                                                                                    \
     do {                                                                                                       \
-        static bool configured = false;                                                                        \
-        if (!configured) {                                                                                     \
-            if (cudaFuncSetAttribute(lora_grad_partial_kernel<RTV, CLV>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                     RTV * 16 * (1024 + 8) * 2) != cudaSuccess) return QLORA_ERR_CUDA;          \
-            configured = true;                                                                                 \
-        }                                                                                                      \
+        static SmemLimit limit;                                                                                \
+        if (!limit.raise(lora_grad_partial_kernel<RTV, CLV>, (size_t)RTV * 16 * (1024 + 8) * 2)) return QLORA_ERR_CUDA; \
         err = launch_pdl(lora_grad_partial_kernel<RTV, CLV>, grid, dim3(LG_WARPS * 32), smem, st, CLV, M, r, rows_cl, sB, sA, accumulate); \
     } while (0)
 #define QLORA_LGC_RT(CLV)                                                                                      \
@@ -427,12 +424,8 @@ int launch_lora_grads(int M, int K, int N, int r, float s, const void* X, const 
     const size_t smem = (size_t)rt * 16 * (plan.rows_per_slice + 8) * sizeof(__nv_bfloat16);
 #define QLORA_LG(RTV)                                                                                          \
     do {                                                                                                       \
-        static bool configured = false;                                                                        \
-        if (!configured) {                                                                                     \
-            if (cudaFuncSetAttribute(lora_grad_partial_kernel<RTV, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                     RTV * 16 * (1024 + 8) * 2) != cudaSuccess) return QLORA_ERR_CUDA;          \
-            configured = true;                                                                                 \
-        }                                                                                                      \
+        static SmemLimit limit;                                                                                \
+        if (!limit.raise(lora_grad_partial_kernel<RTV, 0>, (size_t)RTV * 16 * (1024 + 8) * 2)) return QLORA_ERR_CUDA; \
         err = launch_pdl(lora_grad_partial_kernel<RTV, 0>, grid, dim3(LG_WARPS * 32), smem, st, 1, M, r, plan.rows_per_slice, sB, sA, accumulate); \
     } while (0)
     switch (rt) {

@@ -37,12 +37,13 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "device_state.h"
 #include "launch.h"
 
 namespace qlora {
 namespace {
 
-constexpr int ST_MAX_DEVICES = 64;
+constexpr int ST_MAX_DEVICES = kMaxDevices;
 
 template <int BITS>
 struct Fmt {

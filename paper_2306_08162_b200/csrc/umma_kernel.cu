@@ -21,9 +21,9 @@
 #include <cuda.h>
 
 #include <mutex>
-#include <unordered_map>
 
 #include "common.cuh"
+#include "device_state.h"
 #include "launch.h"
 #include "lora_down.cuh"
 
@@ -31,11 +31,10 @@ namespace qlora {
 
 __device__ unsigned int g_device_status = 0;   // sticky; bit 0: an mbarrier wait timed out
 
-// Counter pairs of the CTA-pair kernel's producer clusters: [0] producer CTAs that have published their rows,
-// [1] tile CTAs that have seen the full count.  Zero whenever no launch is using the pair (the kernel restores that).
-constexpr int kSyncSlots = 4096;
-__device__ unsigned int g_pair_sync[kSyncSlots][2];
-int sync_slot_for(const void* key);   // host: the counter pair of a workspace address (-1: table full)
+// The producer clusters of a launch signal its tile CTAs through a pair of counters in the CALLER's workspace (the layer
+// calls carve two words out of it): [0] producer CTAs that have published their rows, [1] tile CTAs that have seen the
+// full count.  A one-warp kernel ahead of the launch sets the pair to zero (in stream order, with programmatic dependent
+// launch, so the main kernel's set-up still overlaps its predecessor); the last tile CTA zeroes it again.
 
 namespace {
 
@@ -47,7 +46,7 @@ constexpr int kStepC = 64;           // contraction elements per pipeline stage
 constexpr int kWStageBytes = kWRows * kStepC * 2;   // 16 KiB of bf16 per stage
 constexpr int kAccStride = 256;      // tensor-memory columns per accumulator buffer
 constexpr uint32_t kSpinLimit = 1u << 26;
-constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any healthy wait, short enough not to look like a hang
+constexpr int kWaitLimitUs = 250000;   // default limit of a wait, a launch parameter: far beyond any healthy wait (microseconds), short for a hang
 
 struct Params {
     int M, N, K, bits, g, r, r_pad;
@@ -67,7 +66,9 @@ struct Params {
     __nv_bfloat16* Out;
     // producer clusters (n_prod > 0, as in the CTA-pair kernel): the first n_prod clusters of the grid compute
     // P = In * Ldown into Pout (== Pmat) beside the tiles and publish it through counter pair `slot`
-    int n_prod, T, slot, lds_stages;
+    int n_prod, T, lds_stages;
+    unsigned int* sync;   // the counter pair (n_prod > 0)
+    int wait_limit_us;    // every wait inside the kernel gives up after this long
     const __nv_bfloat16* In;         // [M, T]
     const __nv_bfloat16* Ldown;      // A [r, K] (forward) or B [N, r] (backward)
     float* Pout;
@@ -99,7 +100,8 @@ __device__ __forceinline__ uint64_t global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait: gives up after kWaitLimitNs of wall time (or kSpinLimit polls).  Returns false when the kernel is
+// Bounded wait: gives up after abort_flag[1] microseconds of wall time (the launch's limit, set beside the flag when the
+// kernel starts) or kSpinLimit polls.  Returns false when the kernel is
 // aborting (this wait or another one ran out).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     uint64_t t0 = 0;
@@ -109,7 +111,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_flag) return false;
             const uint64_t now = global_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) break;
+            else if (now - t0 > (uint64_t)abort_flag[1] * 1000ull) break;
         }
     }
     *abort_flag = 1;
@@ -173,11 +175,6 @@ __device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t cluster_addr) {
     asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(cluster_addr) : "memory");
     return v;
 }
-__device__ __forceinline__ float ld_cluster_f32(uint32_t cluster_addr) {
-    float v;
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr) : "memory");
-    return v;
-}
 
 
 // Bounded wait until a counter in global memory reaches `target` (written by other CTAs of the same launch).
@@ -192,7 +189,7 @@ __device__ __forceinline__ bool wait_counter(const unsigned* ctr, unsigned targe
             if (*abort_flag) return false;
             const uint64_t now = global_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) break;
+            else if (now - t0 > (uint64_t)abort_flag[1] * 1000ull) break;
         }
     }
     *abort_flag = 1;
@@ -200,7 +197,6 @@ __device__ __forceinline__ bool wait_counter(const unsigned* ctr, unsigned targe
     return false;
 }
 
-int sm_count();
 #include "lora_down_stream.cuh"
 
 // Shared-memory matrix descriptor (version 1).  Offsets in bytes; layout 0 = no swizzle, 2 = 128-byte swizzle.
@@ -227,8 +223,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                  const Params p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t tmem_base_slot;
-    __shared__ int abort_flag_s;
-    volatile int* abort_flag = &abort_flag_s;
+    __shared__ int abort_flag_s[2];   // [0] set when a wait gave up, [1] the launch's wait limit in microseconds
+    volatile int* abort_flag = abort_flag_s;
     pdl_launch_dependents();
 
     const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -247,7 +243,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     const uint32_t bar_lora_full = bar_acc_empty + 16;      // [1]  LoRA operand tiles staged
 
     if (threadIdx.x == 0) {
-        abort_flag_s = 0;
+        abort_flag_s[0] = 0; abort_flag_s[1] = p.wait_limit_us;
         for (uint32_t i = 0; i < S; ++i) {
             mbar_init(bar_full_x + 8 * i, 1 + kGroupWarps);
             mbar_init(bar_empty + 8 * i, 1);
@@ -291,7 +287,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         else          lora_down_stream<!TRANSPOSED, 2>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, n_ctas, smem_gen, p.lds_stages, abort_flag);
         __threadfence();       // every thread's rows of P are visible device-wide before the CTA is counted
         __syncthreads();
-        if (threadIdx.x == 0) atomicAdd(&g_pair_sync[p.slot][0], 1u);
+        if (threadIdx.x == 0) atomicAdd(&p.sync[0], 1u);
     } else if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer: activation tiles
         if (lane == 0) {
@@ -397,11 +393,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             if (p.n_prod > 0 && tile_it == 0 && rank == 0) {
                 // P is being computed by this launch's producer clusters: one thread waits for all of their CTAs, is counted
                 // as done with the counter, and the last such CTA of the launch zeroes the pair for the next one.
-                if (et == 0 && wait_counter(&g_pair_sync[p.slot][0], (unsigned)(p.n_prod * p.split), abort_flag)) {
+                if (et == 0 && wait_counter(&p.sync[0], (unsigned)(p.n_prod * p.split), abort_flag)) {
                     const unsigned n_cons = gridDim.x / (unsigned)p.split - (unsigned)p.n_prod;   // one waiting CTA per tile cluster
-                    if (atomicAdd(&g_pair_sync[p.slot][1], 1u) == n_cons - 1u) {
-                        atomicExch(&g_pair_sync[p.slot][0], 0u);
-                        atomicExch(&g_pair_sync[p.slot][1], 0u);
+                    if (atomicAdd(&p.sync[1], 1u) == n_cons - 1u) {
+                        atomicExch(&p.sync[0], 0u);
+                        atomicExch(&p.sync[1], 0u);
                     }
                 }
                 asm volatile("bar.sync 2, %0;" ::"r"(kEpiWarps * 32) : "memory");
@@ -620,14 +616,18 @@ bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const
               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int sm_count() {
-    static int n = [] {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
-        return v;
-    }();
-    return n;
+// Sets a launch's counter pair to zero.  It is launched like the layer kernels (programmatic stream serialization): it
+// lets its successor start at once and writes only after its own predecessor -- whose last tile CTAs may still be
+// using the pair -- has completed; the kernel behind it touches the pair only after griddepcontrol.wait, i.e. after this
+// grid has completed.
+__global__ void sync_zero_kernel(unsigned int* sync) {
+    pdl_launch_dependents();
+    pdl_wait();
+    if (threadIdx.x < 2) sync[threadIdx.x] = 0u;
+}
+
+int zero_sync_pair(unsigned int* sync, cudaStream_t st) {
+    return launch_pdl(sync_zero_kernel, dim3(1), dim3(32), 0, st, 1, sync) == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
 }
 
 // Ldown != NULL: P = In * Ldown is still to be computed.  Where the tile clusters leave room for more clusters on the GPU
@@ -635,17 +635,18 @@ int sm_count() {
 // it beside the tiles; else a down-projection launch goes ahead of the kernel.
 template <int BITS, bool TRANSPOSED>
 int launch_impl(const CUtensorMap& ta, const CUtensorMap& tq, const CUtensorMap& ts, const CUtensorMap& tz, const Params& p_in,
-                size_t smem_bytes, int grid, cudaStream_t st, const void* Ldown, const void* sync_key) {
-    static bool configured = false;   // raising the dynamic shared-memory limit is a per-function, per-process setting
-    static int max_clusters[5] = {0, 0, 0, 0, 0};   // by cluster width
+                size_t smem_bytes, int grid, cudaStream_t st, const void* Ldown, unsigned int* sync) {
+    static SmemLimit limit;
+    static std::mutex mu;
+    static int max_clusters_dev[kMaxDevices][5] = {};   // per device, by cluster width
     auto kern = umma_gemm_kernel<BITS, TRANSPOSED>;
-    if (!configured) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024) != cudaSuccess) return QLORA_ERR_CUDA;
-        configured = true;
-    }
+    if (!limit.raise(kern, 232448 - 1024)) return QLORA_ERR_CUDA;
     Params p = p_in;
-    p.n_prod = 0; p.slot = 0;
+    p.n_prod = 0; p.sync = nullptr; p.wait_limit_us = kWaitLimitUs;
     if (Ldown != nullptr && p.r > 0) {
+        std::lock_guard<std::mutex> lock(mu);
+        const int dev = device_ordinal();
+        int* max_clusters = max_clusters_dev[dev < 0 ? 0 : dev];
         if (max_clusters[p.split] == 0) {
             cudaLaunchConfig_t cfg{};
             cfg.gridDim = dim3((unsigned)(sm_count() / p.split * p.split));
@@ -665,11 +666,12 @@ int launch_impl(const CUtensorMap& ta, const CUtensorMap& tq, const CUtensorMap&
         int n_prod = (n_blocks + p.split - 1) / p.split;           // one row block per producer CTA when there is room
         if (n_prod > idle) n_prod = idle;
         const bool fits = p.r <= 16 && n_prod > 0 && n_prod * p.split * 2 >= n_blocks && p.lds_stages >= LDS_MIN_STAGES;
-        const int slot = (fits && sync_key != nullptr) ? sync_slot_for(sync_key) : -1;
-        if (slot >= 0) {
+        if (fits && sync != nullptr) {
             p.n_prod = n_prod;
-            p.slot = slot;
+            p.sync = sync;
             grid += n_prod * p.split;
+            const int rc = zero_sync_pair(sync, st);
+            if (rc != QLORA_OK) return rc;
         } else {
             const int rc = launch_lora_down(p.M, p.T, p.r, !TRANSPOSED, p.In, p.Ldown, p.Pout, st);
             if (rc != QLORA_OK) return rc;
@@ -681,91 +683,11 @@ int launch_impl(const CUtensorMap& ta, const CUtensorMap& tq, const CUtensorMap&
 }
 
 #include "umma_pair.cuh"
-#include "skinny_kernel.cuh"
 
 }  // namespace
 
 int launch_lora_down_stream(int M, int T, int r, bool l_is_A, const void* In, const void* L, float* P, cudaStream_t st) {
     return launch_lora_down_stream_impl(M, T, r, l_is_A, In, L, P, st);
-}
-
-bool skinny_supported(const qlora_desc& d, int M) {
-    if (M < 1 || M > 32) return false;
-    if (d.K < 32 || d.N < 8) return false;
-    // a forward stage of 256 k and a backward tile of 128 k must hold whole groups (or lie inside one)
-    return (SK_STAGE % d.group_size == 0 || d.group_size % SK_STAGE == 0) && (SK_TILE % d.group_size == 0 || d.group_size % SK_TILE == 0);
-}
-
-int launch_skinny_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
-                       const void* zeros, const void* Ldown, const void* Lup, float* P, bool p_is_input, void* Out,
-                       cudaStream_t st) {
-    SkinnyParams p{};
-    p.M = M; p.N = d.N; p.K = d.K; p.bits = d.bits; p.g = d.group_size; p.r = d.r;
-    p.T = transposed ? d.N : d.K;
-    p.C = transposed ? d.K : d.N;
-    p.stages_total = (p.T + SK_STAGE - 1) / SK_STAGE;
-    // forward: packed tile 256 k x 128 n, group rows of the stage's 256 k; backward: 128 k x 256 n, group rows of the 128 k
-    const int span_k = transposed ? SK_TILE : SK_STAGE;
-    p.scale_rows = d.group_size < span_k ? span_k / d.group_size : 1;
-    p.words_bytes = (uint32_t)(d.bits * 4096);                       // 256 x 128 codes (either orientation)
-    p.scale_bytes = (uint32_t)(p.scale_rows * (transposed ? SK_STAGE : SK_TILE) * 2);
-    const int ntl = (d.r > 0 && !p_is_input) ? d.r / 8 : 0;          // fused down-projection tiles (r = 8 or 16)
-    if (ntl > 2) return QLORA_ERR_INVALID_ARG;
-    p.act_bytes = 16 * SK_STAGE * 2;                                 // 16 token rows x 256 contraction elements, bf16
-    p.l_bytes = ntl > 0 ? (uint32_t)(transposed ? SK_STAGE * d.r * 2 : 8 * ntl * SK_STAGE * 2) : 0u;
-    p.off_scale = p.words_bytes;
-    p.off_zero = p.off_scale + p.scale_bytes;                        // multiples of 512 bytes
-    p.off_act = (p.off_zero + p.scale_bytes + 1023u) / 1024u * 1024u;
-    p.off_l = p.off_act + p.act_bytes;
-    p.stage_bytes = (p.off_l + p.l_bytes + 1023u) / 1024u * 1024u;
-    const int my_stages = (p.stages_total + SK_SPLIT - 1) / SK_SPLIT;   // stages of the busiest CTA of a cluster
-    int S = (int)((200u * 1024u) / p.stage_bytes);
-    if (S > SK_MAX_STAGES) S = SK_MAX_STAGES;
-    if (S >= my_stages) S = my_stages;
-    else S = S / 2 * 2;   // even and odd stages have their own consumer warps: a slot must keep its parity lap after lap
-    if (S < 1) return QLORA_ERR_UNSUPPORTED;
-    p.S = S;
-    const uint32_t part_bytes = SK_PLANES * 16 * SK_PW * 4;                  // partial tiles; they reuse the ring after the main loop
-    const uint32_t ring_bytes = (uint32_t)S * p.stage_bytes;
-    p.off_p = (ring_bytes > part_bytes ? ring_bytes : part_bytes);
-    p.off_bar = p.off_p + 16 * 16 * 4;
-    const size_t smem_bytes = (size_t)p.off_bar + 2 * 8 * SK_MAX_STAGES + 1024;
-    p.s = d.r > 0 ? d.alpha / (float)d.r : 0.f;
-    p.Lup = (const __nv_bfloat16*)Lup;
-    p.Ldown = (const __nv_bfloat16*)Ldown;
-    p.P = P; p.p_is_input = p_is_input ? 1 : 0; p.Out = (__nv_bfloat16*)Out;
-
-    CUtensorMap tq, ts, tz, ta, tl;
-    const uint32_t bx = transposed ? SK_STAGE : SK_TILE;             // packed columns (n) per box
-    const uint32_t by = (uint32_t)((transposed ? SK_TILE : SK_STAGE) / 32 * d.bits);   // packed rows per box
-    if (!make_map_2d(&tq, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, Q, (uint64_t)d.N, (uint64_t)(d.K * d.bits / 32), bx, by, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-        !make_map_2d(&ts, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, scales, (uint64_t)d.N, (uint64_t)(d.K / d.group_size), bx, (uint32_t)p.scale_rows, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-        !make_map_2d(&tz, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, zeros, (uint64_t)d.N, (uint64_t)(d.K / d.group_size), bx, (uint32_t)p.scale_rows, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-        !make_map_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, In, (uint64_t)p.T, (uint64_t)M, 64, 16, CU_TENSOR_MAP_SWIZZLE_128B))
-        return QLORA_ERR_CUDA;
-    if (ntl > 0) {
-        const bool ok = transposed
-            ? make_map_2d(&tl, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Ldown, (uint64_t)d.r, (uint64_t)d.N, (uint32_t)d.r, SK_STAGE, CU_TENSOR_MAP_SWIZZLE_NONE)
-            : make_map_2d(&tl, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Ldown, (uint64_t)d.K, (uint64_t)d.r, 64, (uint32_t)(8 * ntl), CU_TENSOR_MAP_SWIZZLE_128B);
-        if (!ok) return QLORA_ERR_CUDA;
-    } else {
-        tl = ta;   // unused by the kernel
-    }
-    dim3 grid(SK_SPLIT, (unsigned)((p.C + SK_TILE - 1) / SK_TILE), (unsigned)((M + 15) / 16));
-#define QLORA_SK(B, NT)                                                                                      \
-    return transposed ? launch_skinny_impl<B, NT, true>(tq, ts, tz, ta, tl, p, smem_bytes, grid, st)        \
-                      : launch_skinny_impl<B, NT, false>(tq, ts, tz, ta, tl, p, smem_bytes, grid, st)
-#define QLORA_SK_BITS(NT)                  \
-    switch (d.bits) {                      \
-        case 2: QLORA_SK(2, NT);           \
-        case 3: QLORA_SK(3, NT);           \
-        case 4: QLORA_SK(4, NT);           \
-        case 8: QLORA_SK(8, NT);           \
-    }
-    if (ntl == 0) { QLORA_SK_BITS(0) } else if (ntl == 1) { QLORA_SK_BITS(1) } else { QLORA_SK_BITS(2) }
-#undef QLORA_SK_BITS
-#undef QLORA_SK
-    return QLORA_ERR_UNSUPPORTED;
 }
 
 bool umma_supported(const qlora_desc& d, int M) {
@@ -777,23 +699,9 @@ bool umma_supported(const qlora_desc& d, int M) {
 }
 
 // CTA-pair kernel: 512 tokens x 256 weight rows per pair of SMs (see prefer_pair_kernel for when it is used).
-// One counter pair per key (the caller's workspace address), handed out on first sight and kept: two launches that can
-// overlap in time have different workspaces, hence different pairs.  -1 when the table is full.
-int sync_slot_for(const void* key) {
-    static std::mutex mu;
-    static std::unordered_map<const void*, int> table;
-    std::lock_guard<std::mutex> lock(mu);
-    const auto it = table.find(key);
-    if (it != table.end()) return it->second;
-    if ((int)table.size() >= kSyncSlots) return -1;
-    const int slot = (int)table.size();
-    table.emplace(key, slot);
-    return slot;
-}
-
 static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
                             const void* zeros, const void* L, float* Pmat, void* Out, cudaStream_t st, const void* Ldown,
-                            const void* sync_key) {
+                            unsigned int* sync) {
     PairParams p{};
     p.M = M; p.N = d.N; p.K = d.K; p.bits = d.bits; p.g = d.group_size; p.r = d.r; p.r_pad = (d.r + 15) / 16 * 16;
     p.C = transposed ? d.K : d.N;
@@ -839,7 +747,7 @@ static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const v
     const int pairs = sm_count() / 2;
     // P = In * Ldown still to be computed: on SM pairs the tiles leave idle when they can take all row blocks (they are
     // then done well before the tiles' contractions are), else by a launch ahead of this one.  Both sum in the same order.
-    p.n_prod = 0; p.T = T; p.slot = 0;
+    p.n_prod = 0; p.T = T; p.sync = nullptr; p.wait_limit_us = kWaitLimitUs;
     p.In = (const __nv_bfloat16*)In; p.Ldown = (const __nv_bfloat16*)Ldown; p.Pout = Pmat;
     p.lds_stages = (int)((p.off_bar - LDS_BAR_BYTES) / LDS_STAGE_BYTES);
     if (p.lds_stages > 6) p.lds_stages = 6;
@@ -850,10 +758,11 @@ static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const v
         int n_prod = (n_blocks + 3) / 4;                     // four row blocks per producer CTA pair when there is room
         if (n_prod > idle) n_prod = idle;
         const bool fits = d.r <= 16 && n_prod > 0 && n_prod * 2 * LDS_MAXB >= n_blocks && p.lds_stages >= LDS_MIN_STAGES;
-        const int slot = (fits && sync_key != nullptr) ? sync_slot_for(sync_key) : -1;
-        if (slot >= 0) {
+        if (fits && sync != nullptr) {
             p.n_prod = n_prod;
-            p.slot = slot;
+            p.sync = sync;
+            const int rc = zero_sync_pair(sync, st);
+            if (rc != QLORA_OK) return rc;
         } else {
             const int rc = launch_lora_down(M, T, d.r, !transposed, In, Ldown, Pmat, st);
             if (rc != QLORA_OK) return rc;
@@ -896,8 +805,8 @@ static bool prefer_pair_kernel(const qlora_desc& d, int M, bool transposed) {
 
 int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
                      const void* zeros, const void* L, float* Pmat, void* Out, cudaStream_t st, const void* Ldown,
-                     const void* sync_key) {
-    if (prefer_pair_kernel(d, M, transposed)) return launch_umma_pair(d, M, transposed, In, Q, scales, zeros, L, Pmat, Out, st, Ldown, sync_key);
+                     unsigned int* sync) {
+    if (prefer_pair_kernel(d, M, transposed)) return launch_umma_pair(d, M, transposed, In, Q, scales, zeros, L, Pmat, Out, st, Ldown, sync);
     Params p{};
     p.M = M; p.N = d.N; p.K = d.K; p.bits = d.bits; p.g = d.group_size; p.r = d.r; p.r_pad = (d.r + 15) / 16 * 16;
     p.C = transposed ? d.K : d.N;
@@ -961,8 +870,8 @@ int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In
     p.lds_stages = (int)((p.off_bar - LDS_BAR_BYTES) / LDS_STAGE_BYTES);
     if (p.lds_stages > 6) p.lds_stages = 6;
 #define QLORA_LAUNCH(B)                                                                              \
-    return transposed ? launch_impl<B, true>(ta, tq, ts, tz, p, smem_bytes, grid, st, Ldown, sync_key)  \
-                      : launch_impl<B, false>(ta, tq, ts, tz, p, smem_bytes, grid, st, Ldown, sync_key)
+    return transposed ? launch_impl<B, true>(ta, tq, ts, tz, p, smem_bytes, grid, st, Ldown, sync)  \
+                      : launch_impl<B, false>(ta, tq, ts, tz, p, smem_bytes, grid, st, Ldown, sync)
     switch (d.bits) {
         case 2: QLORA_LAUNCH(2);
         case 3: QLORA_LAUNCH(3);
@@ -973,16 +882,34 @@ int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In
     return QLORA_ERR_UNSUPPORTED;
 }
 
+namespace {
+// The give-up path of the bounded waits, exercised without stalling any real kernel: one thread of one CTA waits with
+// the library's own mbar_wait on a barrier in shared memory that nobody ever arrives at, with `limit_us` as the limit.  The
+// wait runs out, sets the sticky status word and returns false; the kernel then ends normally (no TMA, no tensor memory).
+__global__ void wait_probe_kernel(int limit_us) {
+    __shared__ uint64_t bar;
+    __shared__ int flag[2];
+    if (threadIdx.x == 0) {
+        flag[0] = 0; flag[1] = limit_us;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) (void)mbar_wait(smem_u32(&bar), 0u, flag);
+}
+}  // namespace
+
+int launch_wait_probe(int limit_us, cudaStream_t st) {
+    wait_probe_kernel<<<1, 32, 0, st>>>(limit_us);
+    return cudaGetLastError() == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
+}
+
 int read_device_status(unsigned int* out, int clear) {
     unsigned int v = 0;
     if (cudaMemcpyFromSymbol(&v, g_device_status, sizeof(v)) != cudaSuccess) return QLORA_ERR_CUDA;
     if (clear && v != 0) {
         const unsigned int zero = 0;
         if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(zero)) != cudaSuccess) return QLORA_ERR_CUDA;
-        // a launch that gave up may have left its counter pair non-zero (the caller has synchronised the device)
-        void* sync = nullptr;
-        if (cudaGetSymbolAddress(&sync, g_pair_sync) != cudaSuccess || cudaMemset(sync, 0, sizeof(unsigned int) * 2 * kSyncSlots) != cudaSuccess)
-            return QLORA_ERR_CUDA;
     }
     *out = v;
     return QLORA_OK;

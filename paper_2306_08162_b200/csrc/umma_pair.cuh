@@ -42,7 +42,9 @@ struct PairParams {
     const __nv_bfloat16* L;      // B [N, r] (forward) or A [r, K] (backward)
     __nv_bfloat16* Out;
     // producer clusters (n_prod > 0): P = In * Ldown is computed by this launch and written to Pout (== Pmat)
-    int n_prod, T, slot, lds_stages;
+    int n_prod, T, lds_stages;
+    unsigned int* sync;          // the launch's counter pair (n_prod > 0)
+    int wait_limit_us;           // every wait inside the kernel gives up after this long
     const __nv_bfloat16* In;     // [M, T]
     const __nv_bfloat16* Ldown;  // A [r, K] (forward) or B [N, r] (backward)
     float* Pout;
@@ -70,7 +72,7 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
             if (*abort_flag) return false;
             const uint64_t now = global_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) break;
+            else if (now - t0 > (uint64_t)abort_flag[1] * 1000ull) break;
         }
     }
     *abort_flag = 1;
@@ -119,8 +121,8 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                  const PairParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t tmem_base_slot;
-    __shared__ int abort_flag_s;
-    volatile int* abort_flag = &abort_flag_s;
+    __shared__ int abort_flag_s[2];   // [0] set when a wait gave up, [1] the launch's wait limit in microseconds
+    volatile int* abort_flag = abort_flag_s;
     pdl_launch_dependents();
 
     const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -149,7 +151,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     const uint32_t bar_lora_full = bar_acc_empty + 8;       // [1] leader's: both CTAs' LoRA operand tiles staged
 
     if (threadIdx.x == 0) {
-        abort_flag_s = 0;
+        abort_flag_s[0] = 0; abort_flag_s[1] = p.wait_limit_us;
         for (uint32_t i = 0; i < S; ++i) {
             mbar_init(bar_full_x + 8 * i, 1 + 2 * kGroupWarps);
             mbar_init(bar_empty + 8 * i, 1);
@@ -183,7 +185,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         else          lora_down_stream<!TRANSPOSED, 2>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, 2 * p.n_prod, smem_gen, p.lds_stages, abort_flag);
         __threadfence();       // every thread's rows of P are visible device-wide before the CTA is counted
         __syncthreads();
-        if (threadIdx.x == 0) atomicAdd(&g_pair_sync[p.slot][0], 1u);
+        if (threadIdx.x == 0) atomicAdd(&p.sync[0], 1u);
         fence_proxy_async();   // the shared memory just used goes to the TMA / tensor-core side for this cluster's tiles, if any
         __syncthreads();
     }
@@ -296,11 +298,11 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             if (p.n_prod > 0 && tile_it == 0) {
                 // P is being computed by the producer clusters of this launch: one thread waits for all of their CTAs, is
                 // counted as done with the counter, and the last such CTA of the launch zeroes the pair for the next one.
-                if (et == 0 && wait_counter(&g_pair_sync[p.slot][0], 2u * (unsigned)p.n_prod, abort_flag)) {
+                if (et == 0 && wait_counter(&p.sync[0], 2u * (unsigned)p.n_prod, abort_flag)) {
                     const unsigned n_cons = 2u * (unsigned)(p.n_tiles < tile_stride ? p.n_tiles : tile_stride);   // CTAs that have a tile
-                    if (atomicAdd(&g_pair_sync[p.slot][1], 1u) == n_cons - 1u) {
-                        atomicExch(&g_pair_sync[p.slot][0], 0u);
-                        atomicExch(&g_pair_sync[p.slot][1], 0u);
+                    if (atomicAdd(&p.sync[1], 1u) == n_cons - 1u) {
+                        atomicExch(&p.sync[0], 0u);
+                        atomicExch(&p.sync[1], 0u);
                     }
                 }
                 asm volatile("bar.sync 2, %0;" ::"r"(kEpiWarps * 32) : "memory");
@@ -481,12 +483,9 @@ done:
 template <int BITS, bool TRANSPOSED>
 int launch_pair_impl(const CUtensorMap& ta, const CUtensorMap& tq, const CUtensorMap& ts, const CUtensorMap& tz, const PairParams& p,
                      size_t smem_bytes, int grid, cudaStream_t st) {
-    static bool configured = false;
+    static SmemLimit limit;
     auto kern = umma_pair_kernel<BITS, TRANSPOSED>;
-    if (!configured) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024) != cudaSuccess) return QLORA_ERR_CUDA;
-        configured = true;
-    }
+    if (!limit.raise(kern, 232448 - 1024)) return QLORA_ERR_CUDA;
     return launch_pdl(kern, dim3((unsigned)grid), dim3(kThreads), smem_bytes, st, 1, ta, tq, ts, tz, p) == cudaSuccess
                ? QLORA_OK : QLORA_ERR_CUDA;   // (the cluster width of 2 is a compile-time attribute of the kernel)
 }

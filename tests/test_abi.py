@@ -131,3 +131,19 @@ def test_missing_library_fails_loudly(ql, monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "_LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError, match="no fallback"):
         binding.library()
+
+
+def test_host_state_is_per_device_and_nothing_is_keyed_by_caller_pointers():
+    """What the library remembers between calls is kept per device ordinal (arrays of kMaxDevices in device_state.h and
+    beside the occupancy queries); there is no process-wide 'configured' flag and no table keyed by a workspace address."""
+    import glob
+    import re
+    csrc = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "paper_2306_08162_b200", "csrc")
+    text = {os.path.basename(p): open(p).read() for p in glob.glob(os.path.join(csrc, "*"))}
+    for name, src in text.items():
+        assert "unordered_map" not in src and "static bool configured" not in src, name
+        assert not re.search(r"static\s+int\s+n\s*=\s*\[\]", src), name          # a process-wide cached SM count
+    ds = text["device_state.h"]
+    assert "size_t done[kMaxDevices]" in ds and "int cached[kMaxDevices]" in ds and "cudaGetDevice" in ds
+    assert "max_clusters_dev[kMaxDevices]" in text["umma_kernel.cu"]
+    assert "DeviceFacts facts[ST_MAX_DEVICES]" in text["stream_kernel.cu"]
