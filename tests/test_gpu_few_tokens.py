@@ -110,3 +110,37 @@ def test_adapters_rewritten_in_stream_right_before_the_call():
             assert rel_err(to_f64(Yg), ref["Y"]) <= REL_TOL, (bits, M, step)
             assert rel_err(to_f64(dXg), ref["dX"]) <= REL_TOL, (bits, M, step)
         assert not np.array_equal(A0, to_f64(outs[-1][0])) or not np.array_equal(B0, to_f64(outs[-1][1]))
+
+
+@pytest.mark.parametrize("M", [16, 64, 1100])
+def test_weights_repacked_in_stream_right_before_the_call(M):
+    """The packed matrix is the one tensor the kernels read ahead of their dependency wait.  A kernel of the library that
+    rewrites it (qlora_pack) must therefore hold its dependents back until it is done: two code matrices are packed
+    into the SAME buffer in turn, each time immediately before a forward and a backward call in the same stream, on
+    the few-token path (16 tokens), the single-CTA tensor-core path (64) and the CTA-pair path (1100)."""
+    import paper_2306_08162_b200 as ql
+    bits = 4
+    la = qi.random_codes_layer(K=1024, N=1024, bits=bits, group_size=128, r=8, alpha=16.0, M=M, seed=71)
+    lb = dict(la)
+    lb["codes"] = qi.random_codes_layer(K=1024, N=1024, bits=bits, group_size=128, r=8, alpha=16.0, M=M, seed=72)["codes"]
+    gl = GpuLayer(la)
+    codes = [torch.from_numpy(la["codes"]).cuda(), torch.from_numpy(lb["codes"]).cuda()]
+    Y = torch.empty((M, gl.N), dtype=torch.bfloat16, device="cuda")
+    dX = torch.empty((M, gl.K), dtype=torch.bfloat16, device="cuda")
+    outs = []
+    for step in range(20):
+        ql.qlora_pack(bits, gl.K, gl.N, codes[step % 2], gl.Q)
+        ql.qlora_fwd(gl.desc, M, gl.X, gl.Q, gl.scales, gl.zeros, gl.A, gl.B, Y, None, gl.ws)
+        ql.qlora_bwd_input(gl.desc, M, gl.dY, gl.Q, gl.scales, gl.zeros, gl.A, gl.B, dX, None, gl.ws)
+        outs.append((Y.clone(), dX.clone()))
+    torch.cuda.synchronize()
+    assert ql.qlora_device_status() == 0
+    rows = np.unique(np.concatenate([np.arange(min(M, 8)), np.arange(max(M - 8, 0), M)]))
+    refs = [orc.layer_reference(la, rows=rows), orc.layer_reference(lb, rows=rows)]
+    rows_t = torch.from_numpy(rows).cuda()
+    for step, (Yg, dXg) in enumerate(outs):
+        ref = refs[step % 2]
+        assert rel_err(to_f64(Yg[rows_t]), ref["Y"]) <= REL_TOL, (M, step)
+        assert rel_err(to_f64(dXg[rows_t]), ref["dX"]) <= REL_TOL, (M, step)
+    # the two code matrices give different results, so a stale read would have shown
+    assert rel_err(to_f64(outs[0][0][rows_t]), refs[1]["Y"]) > REL_TOL
