@@ -84,8 +84,12 @@ typedef struct {
 } qlora_desc;
 
 /* Bytes of scratch the three layer calls may need for M tokens (the maximum over the calls, so one buffer
- * serves all).  The paper has no counterpart: it is how a library that allocates nothing gets its scratch.  `out` is a host pointer.  The scratch holds H / G when the caller does not keep them, the
- * split partial sums of the LoRA gradients and of small-M products.  Contents are undefined between calls. */
+ * serves all).  The paper has no counterpart: it is how a library that allocates nothing gets its scratch.  `out` is a
+ * host pointer.  The scratch holds H / G when the caller does not keep them, the partial sums of the LoRA gradients, a
+ * few counters, and -- last, and optional -- the area through which two SM pairs exchange the halves of an output tile
+ * whose contraction they share (many tokens, last wave partly filled: up to 12 MiB on LLaMA-7B MLP shapes).  A call
+ * given less than that last part still works, without the split.  Contents are undefined between calls.  The figure is
+ * computed for the current device (its SM count decides what is split). */
 int qlora_workspace_bytes(const qlora_desc* desc, int M, size_t* out);
 
 /* Forward (Figure 1, forward path):  Y = X W^T + s (X A^T) B^T,  bf16 output, fp32 accumulation.
@@ -139,8 +143,9 @@ int qlora_bwd_lora_dropout(const qlora_desc* desc, int M, const void* X, const u
  * because cudaMalloc / cudaFree synchronise the device.  The paper has no counterpart; this is a packaging variant of
  * qlora_bwd_lora: same arguments otherwise, same kernels, same results bit for bit.  Its scratch is a fixed array of
  * QLORA_STATIC_SCRATCH_BYTES inside the library; the call itself allocates and frees nothing.
- *   - Limit: returns QLORA_ERR_STATIC_LIMIT, with nothing enqueued, when qlora_workspace_bytes(desc, M) exceeds
- *     QLORA_STATIC_SCRATCH_BYTES (LLaMA-7B projections at M = 2048 with r <= 16 need 5 - 11 MiB).
+ *   - Limit: returns QLORA_ERR_STATIC_LIMIT, with nothing enqueued, when the scratch qlora_bwd_lora needs (the part of
+ *     qlora_workspace_bytes(desc, M) that is not optional) exceeds QLORA_STATIC_SCRATCH_BYTES (LLaMA-7B projections at
+ *     M = 2048 with r <= 16 need 5 - 11 MiB).
  *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device
  *     current) and remembers it; make that first call before any stream capture begins.
  *   - All calls on a device share the one array, which still holds what the previous call left there.  A call

@@ -35,7 +35,9 @@ int check_desc(const qlora_desc* d, bool need_lora) {
 }
 
 struct Workspace {
-    size_t p0_off, p1_off, grad_off, sync_off, total;
+    size_t p0_off, p1_off, grad_off, sync_off, split_off;
+    size_t required;   // what a call cannot do without
+    size_t total;      // ... plus the exchange area of split tiles (used when it is there)
 };
 
 Workspace carve(const qlora_desc& d, int M) {
@@ -45,11 +47,17 @@ Workspace carve(const qlora_desc& d, int M) {
     w.p1_off = p;
     w.grad_off = 2 * p;
     w.sync_off = w.grad_off + align_up(lora_grad_scratch_bytes(M, d.K, d.N, d.r), 256);
-    w.total = w.sync_off + 256;          // two counters of the tensor-core kernels' producer clusters
+    w.split_off = w.sync_off + 256;      // the counters of the tensor-core kernels: producer clusters, split tiles
+    w.required = w.split_off;
+    w.total = w.split_off + umma_split_scratch_bytes(d, M);
     return w;
 }
 
 }  // namespace
+
+// What the layer calls cannot do without: qlora_workspace_bytes minus the exchange area of split tiles, which
+// qlora_fwd / qlora_bwd_input use only when it is there (and qlora_bwd_lora never).
+size_t qlora::required_workspace_bytes(const qlora_desc& d, int M) { return carve(d, M).required; }
 
 extern "C" {
 
@@ -164,7 +172,7 @@ static int fwd_common(const qlora_desc* desc, int M, const void* X, const uint8_
         !aligned16(A) || !aligned16(B) || !aligned16(H_out) || !aligned16(workspace))
         return QLORA_ERR_ALIGNMENT;
     const Workspace w = carve(d, M);
-    if (workspace == nullptr || workspace_bytes < w.total) return QLORA_ERR_WORKSPACE;
+    if (workspace == nullptr || workspace_bytes < w.required) return QLORA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     float* H = H_out ? H_out : reinterpret_cast<float*>(static_cast<char*>(workspace) + w.p0_off);
     unsigned int* sync = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + w.sync_off);
@@ -177,7 +185,8 @@ static int fwd_common(const qlora_desc* desc, int M, const void* X, const uint8_
         return launch_stream_gemm(d, M, false, X, Q, scales, zeros, A, B, H, !fused, Y, st);
     }
     // the tensor-core path computes H itself when given A (beside its tiles where SM pairs are idle, else ahead of them)
-    if (umma_supported(d, M) && mask == nullptr) return launch_umma_gemm(d, M, false, X, Q, scales, zeros, B, H, Y, st, A, sync);
+    if (umma_supported(d, M) && mask == nullptr) return launch_umma_gemm(d, M, false, X, Q, scales, zeros, B, H, Y, st, A, sync, static_cast<char*>(workspace) + w.split_off,
+                                workspace_bytes - w.split_off);
     if (d.r > 0) {
         rc = launch_lora_down(M, d.K, d.r, true, X, A, H, st, mask, keep_scale);
         if (rc != QLORA_OK) return rc;
@@ -202,7 +211,7 @@ static int bwd_input_common(const qlora_desc* desc, int M, const void* dY, const
         !aligned16(A) || !aligned16(B) || !aligned16(G_out) || !aligned16(workspace))
         return QLORA_ERR_ALIGNMENT;
     const Workspace w = carve(d, M);
-    if (workspace == nullptr || workspace_bytes < w.total) return QLORA_ERR_WORKSPACE;
+    if (workspace == nullptr || workspace_bytes < w.required) return QLORA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     float* G = G_out ? G_out : reinterpret_cast<float*>(static_cast<char*>(workspace) + w.p0_off);
     if (mask != nullptr && d.r > 0) {
@@ -225,7 +234,8 @@ static int bwd_input_common(const qlora_desc* desc, int M, const void* dY, const
         return launch_stream_gemm(d, M, true, dY, Q, scales, zeros, B, A, G, !fused, dX, st);
     }
     unsigned int* sync = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + w.sync_off);
-    if (umma_supported(d, M)) return launch_umma_gemm(d, M, true, dY, Q, scales, zeros, A, G, dX, st, B, sync);   // computes G
+    if (umma_supported(d, M)) return launch_umma_gemm(d, M, true, dY, Q, scales, zeros, A, G, dX, st, B, sync, static_cast<char*>(workspace) + w.split_off,
+                                workspace_bytes - w.split_off);   // computes G
     if (d.r > 0) {
         rc = launch_lora_down(M, d.N, d.r, false, dY, B, G, st);
         if (rc != QLORA_OK) return rc;
@@ -249,7 +259,7 @@ static int bwd_lora_common(const qlora_desc* desc, int M, const void* X, const u
         !aligned16(dA) || !aligned16(dB) || !aligned16(workspace))
         return QLORA_ERR_ALIGNMENT;
     const Workspace w = carve(d, M);
-    if (workspace == nullptr || workspace_bytes < w.total) return QLORA_ERR_WORKSPACE;
+    if (workspace == nullptr || workspace_bytes < w.required) return QLORA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     char* ws = static_cast<char*>(workspace);
     const float s = d.alpha / (float)d.r;

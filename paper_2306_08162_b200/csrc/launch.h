@@ -51,7 +51,13 @@ int launch_lora_masked_update(int M, int K, int r, float c, const float* G, cons
 bool umma_supported(const qlora_desc& d, int M);
 int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q,
                      const void* scales, const void* zeros, const void* L, float* P, void* Out,
-                     cudaStream_t st, const void* Ldown = nullptr, unsigned int* sync = nullptr);
+                     cudaStream_t st, const void* Ldown = nullptr, unsigned int* sync = nullptr, void* split_buf = nullptr,
+                     size_t split_bytes = 0);
+// Bytes of workspace (`split_buf`) with which the CTA-pair kernel splits the tiles of a partly filled last wave along the
+// contraction (two SM pairs per tile, exchanging halves of the result); 0 when it would not.  Needs `sync` as well.
+size_t umma_split_scratch_bytes(const qlora_desc& d, int M);
+// api.cu -- the workspace a layer call needs at least (qlora_workspace_bytes less the optional exchange area above)
+size_t required_workspace_bytes(const qlora_desc& d, int M);
 // stream_kernel.cu -- few tokens (M <= 16): cp.async-fed mma.sync kernels on raw codes, the contraction split over a
 // cluster.  Ldown / Lup: the adapter applied first / second (forward A, B; backward B, A).  P = H or G, fp32 [M, r]: read
 // when p_is_input, otherwise computed inside the kernel (ranks up to 16) and written out.

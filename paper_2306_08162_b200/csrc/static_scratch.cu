@@ -13,6 +13,7 @@
 
 #include <mutex>
 
+#include "launch.h"
 #include "qlora.h"
 
 namespace {
@@ -45,6 +46,7 @@ extern "C" int qlora_bwd_lora_static(const qlora_desc* desc, int M, const void* 
     size_t need = 0;
     const int rc = qlora_workspace_bytes(desc, M, &need);   // also validates the descriptor and M
     if (rc != QLORA_OK) return rc;
+    need = qlora::required_workspace_bytes(*desc, M);         // (the part of it that qlora_bwd_lora can use)
     if (need > (size_t)QLORA_STATIC_SCRATCH_BYTES) return QLORA_ERR_STATIC_LIMIT;
     void* scratch = nullptr;
     const int rs = static_scratch_for_current_device(&scratch);

@@ -41,6 +41,8 @@ namespace {
 constexpr int kThreads = 480;
 constexpr int kDequantWarp0 = 7, kGroupWarps = 4;   // two dequant groups of four warps
 constexpr int kEpiWarp0 = 3, kEpiWarps = 4;
+constexpr int kSyncWords = 64;                       // counters in the workspace: [0], [1] producer clusters, [2 ..] one per split tile
+constexpr size_t kSplitTileBytes = 2 * 2 * 8 * 8 * 128 * 16;   // exchange area of one split tile: 2 halves x 2 CTAs x 8 chunks x 4 KiB
 constexpr int kWRows = 128;          // weight rows (MMA M) per tile: n in forward, k in backward
 constexpr int kStepC = 64;           // contraction elements per pipeline stage
 constexpr int kWStageBytes = kWRows * kStepC * 2;   // 16 KiB of bf16 per stage
@@ -623,11 +625,11 @@ bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const
 __global__ void sync_zero_kernel(unsigned int* sync) {
     pdl_launch_dependents();
     pdl_wait();
-    if (threadIdx.x < 2) sync[threadIdx.x] = 0u;
+    if (threadIdx.x < kSyncWords) sync[threadIdx.x] = 0u;
 }
 
 int zero_sync_pair(unsigned int* sync, cudaStream_t st) {
-    return launch_pdl(sync_zero_kernel, dim3(1), dim3(32), 0, st, 1, sync) == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
+    return launch_pdl(sync_zero_kernel, dim3(1), dim3(kSyncWords), 0, st, 1, sync) == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
 }
 
 // Ldown != NULL: P = In * Ldown is still to be computed.  Where the tile clusters leave room for more clusters on the GPU
@@ -698,10 +700,30 @@ bool umma_supported(const qlora_desc& d, int M) {
     return true;
 }
 
+// Tiles of a partly filled last wave that are split two ways along the contraction (0: none).  Worth it when at most
+// half a wave is left over, so that every left-over tile finds two pairs, and the halves are still long enough.
+static int pair_split_tiles(int n_tiles, int steps, int pairs) {
+    if (n_tiles <= pairs || steps < 16) return 0;
+    const int rem = n_tiles % pairs;
+    if (rem == 0 || 2 * rem > pairs || 2 + rem > kSyncWords) return 0;
+    return rem;
+}
+
+// Workspace the CTA-pair kernel may use to exchange the halves of split tiles, forward or backward (0 when M is too small
+// for that kernel or nothing is split).
+size_t umma_split_scratch_bytes(const qlora_desc& d, int M) {
+    if (M <= 256 || !umma_supported(d, M)) return 0;
+    const int pairs = sm_count() / 2;
+    const int tok_tiles = (M + 4 * kPairTok - 1) / (4 * kPairTok);
+    const int rem_f = pair_split_tiles(tok_tiles * ((d.N + 2 * kPairW - 1) / (2 * kPairW)), d.K / kStepC, pairs);
+    const int rem_b = pair_split_tiles(tok_tiles * ((d.K + 2 * kPairW - 1) / (2 * kPairW)), d.N / kStepC, pairs);
+    return (size_t)(rem_f > rem_b ? rem_f : rem_b) * kSplitTileBytes;
+}
+
 // CTA-pair kernel: 512 tokens x 256 weight rows per pair of SMs (see prefer_pair_kernel for when it is used).
 static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
                             const void* zeros, const void* L, float* Pmat, void* Out, cudaStream_t st, const void* Ldown,
-                            unsigned int* sync) {
+                            unsigned int* sync, void* split_buf, size_t split_bytes) {
     PairParams p{};
     p.M = M; p.N = d.N; p.K = d.K; p.bits = d.bits; p.g = d.group_size; p.r = d.r; p.r_pad = (d.r + 15) / 16 * 16;
     p.C = transposed ? d.K : d.N;
@@ -745,28 +767,45 @@ static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const v
         return QLORA_ERR_CUDA;
 
     const int pairs = sm_count() / 2;
-    // P = In * Ldown still to be computed: on SM pairs the tiles leave idle when they can take all row blocks (they are
-    // then done well before the tiles' contractions are), else by a launch ahead of this one.  Both sum in the same order.
     p.n_prod = 0; p.T = T; p.sync = nullptr; p.wait_limit_us = kWaitLimitUs;
     p.In = (const __nv_bfloat16*)In; p.Ldown = (const __nv_bfloat16*)Ldown; p.Pout = Pmat;
     p.lds_stages = (int)((p.off_bar - LDS_BAR_BYTES) / LDS_STAGE_BYTES);
     if (p.lds_stages > 6) p.lds_stages = 6;
-    if (Ldown != nullptr && d.r > 0) {
-        const int n_blocks = (M + 15) / 16;
-        // pairs with less to do: no tile at all, or one tile fewer than the rest when the last wave is partly filled
-        const int idle = p.n_tiles < pairs ? pairs - p.n_tiles : (p.n_tiles % pairs ? pairs - p.n_tiles % pairs : 0);
+    // P = In * Ldown still to be computed (Ldown given): on SM pairs the tiles leave idle when those can take all row
+    // blocks (they are then done well before the tiles' contractions are), else by a launch ahead of this one.  Both sum
+    // in the same order.  producers(last) = how many pairs would do it when the last wave has `last` items (0: none can).
+    const bool want_p = Ldown != nullptr && d.r > 0;
+    const int n_blocks = (M + 15) / 16;
+    auto producers = [&](int last) {
+        // pairs with less to do: no tile at all, or one item fewer than the rest when the last wave is partly filled
+        const int idle = p.n_tiles < pairs ? pairs - p.n_tiles : (last ? pairs - last : 0);
         int n_prod = (n_blocks + 3) / 4;                     // four row blocks per producer CTA pair when there is room
         if (n_prod > idle) n_prod = idle;
-        const bool fits = d.r <= 16 && n_prod > 0 && n_prod * 2 * LDS_MAXB >= n_blocks && p.lds_stages >= LDS_MIN_STAGES;
-        if (fits && sync != nullptr) {
-            p.n_prod = n_prod;
-            p.sync = sync;
-            const int rc = zero_sync_pair(sync, st);
-            if (rc != QLORA_OK) return rc;
-        } else {
+        const bool fits = want_p && sync != nullptr && d.r <= 16 && n_prod > 0 && n_prod * 2 * LDS_MAXB >= n_blocks &&
+                          p.lds_stages >= LDS_MIN_STAGES;
+        return fits ? n_prod : 0;
+    };
+    // A partly filled last wave (more tiles than pairs, at most half a wave left over): each left-over tile goes to two
+    // pairs, half of the contraction each, which exchange halves of the result through the workspace -- unless that
+    // takes away the idle pairs that would otherwise have computed P beside the tiles (8192 tokens on 4096 x 4096: the
+    // down-projection launch it then needs costs what the split wins).
+    p.n_full = p.n_tiles; p.nsplit = 1; p.split_buf = nullptr;
+    const int rem = pair_split_tiles(p.n_tiles, p.steps, pairs);
+    if (rem > 0 && sync != nullptr && split_buf != nullptr && (size_t)rem * kSplitTileBytes <= split_bytes &&
+        !(want_p && producers(2 * rem) == 0 && producers(p.n_tiles % pairs) > 0)) {
+        p.n_full = p.n_tiles - rem; p.nsplit = 2; p.split_buf = static_cast<float4*>(split_buf);
+    }
+    if (want_p) {
+        p.n_prod = producers(p.nsplit > 1 ? 2 * rem : p.n_tiles % pairs);
+        if (p.n_prod == 0) {
             const int rc = launch_lora_down(M, T, d.r, !transposed, In, Ldown, Pmat, st);
             if (rc != QLORA_OK) return rc;
         }
+    }
+    if (p.n_prod > 0 || p.nsplit > 1) {                      // the counters in the workspace are in use: zero them in stream order
+        p.sync = sync;
+        const int rc = zero_sync_pair(sync, st);
+        if (rc != QLORA_OK) return rc;
     }
     const int grid = 2 * (p.n_tiles < pairs ? p.n_tiles + p.n_prod : pairs);
 #define QLORA_LAUNCH_PAIR(B)                                                                              \
@@ -805,8 +844,9 @@ static bool prefer_pair_kernel(const qlora_desc& d, int M, bool transposed) {
 
 int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
                      const void* zeros, const void* L, float* Pmat, void* Out, cudaStream_t st, const void* Ldown,
-                     unsigned int* sync) {
-    if (prefer_pair_kernel(d, M, transposed)) return launch_umma_pair(d, M, transposed, In, Q, scales, zeros, L, Pmat, Out, st, Ldown, sync);
+                     unsigned int* sync, void* split_buf, size_t split_bytes) {
+    if (prefer_pair_kernel(d, M, transposed))
+        return launch_umma_pair(d, M, transposed, In, Q, scales, zeros, L, Pmat, Out, st, Ldown, sync, split_buf, split_bytes);
     Params p{};
     p.M = M; p.N = d.N; p.K = d.K; p.bits = d.bits; p.g = d.group_size; p.r = d.r; p.r_pad = (d.r + 15) / 16 * 16;
     p.C = transposed ? d.K : d.N;

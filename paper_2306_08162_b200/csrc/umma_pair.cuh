@@ -24,6 +24,14 @@
 // once the tile's contraction is through.  The counter pair belongs to one launch at a time (the host hands out one
 // pair per workspace) and the last CTA to have seen the count zeroes it again.
 
+//
+// When the tiles make more than one wave and at most half a wave is left over (172 tiles on 74 pairs: 24), each left-over
+// tile is worked on by two pairs, one half of the contraction steps each, as the last thing both do.  Their epilogues
+// then trade halves of the fp32 result through the caller's workspace -- each writes the eight 32-column chunks it does
+// not finish, both count themselves in at the tile's counter and wait for the other (bounded), each adds the peer's
+// part to the chunks it keeps -- so the third wave costs about two thirds of a tile instead of a whole one.  Nothing can
+// wait in a circle: the split item is every worker's last, and all workers are resident (one CTA per SM).
+
 constexpr int kPairTok = 128;                          // token rows per CTA per accumulator
 constexpr int kPairW = 128;                            // weight rows per CTA (256 per pair tile)
 constexpr int kPairXSub = kPairTok * kStepC * 2;       // 16 KiB: one 128-token sub-tile of a stage
@@ -33,6 +41,10 @@ struct PairParams {
     int M, N, K, bits, g, r, r_pad;
     int C;                       // output columns (N forward, K backward)
     int n_tok_tiles, n_tiles, steps;
+    // Last wave split along the contraction: tiles [n_full, n_tiles) are each worked on by two SM pairs (nsplit == 2), one
+    // half of the steps each; nsplit == 1: n_full == n_tiles, nothing is split.
+    int n_full, nsplit;
+    float4* split_buf;           // fp32 exchange area of the split tiles (workspace)
     int S, P;
     int packed_cols, packed_rows, scale_rows;
     uint32_t words_bytes, scale_bytes, packed_slot_bytes;
@@ -114,6 +126,24 @@ __device__ __forceinline__ uint32_t instr_desc_pair(uint32_t n_mma, uint32_t a_m
            ((256u >> 4) << 24);
 }
 
+// What worker pair `w` of `W` does, in order: the whole tiles w, w + W, ... below n_full, then (last, if at all) its half
+// of a split tile.  Workers 2i and 2i + 1 share split tile n_full + i.
+struct PairItem { int tile, s0, s1, part, nparts; };
+__device__ __forceinline__ int pair_item_count(const PairParams& p, int w, int W) {
+    const int full = w < p.n_full ? (p.n_full - w + W - 1) / W : 0;
+    return full + ((p.nsplit > 1 && w < (p.n_tiles - p.n_full) * p.nsplit) ? 1 : 0);
+}
+__device__ __forceinline__ PairItem pair_item(const PairParams& p, int w, int W, int it) {
+    PairItem r;
+    const int full = w < p.n_full ? (p.n_full - w + W - 1) / W : 0;
+    if (it < full) { r.tile = w + it * W; r.s0 = 0; r.s1 = p.steps; r.part = 0; r.nparts = 1; }
+    else {
+        r.tile = p.n_full + w / p.nsplit; r.part = w % p.nsplit; r.nparts = p.nsplit;
+        r.s0 = p.steps * r.part / p.nsplit; r.s1 = p.steps * (r.part + 1) / p.nsplit;
+    }
+    return r;
+}
+
 template <int BITS, bool TRANSPOSED>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_q,
@@ -135,7 +165,8 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     // i.e. the workers with the fewest tiles -- none at all when the tiles do not fill a wave.
     const int tile_stride = (int)(gridDim.x >> 1);
     const bool is_producer = (int)(blockIdx.x >> 1) < p.n_prod;
-    const int first_tile = is_producer ? tile_stride - 1 - (int)(blockIdx.x >> 1) : (int)(blockIdx.x >> 1) - p.n_prod;
+    const int first_tile = is_producer ? tile_stride - 1 - (int)(blockIdx.x >> 1) : (int)(blockIdx.x >> 1) - p.n_prod;   // = the worker index
+    const int n_items = pair_item_count(p, first_tile, tile_stride);
 
     // barriers (same offsets in both CTAs)
     // One "stage full" barrier per slot collects both operand streams -- the TMA bytes of both CTAs' activation sub-tiles
@@ -195,9 +226,11 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             pdl_wait();
             Ring ring;
             const uint32_t leader_full_x = map_to_cta(bar_full_x, 0);
-            for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride) {
+            for (int it = 0; it < n_items; ++it) {
+                const PairItem item = pair_item(p, first_tile, tile_stride, it);
+                const int tile = item.tile;
                 const int m0 = (tile % p.n_tok_tiles) * (4 * kPairTok) + (int)cta * kPairTok;
-                for (int step = 0; step < p.steps; ++step) {
+                for (int step = item.s0; step < item.s1; ++step) {
                     if (!mbar_wait(bar_empty + 8 * ring.slot, ring.phase ^ 1u, abort_flag)) goto done;
                     if (cta == 0) mbar_expect_tx(bar_full_x + 8 * ring.slot, 2 * kPairXStage);   // both CTAs' bytes
                     const uint32_t dst = smem0 + p.off_x + ring.slot * kPairXStage;
@@ -213,10 +246,12 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         if (lane == 0) {
             Ring ring;
             const uint32_t tx_bytes = p.words_bytes + 2 * p.scale_bytes;
-            for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride) {
+            for (int it = 0; it < n_items; ++it) {
+                const PairItem item = pair_item(p, first_tile, tile_stride, it);
+                const int tile = item.tile;
                 const int w0 = (tile / p.n_tok_tiles) * (2 * kPairW) + (int)cta * kPairW;
                 const int g_row = TRANSPOSED ? w0 / p.g : 0;
-                for (int step = 0; step < p.steps; ++step) {
+                for (int step = item.s0; step < item.s1; ++step) {
                     if (!mbar_wait(bar_empty_p + 8 * ring.slot, ring.phase ^ 1u, abort_flag)) goto done;
                     const uint32_t dst = smem0 + p.off_p + ring.slot * p.packed_slot_bytes;
                     const uint32_t bar = bar_full_p + 8 * ring.slot;
@@ -249,11 +284,12 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             constexpr uint32_t b_k16 = TRANSPOSED ? (2048u >> 4) : (32u >> 4);
             Ring ring;
             uint32_t tile_it = 0;
-            for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride, ++tile_it) {
+            for (int it = 0; it < n_items; ++it, ++tile_it) {
+                const PairItem item = pair_item(p, first_tile, tile_stride, it);
                 if (!mbar_wait_cluster(bar_acc_empty, (tile_it & 1u) ^ 1u, abort_flag)) goto done;
                 tc_fence_after();
                 uint32_t acc = 0;
-                for (int step = 0; step < p.steps; ++step) {
+                for (int step = item.s0; step < item.s1; ++step) {
                     if (!mbar_wait_cluster(bar_full_x + 8 * ring.slot, ring.phase, abort_flag)) goto done;
                     tc_fence_after();
                     const uint64_t a_desc = a_desc0 + ring.slot * (uint32_t)(kPairXStage >> 4);
@@ -268,7 +304,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                     tc_commit_pair(bar_empty + 8 * ring.slot);
                     ring.advance(S);
                 }
-                if (p.r > 0) {
+                if (p.r > 0 && item.part == 0) {       // (the LoRA update goes into part 0's sum only; a split item is a worker's last)
                     if (!mbar_wait_cluster(bar_lora_full, tile_it & 1u, abort_flag)) goto done;
                     tc_fence_after();
                     for (int a = 0; a < 2; ++a)
@@ -291,7 +327,9 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         const uint32_t leader_lora_full = map_to_cta(bar_lora_full, 0);
         pdl_wait();
         uint32_t tile_it = 0;
-        for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride, ++tile_it) {
+        for (int it = 0; it < n_items; ++it, ++tile_it) {
+            const PairItem item = pair_item(p, first_tile, tile_stride, it);
+            const int tile = item.tile;
             const int wt = tile / p.n_tok_tiles, tt = tile % p.n_tok_tiles;
             const int w0 = wt * (2 * kPairW);                          // first weight row (output column) of the pair tile
             const int m0 = tt * (4 * kPairTok) + (int)cta * kPairTok;  // this CTA's first token row of accumulator 0
@@ -308,7 +346,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                 asm volatile("bar.sync 2, %0;" ::"r"(kEpiWarps * 32) : "memory");
                 if (*abort_flag) break;
             }
-            if (p.r > 0) {
+            if (p.r > 0 && item.part == 0) {
                 // (the previous tile's LoRA MMA has completed: its accumulator-full barrier was observed below)
                 uint8_t* ll = smem_gen + p.off_lora_l;
                 uint8_t* lp = smem_gen + p.off_lora_p;
@@ -386,7 +424,75 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                         *reinterpret_cast<uint4*>(p.Out + (size_t)m * p.C + w0 + cb) = val;
                 }
             };
-            {
+            if (item.nparts > 1) {
+                // A split tile: this pair holds the sum over its half of the contraction.  The two pairs exchange halves of
+                // the tile through the workspace: each gives away the eight 32-column chunks it does not finish (fp32,
+                // laid out so that a warp's stores and the peer's loads are contiguous), counts itself in at the tile's
+                // counter, waits for all four CTAs, then adds the peer's part to the chunks it keeps and stores them.
+                // (a + b is the same in either order, so both halves of the tile see one summation order.)
+                const int slot = tile - p.n_full;
+                float4* mine = p.split_buf + (size_t)((slot * 2 + item.part) * 2 + (int)cta) * (8 * 8 * 128);
+                const float4* peer = p.split_buf + (size_t)((slot * 2 + (1 - item.part)) * 2 + (int)cta) * (8 * 8 * 128);
+                auto chunk_addr = [&](int idx) { return taddr + (uint32_t)((idx >> 3) * kAccStride + (idx & 7) * 32); };
+                auto give = [&](const uint32_t (&v)[32], int k) {
+#pragma unroll
+                    for (int j4 = 0; j4 < 8; ++j4)
+                        mine[(k * 8 + j4) * 128 + et] = make_float4(__uint_as_float(v[4 * j4]), __uint_as_float(v[4 * j4 + 1]),
+                                                                    __uint_as_float(v[4 * j4 + 2]), __uint_as_float(v[4 * j4 + 3]));
+                };
+                {   // the chunks given away: the tensor-memory load of the next one is in flight while this one is stored
+                    uint32_t va[32], vb[32];
+                    tc_ld32(chunk_addr(1 - item.part), va);
+#pragma unroll 1
+                    for (int k = 0; k < 8; k += 2) {
+                        tc_wait_ld();
+                        tc_ld32(chunk_addr(2 * (k + 1) + (1 - item.part)), vb);
+                        give(va, k);
+                        tc_wait_ld();
+                        if (k + 2 < 8) tc_ld32(chunk_addr(2 * (k + 2) + (1 - item.part)), va);
+                        give(vb, k + 1);
+                    }
+                }
+                __threadfence();
+                asm volatile("bar.sync 2, %0;" ::"r"(kEpiWarps * 32) : "memory");
+                if (et == 0) {
+                    atomicAdd(&p.sync[2 + slot], 1u);
+                    wait_counter(&p.sync[2 + slot], 4u, abort_flag);
+                }
+                asm volatile("bar.sync 2, %0;" ::"r"(kEpiWarps * 32) : "memory");
+                if (*abort_flag) break;
+                {   // the chunks kept: the peer's part of the next one is requested before this one is added and stored
+                    uint32_t va[32];
+                    float4 pa[8], pb[8];
+                    auto take = [&](float4 (&pv)[8], int k) {
+#pragma unroll
+                        for (int j4 = 0; j4 < 8; ++j4) pv[j4] = __ldcg(peer + (k * 8 + j4) * 128 + et);
+                    };
+                    auto add = [&](uint32_t (&v)[32], const float4 (&pv)[8]) {
+#pragma unroll
+                        for (int j4 = 0; j4 < 8; ++j4) {
+                            v[4 * j4] = __float_as_uint(__uint_as_float(v[4 * j4]) + pv[j4].x);
+                            v[4 * j4 + 1] = __float_as_uint(__uint_as_float(v[4 * j4 + 1]) + pv[j4].y);
+                            v[4 * j4 + 2] = __float_as_uint(__uint_as_float(v[4 * j4 + 2]) + pv[j4].z);
+                            v[4 * j4 + 3] = __float_as_uint(__uint_as_float(v[4 * j4 + 3]) + pv[j4].w);
+                        }
+                    };
+                    take(pa, 0);
+#pragma unroll 1
+                    for (int k = 0; k < 8; k += 2) {
+                        tc_ld32(chunk_addr(2 * k + item.part), va);
+                        take(pb, k + 1);
+                        tc_wait_ld();
+                        add(va, pa);
+                        store_chunk(va, 2 * k + item.part);
+                        tc_ld32(chunk_addr(2 * (k + 1) + item.part), va);
+                        if (k + 2 < 8) take(pa, k + 2);
+                        tc_wait_ld();
+                        add(va, pb);
+                        store_chunk(va, 2 * (k + 1) + item.part);
+                    }
+                }
+            } else {
                 uint32_t va[32], vb[32];
                 tc_ld32(taddr, va);
 #pragma unroll 1
@@ -422,8 +528,11 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         }
         const uint32_t pcols = (uint32_t)p.packed_cols;
         const uint32_t leader_full_w = map_to_cta(bar_full_w, 0);
-        const int my_tiles = first_tile < p.n_tiles ? (p.n_tiles - first_tile + tile_stride - 1) / tile_stride : 0;
-        const int total = my_tiles * p.steps;
+        int total = 0;                                           // this worker's stages, whole tiles and split item alike
+        for (int it = 0; it < n_items; ++it) {
+            const PairItem item = pair_item(p, first_tile, tile_stride, it);
+            total += item.s1 - item.s0;
+        }
         Ring ring_w, ring_p;
         if (group == 1) { ring_w.advance(S); ring_p.advance(P); }
         for (int it = group; it < total; it += 2) {

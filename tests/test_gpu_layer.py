@@ -361,3 +361,17 @@ def test_empty_batch_is_a_no_op():
     gl = GpuLayer(layer)
     out = gl.run(X=gl.X[:0], dY=gl.dY[:0], check_canaries=True)
     assert float(out["dA"].abs().max()) == 0.0 and float(out["dB"].abs().max()) == 0.0
+
+
+@pytest.mark.parametrize("K,N,M,bits,g,r", [(1024, 6656, 1536, 4, 128, 8), (6656, 1024, 1536, 2, 64, 16),
+                                            (1024, 6656, 1400, 3, 128, 8), (1024, 6656, 1536, 8, 128, 0)])
+def test_last_wave_split_along_the_contraction(K, N, M, bits, g, r):
+    """78 tiles of 512 tokens x 256 weight rows on 74 SM pairs: the four left-over tiles are each shared by two pairs,
+    half of the contraction each, which exchange halves of the result through the workspace (forward for N = 6656,
+    backward for K = 6656).  Parity on sampled rows of every token tile, and the same bits on a second run."""
+    layer = qi.random_codes_layer(K=K, N=N, bits=bits, group_size=g, r=r, alpha=16.0, M=M, seed=K // 64 + bits)
+    rows = sorted(set(sample_rows(M, n=60, seed=3)) | {511, 512, 1023, 1024})
+    _, out, gl = check_layer(layer, rows=rows)
+    again = gl.run()
+    for key in ("Y", "dX"):
+        assert torch.equal(out[key].view(torch.int16), again[key].view(torch.int16)), key
