@@ -174,7 +174,7 @@ static GradPlan lora_grad_plan(int M, int K, int N) {
     if (slices > LG_MAX_SLICES) slices = LG_MAX_SLICES;
     if (slices < 1) slices = 1;
     int rows = (M + slices - 1) / slices;
-    rows = (rows + 15) / 16 * 16;                                // whole 16-row MMA steps; (rows + 8) / 2 = 4 x odd keeps the staged P^T conflict-free
+    rows = (rows + 63) / 64 * 64;                                // whole 16-row MMA steps; keeps the staged P^T conflict-free
     if (rows < 64) rows = 64;
     if (rows > 1024) rows = 1024;                                // bounds the staged P^T (64 ranks x 1032 x 2 B = 129 KiB at most)
     GradPlan g;
@@ -232,15 +232,29 @@ lora_grad_partial_kernel(int M, int r, int rows_per_slice, GradSide side0, GradS
     const int g = lane >> 2, q = lane & 3;
     const int slice = CL > 0 ? (int)blockIdx.x % CL : (int)blockIdx.y;
     const int m_begin = slice * rows_per_slice;
-    const int stride = rows_per_slice + 8;                     // in bf16: stride / 2 = 4 x odd -> conflict-free fragment loads
+    const int stride = rows_per_slice + 8;                     // in bf16: (stride / 2) % 32 == 4 -> conflict-free fragment loads
     constexpr int RP = RT * 16;
+    // stage P^T (bf16) of this slice: rows beyond M and ranks beyond r are zero
+    for (int e = threadIdx.x; e < rows_per_slice * RP; e += LG_WARPS * 32) {
+        const int ml = e / RP, j = e % RP;
+        const int m = m_begin + ml;
+        const float v = (m < M && j < r) ? __ldg(sd.P + (size_t)m * r + j) : 0.f;
+        Pt[j * stride + ml] = __float2bfloat16_rn(v);
+    }
+    __syncthreads();
+
     const int c0 = cb + warp * 32 + q * 8;                     // this lane loads columns c0 .. c0 + 7
     const bool live = c0 < C;                                  // C is a multiple of 8
     const __nv_bfloat16* src = sd.In + c0;
+    float acc[RT][4][4];
+#pragma unroll
+    for (int rt = 0; rt < RT; ++rt)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[rt][c][0] = acc[rt][c][1] = acc[rt][c][2] = acc[rt][c][3] = 0.f;
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
     const int m_stop = min(M, m_begin + rows_per_slice);
-    uint4 x0[LG_UNROLL], x1[LG_UNROLL];
-    auto load_round = [&](int mm) {
+    for (int mm = m_begin; mm < m_stop; mm += 16 * LG_UNROLL) {
+        uint4 x0[LG_UNROLL], x1[LG_UNROLL];
 #pragma unroll
         for (int u = 0; u < LG_UNROLL; ++u) {
             const int ma = mm + 16 * u + g, mb = ma + 8;
@@ -251,35 +265,6 @@ lora_grad_partial_kernel(int M, int r, int rows_per_slice, GradSide side0, GradS
                 if (live && mb < m_stop) x1[u] = mask_eight(x1[u], __ldg(reinterpret_cast<const uint2*>(sd.mask + (size_t)mb * C + c0)));
             }
         }
-    };
-    load_round(m_begin);                                       // the first round is in flight while P^T is staged
-    // stage P^T (bf16) of this slice, four ranks of a row per load (all loads of a thread independent): rows beyond M and
-    // ranks beyond r are zero
-    {
-        const int r4 = r >> 2;                                 // r is a multiple of 8
-        const int n_ld = rows_per_slice * r4;
-#pragma unroll 4
-        for (int e = threadIdx.x; e < n_ld; e += LG_WARPS * 32) {
-            const int ml = e / r4, j = (e - ml * r4) * 4;
-            const int m = m_begin + ml;
-            const float4 v = m < M ? __ldg(reinterpret_cast<const float4*>(sd.P + (size_t)m * r + j)) : make_float4(0.f, 0.f, 0.f, 0.f);
-            Pt[j * stride + ml] = __float2bfloat16_rn(v.x);
-            Pt[(j + 1) * stride + ml] = __float2bfloat16_rn(v.y);
-            Pt[(j + 2) * stride + ml] = __float2bfloat16_rn(v.z);
-            Pt[(j + 3) * stride + ml] = __float2bfloat16_rn(v.w);
-        }
-        for (int e = threadIdx.x; e < (RP - r) * rows_per_slice; e += LG_WARPS * 32)
-            Pt[(r + e / rows_per_slice) * stride + e % rows_per_slice] = __float2bfloat16_rn(0.f);
-    }
-    __syncthreads();
-
-    float acc[RT][4][4];
-#pragma unroll
-    for (int rt = 0; rt < RT; ++rt)
-#pragma unroll
-        for (int c = 0; c < 4; ++c) acc[rt][c][0] = acc[rt][c][1] = acc[rt][c][2] = acc[rt][c][3] = 0.f;
-    for (int mm = m_begin; mm < m_stop; mm += 16 * LG_UNROLL) {
-        if (mm != m_begin) load_round(mm);
 #pragma unroll
         for (int u = 0; u < LG_UNROLL; ++u) {
             const int ml = mm + 16 * u - m_begin;              // warp-uniform
@@ -369,13 +354,6 @@ __global__ void lora_grad_reduce_kernel(int r, int slices, int accumulate, GradS
     const size_t step = (size_t)sd.C * r;
     float v = 0.f;
     int sl = 0;
-    for (; sl + 8 <= slices; sl += 8) {               // eight independent loads in flight, added in slice order
-        float pp[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) pp[i] = sd.partial[(size_t)(sl + i) * step + e];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) v += pp[i];
-    }
     for (; sl + 4 <= slices; sl += 4) {               // four independent loads in flight, added in slice order
         const float p0 = sd.partial[(size_t)sl * step + e], p1 = sd.partial[(size_t)(sl + 1) * step + e];
         const float p2 = sd.partial[(size_t)(sl + 2) * step + e], p3 = sd.partial[(size_t)(sl + 3) * step + e];
