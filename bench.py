@@ -3,7 +3,7 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME] [--no-graph]
 
-One "step" = qlora_fwd + qlora_bwd_input + qlora_bwd_lora on one projection (K = N = 4096, INT4, group 128,
+One "step" = qlora_fwd + qlora_bwd_input_db (dX, G and dB) + qlora_bwd_lora (dA) on one projection (K = N = 4096, INT4, group 128,
 LoRA r = 8, alpha = 16, M = 2048 bf16 tokens; synthetic seeded inputs).  Consecutive steps rotate through several
 independent copies of the layer (own weights, activations and outputs) whose combined footprint exceeds the L2
 cache, so no step finds its operands cached by the previous one.  Prints ONE JSON line (rank 0).
@@ -406,16 +406,33 @@ def run_ours(args):
     host_out = dict(Y=torch.empty((M, N), dtype=torch.int16).pin_memory(), dX=torch.empty((M, K), dtype=torch.int16).pin_memory(),
                     dA=torch.empty((r, K), dtype=torch.float32).pin_memory(), dB=torch.empty((N, r), dtype=torch.float32).pin_memory())
 
+    # With many tokens dB rides on the backward call (qlora_bwd_input_db: dY is read once) and the gradient call computes
+    # dA alone; with few tokens the three plain calls.  Either way a step produces Y, H, dX, G, dA and dB.
+    fused_db = M > 256 and r > 0
+    bwd_name = "qlora_bwd_input_db" if fused_db else "qlora_bwd_input"
+
+    def bwd_input_call(L):
+        if fused_db:
+            ql.qlora_bwd_input_db(d, M, L["dY"], L["Q"], L["scales"], L["zeros"], L["A"], L["B"], L["H"], L["dX"], L["G"], L["dB"], 0, ws)
+        else:
+            ql.qlora_bwd_input(d, M, L["dY"], L["Q"], L["scales"], L["zeros"], L["A"], L["B"], L["dX"], L["G"], ws)
+
+    def bwd_lora_call(L):
+        if fused_db:
+            ql.qlora_bwd_lora(d, M, L["X"], None, L["A"], L["B"], None, L["G"], L["dA"], None, 0, ws)
+        else:
+            ql.qlora_bwd_lora(d, M, L["X"], L["dY"], L["A"], L["B"], L["H"], L["G"], L["dA"], L["dB"], 0, ws)
+
     def step(L, events=None):
         if events is not None:
             events[0].record()
         ql.qlora_fwd(d, M, L["X"], L["Q"], L["scales"], L["zeros"], L["A"], L["B"], L["Y"], L["H"], ws)
         if events is not None:
             events[1].record()
-        ql.qlora_bwd_input(d, M, L["dY"], L["Q"], L["scales"], L["zeros"], L["A"], L["B"], L["dX"], L["G"], ws)
+        bwd_input_call(L)
         if events is not None:
             events[2].record()
-        ql.qlora_bwd_lora(d, M, L["X"], L["dY"], L["A"], L["B"], L["H"], L["G"], L["dA"], L["dB"], 0, ws)
+        bwd_lora_call(L)
         if events is not None:
             events[3].record()
 
@@ -460,8 +477,7 @@ def run_ours(args):
         del gt
         call_ms = []
         for call in (lambda L: ql.qlora_fwd(d, M, L["X"], L["Q"], L["scales"], L["zeros"], L["A"], L["B"], L["Y"], L["H"], ws),
-                     lambda L: ql.qlora_bwd_input(d, M, L["dY"], L["Q"], L["scales"], L["zeros"], L["A"], L["B"], L["dX"], L["G"], ws),
-                     lambda L: ql.qlora_bwd_lora(d, M, L["X"], L["dY"], L["A"], L["B"], L["H"], L["G"], L["dA"], L["dB"], 0, ws)):
+                     bwd_input_call, bwd_lora_call):
             gtc = GraphTimer(steps_body(call), barrier)
             call_ms.append(gtc.region(20.0)[0] / args.steps)
             del gtc
@@ -534,7 +550,7 @@ def run_ours(args):
         peaks = measured_peaks()
         # dominant kernel: the dequant-GEMM of the forward or backward-input call, whichever takes longer
         dom = 0 if call_ms[0] >= call_ms[1] else 1
-        dom_name = ("qlora_fwd", "qlora_bwd_input")[dom]
+        dom_name = ("qlora_fwd", bwd_name)[dom]
         long_run = False
         if M > 64:    # a dense contraction: tensor roofline
             bound, r_unit = "tensor", "TFLOP/s"
@@ -560,7 +576,8 @@ def run_ours(args):
                        "eager_ms_per_step": eager_ms_per_step,
                        "l2": f"inputs larger than L2: steps rotate through {ROTATION} independent layer copies "
                              f"(~{ROTATION * layer_bytes(w) // 2**20} MiB)",
-                       "calls_ms": {"qlora_fwd": call_ms[0], "qlora_bwd_input": call_ms[1], "qlora_bwd_lora": call_ms[2]}},
+                       "step_calls": ["qlora_fwd", bwd_name, "qlora_bwd_lora" + (" (dA only)" if fused_db else "")],
+                       "calls_ms": {"qlora_fwd": call_ms[0], bwd_name: call_ms[1], "qlora_bwd_lora": call_ms[2]}},
             "roofline": {"bound": bound, "kernel": dom_name, "achieved": achieved, "peak": peak, "unit": r_unit,
                          "frac": achieved / peak,
                          "frac_sustained": ((achieved * total_ms / sus_ms) / peaks["bf16_sustained"]
@@ -591,7 +608,7 @@ def run_ours(args):
 def run_chain(args):
     """--workload config5: the projection set of configs[4] -- 32 decoder blocks x (q, k, v, o 4096x4096; gate, up
     4096->11008; down 11008->4096), INT2 group 64, LoRA r = 8 on all 224 projections, M = 4096 tokens (8 x 512) -- run as
-    a chain: forward through every projection, then backward (qlora_bwd_input + qlora_bwd_lora) in reverse order.  One step
+    a chain: forward through every projection, then backward (qlora_bwd_input_db + qlora_bwd_lora for dA) in reverse order.  One step
     streams 2 GB of packed weights and 12 GB of saved activations, far more than the L2.  The codes are random (drawn on
     the device: 6.5 G weights), the scales sized so that the activations keep their magnitude along the chain."""
     import torch
@@ -641,8 +658,8 @@ def run_chain(args):
                 dY = {"down": grad, "up": seed_grad[11008], "v": seed_grad[4096], "k": seed_grad[4096]}.get(name)
                 if dY is None:
                     dY = row[{"gate": "down", "o": "gate", "q": "o"}[name]]["dX"]
-                ql.qlora_bwd_input(P["d"], M, dY, P["Q"], P["s"], P["z"], P["A"], P["B"], P["dX"], P["G"], ws)
-                ql.qlora_bwd_lora(P["d"], M, P["X"], dY, P["A"], P["B"], P["H"], P["G"], P["dA"], P["dB"], 0, ws)
+                ql.qlora_bwd_input_db(P["d"], M, dY, P["Q"], P["s"], P["z"], P["A"], P["B"], P["H"], P["dX"], P["G"], P["dB"], 0, ws)
+                ql.qlora_bwd_lora(P["d"], M, P["X"], None, P["A"], P["B"], None, P["G"], P["dA"], None, 0, ws)
             grad = row["q"]["dX"]
 
     def barrier():

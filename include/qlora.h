@@ -86,10 +86,12 @@ typedef struct {
 /* Bytes of scratch the three layer calls may need for M tokens (the maximum over the calls, so one buffer
  * serves all).  The paper has no counterpart: it is how a library that allocates nothing gets its scratch.  `out` is a
  * host pointer.  The scratch holds H / G when the caller does not keep them, the partial sums of the LoRA gradients, a
- * few counters, and -- last, and optional -- the area through which two SM pairs exchange the halves of an output tile
- * whose contraction they share (many tokens, last wave partly filled: up to 12 MiB on LLaMA-7B MLP shapes).  A call
- * given less than that last part still works, without the split.  Contents are undefined between calls.  The figure is
- * computed for the current device (its SM count decides what is split). */
+ * few counters, and -- last, and optional -- two areas the tensor-core kernels use when the workspace reaches that far:
+ * the one through which two SM pairs exchange the halves of an output tile whose contraction they share (many tokens,
+ * last wave partly filled: up to 12 MiB on LLaMA-7B MLP shapes), and the parts of dB of qlora_bwd_input_db (8 MiB at
+ * N = 4096, r = 8, 2048 tokens).  A call given less still works, without the split and with dB from the gradient
+ * kernels.  Contents are undefined between calls.  The figure is computed for the current device (its SM count decides
+ * what is split and how many SMs can take dB on). */
 int qlora_workspace_bytes(const qlora_desc* desc, int M, size_t* out);
 
 /* Forward (Figure 1, forward path):  Y = X W^T + s (X A^T) B^T,  bf16 output, fp32 accumulation.
@@ -105,11 +107,24 @@ int qlora_bwd_input(const qlora_desc* desc, int M, const void* dY, const int32_t
                     const void* zeros, const void* A, const void* B, void* dX, float* G_out, void* workspace,
                     size_t workspace_bytes, void* cuda_stream);
 
+/* qlora_bwd_input that also produces dB = s dY^T H (Figure 1: the backward arrow into the second LoRA block leaves the
+ * same dY that flows back through the frozen weight), so that dY is read once for both.  H: fp32 [M, r], the forward's
+ * H_out (required when r > 0); dB: fp32 [N, r]; accumulate as in qlora_bwd_lora.  With many tokens and r <= 8 the SMs
+ * that stream dY to form G inside the backward kernel form dB on the same pass (each leaves a part in the workspace,
+ * they add the parts in a fixed order before they go on); for other shapes dB comes from the gradient kernels after
+ * the backward kernel.  Either way dB is complete when the call's work is, and the same inputs give the same bits on a
+ * given device; the two routes group the sum over tokens differently, so their bits differ from each other (and from
+ * qlora_bwd_lora's) in the last places.  Follow it with qlora_bwd_lora(..., dB = NULL) for dA. */
+int qlora_bwd_input_db(const qlora_desc* desc, int M, const void* dY, const int32_t* Q, const void* scales,
+                       const void* zeros, const void* A, const void* B, const float* H, void* dX, float* G_out, float* dB,
+                       int accumulate, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Gradients of the trainable pair (Section 3.1: only theta_l is updated; Figure 1, arrows into the LoRA blocks):
  *   dA = s (dY B)^T X  fp32 [r, K],     dB = s dY^T (X A^T)  fp32 [N, r].
  * H, G: fp32 [M, r] saved by the calls above, or NULL to recompute them here (the case under gradient
  * checkpointing, Section 4.1).  accumulate = 0 overwrites dA / dB, 1 adds to their current contents
- * (micro-batch accumulation, Appendix B). */
+ * (micro-batch accumulation, Appendix B).  dB may be NULL (it came from qlora_bwd_input_db): only dA is computed, and
+ * dY may then be NULL too when G is given. */
 int qlora_bwd_lora(const qlora_desc* desc, int M, const void* X, const void* dY, const void* A, const void* B,
                    const float* H, const float* G, float* dA, float* dB, int accumulate, void* workspace,
                    size_t workspace_bytes, void* cuda_stream);

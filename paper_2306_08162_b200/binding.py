@@ -47,6 +47,7 @@ def library() -> ctypes.CDLL:
     lib.qlora_fwd.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.qlora_bwd_input.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.qlora_bwd_lora.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
+    lib.qlora_bwd_input_db.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
     f32 = ctypes.c_float
     lib.qlora_fwd_dropout.argtypes = [dp, i32, vp, vp, f32, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.qlora_bwd_input_dropout.argtypes = [dp, i32, vp, vp, f32, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -60,7 +61,7 @@ def library() -> ctypes.CDLL:
     lib.qlora_lrec_loss.argtypes = [i32, i32, vp, vp, vp, ctypes.c_float, ctypes.c_float, ctypes.c_float, vp, vp, vp]
     lib.qlora_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint), i32]
     lib.qlora_selftest_bounded_wait.argtypes = [i32, vp]
-    for name in ("qlora_workspace_bytes", "qlora_fwd", "qlora_bwd_input", "qlora_bwd_lora", "qlora_bwd_lora_static", "qlora_fwd_dropout", "qlora_bwd_input_dropout",
+    for name in ("qlora_workspace_bytes", "qlora_fwd", "qlora_bwd_input", "qlora_bwd_input_db", "qlora_bwd_lora", "qlora_bwd_lora_static", "qlora_fwd_dropout", "qlora_bwd_input_dropout",
                  "qlora_bwd_lora_dropout", "qlora_pack",
                  "qlora_unpack", "qlora_dequant", "qlora_quantize_rtn", "qlora_gather_columns", "qlora_lrec_loss", "qlora_device_status", "qlora_selftest_bounded_wait"):
         getattr(lib, name).restype = i32
@@ -118,6 +119,13 @@ def qlora_bwd_input(d, M, dY, Q, scales, zeros, A, B, dX, G_out, workspace, stre
     _check(library().qlora_bwd_input(ctypes.byref(d), int(M), _ptr(dY), _ptr(Q), _ptr(scales), _ptr(zeros), _ptr(A),
                                      _ptr(B), _ptr(dX), _ptr(G_out), _ptr(workspace), wb, _stream(stream)),
            "qlora_bwd_input")
+
+
+def qlora_bwd_input_db(d, M, dY, Q, scales, zeros, A, B, H, dX, G_out, dB, accumulate, workspace, stream=None, workspace_bytes=None):
+    wb = _nbytes(workspace) if workspace_bytes is None else int(workspace_bytes)
+    _check(library().qlora_bwd_input_db(ctypes.byref(d), int(M), _ptr(dY), _ptr(Q), _ptr(scales), _ptr(zeros), _ptr(A),
+                                        _ptr(B), _ptr(H), _ptr(dX), _ptr(G_out), _ptr(dB), int(accumulate), _ptr(workspace), wb,
+                                        _stream(stream)), "qlora_bwd_input_db")
 
 
 def qlora_bwd_lora(d, M, X, dY, A, B, H, G, dA, dB, accumulate, workspace, stream=None, workspace_bytes=None):

@@ -35,9 +35,10 @@ int check_desc(const qlora_desc* d, bool need_lora) {
 }
 
 struct Workspace {
-    size_t p0_off, p1_off, grad_off, sync_off, split_off;
+    size_t p0_off, p1_off, grad_off, sync_off, split_off, db_off;
     size_t required;   // what a call cannot do without
-    size_t total;      // ... plus the exchange area of split tiles (used when it is there)
+    size_t total;      // ... plus the optional areas, each used when the workspace reaches that far: the exchange area
+                       // of split tiles, then the producers' parts of dB (qlora_bwd_input_db)
 };
 
 Workspace carve(const qlora_desc& d, int M) {
@@ -49,7 +50,8 @@ Workspace carve(const qlora_desc& d, int M) {
     w.sync_off = w.grad_off + align_up(lora_grad_scratch_bytes(M, d.K, d.N, d.r), 256);
     w.split_off = w.sync_off + 256;      // the counters of the tensor-core kernels: producer clusters, split tiles
     w.required = w.split_off;
-    w.total = w.split_off + umma_split_scratch_bytes(d, M);
+    w.db_off = w.split_off + align_up(umma_split_scratch_bytes(d, M), 256);
+    w.total = w.db_off + umma_db_part_bytes(d, M);
     return w;
 }
 
@@ -199,7 +201,7 @@ static int fwd_common(const qlora_desc* desc, int M, const void* X, const uint8_
 // kernels then run without the branch (rank 0) and an elementwise pass adds the masked term.
 static int bwd_input_common(const qlora_desc* desc, int M, const void* dY, const uint8_t* mask, float keep_scale,
                             const int32_t* Q, const void* scales, const void* zeros, const void* A, const void* B, void* dX,
-                            float* G_out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+                            float* G_out, void* workspace, size_t workspace_bytes, void* cuda_stream, DbFuse* db = nullptr) {
     int rc = check_desc(desc, true);
     if (rc != QLORA_OK) return rc;
     if (M < 0) return QLORA_ERR_INVALID_ARG;
@@ -234,8 +236,15 @@ static int bwd_input_common(const qlora_desc* desc, int M, const void* dY, const
         return launch_stream_gemm(d, M, true, dY, Q, scales, zeros, B, A, G, !fused, dX, st);
     }
     unsigned int* sync = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + w.sync_off);
-    if (umma_supported(d, M)) return launch_umma_gemm(d, M, true, dY, Q, scales, zeros, A, G, dX, st, B, sync, static_cast<char*>(workspace) + w.split_off,
-                                workspace_bytes - w.split_off);   // computes G
+    if (umma_supported(d, M)) {                                        // computes G (and takes dB on where it can)
+        const size_t split_bytes = workspace_bytes < w.db_off ? workspace_bytes - w.split_off : w.db_off - w.split_off;
+        if (db != nullptr) {
+            db->part = reinterpret_cast<float*>(static_cast<char*>(workspace) + w.db_off);
+            db->part_bytes = workspace_bytes > w.db_off ? workspace_bytes - w.db_off : 0;
+        }
+        return launch_umma_gemm(d, M, true, dY, Q, scales, zeros, A, G, dX, st, B, sync, static_cast<char*>(workspace) + w.split_off,
+                                split_bytes, db);
+    }
     if (d.r > 0) {
         rc = launch_lora_down(M, d.N, d.r, false, dY, B, G, st);
         if (rc != QLORA_OK) return rc;
@@ -252,9 +261,10 @@ static int bwd_lora_common(const qlora_desc* desc, int M, const void* X, const u
     if (M < 0 || (accumulate != 0 && accumulate != 1)) return QLORA_ERR_INVALID_ARG;
     const qlora_desc& d = *desc;
     if (d.r == 0) return QLORA_OK;
-    if (!dA || !dB) return QLORA_ERR_INVALID_ARG;
-    if (M > 0 && (!X || !dY)) return QLORA_ERR_INVALID_ARG;
-    if (M > 0 && ((!H && !A) || (!G && !B))) return QLORA_ERR_INVALID_ARG;
+    if (!dA) return QLORA_ERR_INVALID_ARG;
+    const bool want_dB = dB != nullptr;                     // NULL: dB was computed by qlora_bwd_input_db; only dA is wanted
+    if (M > 0 && (!X || (!dY && (want_dB || !G)))) return QLORA_ERR_INVALID_ARG;
+    if (M > 0 && ((want_dB && !H && !A) || (!G && !B))) return QLORA_ERR_INVALID_ARG;
     if (!aligned16(X) || !aligned16(dY) || !aligned16(A) || !aligned16(B) || !aligned16(H) || !aligned16(G) ||
         !aligned16(dA) || !aligned16(dB) || !aligned16(workspace))
         return QLORA_ERR_ALIGNMENT;
@@ -263,7 +273,7 @@ static int bwd_lora_common(const qlora_desc* desc, int M, const void* X, const u
     cudaStream_t st = (cudaStream_t)cuda_stream;
     char* ws = static_cast<char*>(workspace);
     const float s = d.alpha / (float)d.r;
-    if (M > 0 && !H) {
+    if (M > 0 && !H && want_dB) {
         float* Hs = reinterpret_cast<float*>(ws + w.p0_off);
         rc = launch_lora_down(M, d.K, d.r, true, X, A, Hs, st, mask, keep_scale);
         if (rc != QLORA_OK) return rc;
@@ -275,7 +285,7 @@ static int bwd_lora_common(const qlora_desc* desc, int M, const void* X, const u
         if (rc != QLORA_OK) return rc;
         G = Gs;
     }
-    return launch_lora_grads(M, d.K, d.N, d.r, s, X, dY, H, G, dA, dB, accumulate, ws + w.grad_off, st, mask, keep_scale);
+    return launch_lora_grads(M, d.K, d.N, d.r, s, X, dY, H, G, dA, dB, accumulate, ws + w.grad_off, st, mask, keep_scale, want_dB ? 3 : 2);
 }
 
 static int check_dropout(const void* mask, float keep_scale, int M) {
@@ -295,6 +305,25 @@ int qlora_bwd_input(const qlora_desc* desc, int M, const void* dY, const int32_t
                     const void* zeros, const void* A, const void* B, void* dX, float* G_out, void* workspace,
                     size_t workspace_bytes, void* cuda_stream) {
     return bwd_input_common(desc, M, dY, nullptr, 1.0f, Q, scales, zeros, A, B, dX, G_out, workspace, workspace_bytes, cuda_stream);
+}
+
+int qlora_bwd_input_db(const qlora_desc* desc, int M, const void* dY, const int32_t* Q, const void* scales,
+                       const void* zeros, const void* A, const void* B, const float* H, void* dX, float* G_out, float* dB,
+                       int accumulate, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (desc == nullptr) return QLORA_ERR_INVALID_ARG;
+    if (accumulate != 0 && accumulate != 1) return QLORA_ERR_INVALID_ARG;
+    if (desc->r > 0 && M > 0 && (!H || !dB)) return QLORA_ERR_INVALID_ARG;
+    if (!aligned16(H) || !aligned16(dB)) return QLORA_ERR_ALIGNMENT;
+    DbFuse db{H, dB, accumulate, nullptr, 0, false};
+    int rc = bwd_input_common(desc, M, dY, nullptr, 1.0f, Q, scales, zeros, A, B, dX, G_out, workspace, workspace_bytes, cuda_stream,
+                              desc->r > 0 ? &db : nullptr);
+    if (rc != QLORA_OK || desc->r == 0 || db.done || M < 0) return rc;
+    // the backward kernel of this shape has no producer clusters to do it: dB by the LoRA-gradient kernels (dY is read again)
+    const qlora_desc& d = *desc;
+    if (d.N == 0) return QLORA_OK;
+    const Workspace w = carve(d, M);
+    return launch_lora_grads(M, d.K, d.N, d.r, d.alpha / (float)d.r, nullptr, dY, H, nullptr, nullptr, dB, accumulate,
+                             static_cast<char*>(workspace) + w.grad_off, (cudaStream_t)cuda_stream, nullptr, 1.0f, 1);
 }
 
 int qlora_bwd_lora(const qlora_desc* desc, int M, const void* X, const void* dY, const void* A, const void* B,

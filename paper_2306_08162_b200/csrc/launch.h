@@ -36,9 +36,10 @@ int launch_lora_down_stream(int M, int T, int r, bool l_is_A, const void* In, co
 // dB = s dY^T H [N, r] and dA = s G^T X [r, K] in one pair of launches (partial sums per row slice, then a fixed-order
 // reduction); scratch needs lora_grad_scratch_bytes().
 size_t lora_grad_scratch_bytes(int M, int K, int N, int r);
+// sides: 1 = dB only, 2 = dA only, 3 = both (the tensors of a side that is left out may be NULL)
 int launch_lora_grads(int M, int K, int N, int r, float s, const void* X, const void* dY, const float* H, const float* G,
                       float* dA, float* dB, int accumulate, void* scratch, cudaStream_t st, const uint8_t* x_mask = nullptr,
-                      float keep_scale = 1.0f);
+                      float keep_scale = 1.0f, int sides = 3);
 // dX[m, k] += mask[m, k] * c * sum_j G[m, j] A[j, k]: the LoRA term of the backward pass under dropout.
 int launch_lora_masked_update(int M, int K, int r, float c, const float* G, const void* A, const uint8_t* mask, void* dX,
                               cudaStream_t st);
@@ -49,10 +50,23 @@ int launch_lora_masked_update(int M, int K, int r, float c, const float* G, cons
 // tiles through the two counters at `sync`, device memory the caller owns: the layer calls carve them out of their
 // workspace, so calls that may overlap in time have different ones), otherwise by a down-projection launch ahead of it.
 bool umma_supported(const qlora_desc& d, int M);
+// dB = s dY^T H as a by-product of the backward call: the producer clusters of the CTA-pair kernel stream every row of dY
+// to form G, and the same pass gives dB (ranks up to 8).  `part`: workspace for one [N, r] fp32 part per producer CTA.
+// `done` is set when the launch took it on; otherwise dB is still to be computed by the caller.
+struct DbFuse {
+    const float* H;
+    float* dB;
+    int accumulate;
+    float* part;
+    size_t part_bytes;
+    bool done;
+};
+// Workspace bytes with which any backward call of this shape can take dB on (0: none can).
+size_t umma_db_part_bytes(const qlora_desc& d, int M);
 int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q,
                      const void* scales, const void* zeros, const void* L, float* P, void* Out,
                      cudaStream_t st, const void* Ldown = nullptr, unsigned int* sync = nullptr, void* split_buf = nullptr,
-                     size_t split_bytes = 0);
+                     size_t split_bytes = 0, DbFuse* db = nullptr);
 // Bytes of workspace (`split_buf`) with which the CTA-pair kernel splits the tiles of a partly filled last wave along the
 // contraction (two SM pairs per tile, exchanging halves of the result); 0 when it would not.  Needs `sync` as well.
 size_t umma_split_scratch_bytes(const qlora_desc& d, int M);

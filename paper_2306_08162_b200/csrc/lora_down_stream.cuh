@@ -31,10 +31,18 @@ constexpr int LDS_MIN_STAGES = (LDS_CWARPS * LDS_MAXB * 2 * 128 * 4 + LDS_STAGE_
 // Row blocks first_block, first_block + block_stride, ... (at most LDS_MAXB of them below ceil(M / 16)).
 // Called by all threads of the CTA (15 warps or more; the first 15 work); `smem` is 128-byte aligned with room for lds_smem_bytes(stages), stages >=
 // LDS_MIN_STAGES.  Returns with no copy in flight (every issued stage has been waited for) unless the kernel is aborting.
-template <bool L_IS_A, int NT>
+// WITH_DB (backward only: In = dY [M, T = N], L = B): the rows that pass through for G = dY B also give this CTA's part of
+//   dB[n, j] = sum_m dY[m, n] H[m, j]   (H fp32 [M, r], the forward's down-projection; the scale s is applied by whoever adds the parts up)
+// as a second product per fragment: the tokens are now the contraction, so the 8 x 8 blocks of the dY fragments are
+// transposed across the warp (movmatrix) into the 16-row operand and H supplies the 8-column one.  A warp owns the columns
+// n of its own contraction steps, so nothing is summed across warps; its accumulators live for one chunk and are then
+// written to dBpart [T, r] (fp32, this CTA's own: every n below T is written exactly once, provided the CTA has a row block).
+template <bool L_IS_A, int NT, bool WITH_DB = false>
 __device__ __forceinline__ void lora_down_stream(int M, int T, int r, const __nv_bfloat16* __restrict__ In,
                                                  const __nv_bfloat16* __restrict__ L, float* __restrict__ P, int first_block,
-                                                 int block_stride, uint8_t* smem, int stages, volatile int* abort_flag) {
+                                                 int block_stride, uint8_t* smem, int stages, volatile int* abort_flag,
+                                                 const float* __restrict__ Hm = nullptr, float* __restrict__ dBpart = nullptr) {
+    static_assert(!(WITH_DB && L_IS_A), "dB rides on the backward's pass over dY");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, q = lane & 3;
     const uint32_t ring = smem_u32(smem);
@@ -121,9 +129,36 @@ __device__ __forceinline__ void lora_down_stream(int M, int T, int r, const __nv
                     lf[i][nt] = lv;
                 }
             }
+            float dbacc[WITH_DB ? LDS_STEPS : 1][2][NT][4];
+            if constexpr (WITH_DB) {
+#pragma unroll
+                for (int i = 0; i < LDS_STEPS; ++i)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) dbacc[i][h][nt][0] = dbacc[i][h][nt][1] = dbacc[i][h][nt][2] = dbacc[i][h][nt][3] = 0.f;
+            }
 #pragma unroll
             for (int b = 0; b < LDS_MAXB; ++b) {
                 if (b < nb && live) {
+                    uint32_t hb[NT][2];                                    // H rows of the block as the 8-column operand (tokens = contraction)
+                    if constexpr (WITH_DB) {
+                        const int mh = (first_block + b * block_stride) * 16 + 2 * q;
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            const int j = nt * 8 + g;
+                            float h0 = 0.f, h1 = 0.f, h2 = 0.f, h3 = 0.f;
+                            if (j < r) {
+                                if (mh < M) h0 = Hm[(size_t)mh * r + j];
+                                if (mh + 1 < M) h1 = Hm[(size_t)(mh + 1) * r + j];
+                                if (mh + 8 < M) h2 = Hm[(size_t)(mh + 8) * r + j];
+                                if (mh + 9 < M) h3 = Hm[(size_t)(mh + 9) * r + j];
+                            }
+                            const __nv_bfloat162 p0 = __floats2bfloat162_rn(h0, h1), p1 = __floats2bfloat162_rn(h2, h3);
+                            hb[nt][0] = *reinterpret_cast<const uint32_t*>(&p0);
+                            hb[nt][1] = *reinterpret_cast<const uint32_t*>(&p1);
+                        }
+                    }
                     if (!warp_wait(bar_full + 8 * slot, phase, abort_flag, lane)) { live = false; break; }
                     const int m0 = (first_block + b * block_stride) * 16;
                     const bool v0 = m0 + g < M, v1 = m0 + g + 8 < M;       // rows beyond M were not copied
@@ -140,11 +175,43 @@ __device__ __forceinline__ void lora_down_stream(int M, int T, int r, const __nv
                                 mma_bf16_16816(acc[b][nt], xlo.x, xhi.x, xlo.y, xhi.y, lf[i][nt].x, lf[i][nt].y);
                                 mma_bf16_16816(acc[b][nt], xlo.z, xhi.z, xlo.w, xhi.w, lf[i][nt].z, lf[i][nt].w);
                             }
+                            if constexpr (WITH_DB) {
+                                // transposed 8 x 8 blocks: lane (g, q) then holds tokens 2q, 2q + 1 (+ 8) of column
+                                // kl + 8 (g >> 1) + (g & 1) + {0, 2, 4, 6} -- the rows of the two products below
+                                const uint32_t t0x = movmatrix_trans(xlo.x), t0y = movmatrix_trans(xlo.y), t1x = movmatrix_trans(xhi.x), t1y = movmatrix_trans(xhi.y);
+                                const uint32_t t0z = movmatrix_trans(xlo.z), t0w = movmatrix_trans(xlo.w), t1z = movmatrix_trans(xhi.z), t1w = movmatrix_trans(xhi.w);
+#pragma unroll
+                                for (int nt = 0; nt < NT; ++nt) {
+                                    mma_bf16_16816(dbacc[i][0][nt], t0x, t0y, t1x, t1y, hb[nt][0], hb[nt][1]);
+                                    mma_bf16_16816(dbacc[i][1][nt], t0z, t0w, t1z, t1w, hb[nt][0], hb[nt][1]);
+                                }
+                            }
                         }
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_empty + 8 * slot);
                     if (++slot == (uint32_t)stages) { slot = 0; phase ^= 1u; }
+                }
+            }
+            if constexpr (WITH_DB) {
+                // accumulator (i, h, nt): rows g / g + 8 = columns n and n + 2, n = step base + 4 h + 8 (g >> 1) + (g & 1); ranks 2q, 2q + 1
+                if (live && nb > 0) {
+#pragma unroll
+                    for (int i = 0; i < LDS_STEPS; ++i) {
+                        const int kl = (warp + i * LDS_CWARPS) * 32;
+                        if (kl < chunk_len) {
+#pragma unroll
+                            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                                for (int nt = 0; nt < NT; ++nt) {
+                                    const int n = t0 + kl + 4 * h + 8 * (g >> 1) + (g & 1), j = nt * 8 + 2 * q;
+                                    if (j < r) {
+                                        if (n < T) *reinterpret_cast<float2*>(dBpart + (size_t)n * r + j) = make_float2(dbacc[i][h][nt][0], dbacc[i][h][nt][1]);
+                                        if (n + 2 < T) *reinterpret_cast<float2*>(dBpart + (size_t)(n + 2) * r + j) = make_float2(dbacc[i][h][nt][2], dbacc[i][h][nt][3]);
+                                    }
+                                }
+                        }
+                    }
                 }
             }
         }

@@ -195,6 +195,7 @@ struct GradSide {
     int C;
     const uint8_t* mask;       // [M, C] dropout mask on In (non-zero = keep), or NULL
     float scale;               // s (times the dropout keep scale on the masked side)
+    int out_is_dB;             // Out is dB [C, r] (else dA [r, C])
 };
 
 // thread-block cluster helpers of the one-launch form below
@@ -303,7 +304,7 @@ lora_grad_partial_kernel(int M, int r, int rows_per_slice, GradSide side0, GradS
         uint32_t peer[CL];
 #pragma unroll
         for (int k = 0; k < CL; ++k) peer[k] = lg_map_to_cta(tile, (uint32_t)k);
-        const bool is_dB = blockIdx.z == 0;
+        const bool is_dB = sd.out_is_dB != 0;
         for (int e = threadIdx.x; e < COLS_PER * (RP / 4); e += LG_WARPS * 32) {
             const int cl = slice * COLS_PER + e / (RP / 4), j = (e % (RP / 4)) * 4;     // column inside the block, first of four ranks
             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -367,16 +368,20 @@ __global__ void lora_grad_reduce_kernel(int r, int slices, int accumulate, GradS
 }
 
 int launch_lora_grads(int M, int K, int N, int r, float s, const void* X, const void* dY, const float* H, const float* G,
-                      float* dA, float* dB, int accumulate, void* scratch, cudaStream_t st, const uint8_t* x_mask, float keep_scale) {
+                      float* dA, float* dB, int accumulate, void* scratch, cudaStream_t st, const uint8_t* x_mask, float keep_scale,
+                      int sides) {
     if (r == 0) return QLORA_OK;
+    const bool want_dB = (sides & 1) != 0, want_dA = (sides & 2) != 0;
+    if (!want_dB && !want_dA) return QLORA_OK;
     if (M == 0) {   // empty sums: dA = dB = 0 unless accumulating
         if (!accumulate) {
-            if (cudaMemsetAsync(dA, 0, (size_t)r * K * sizeof(float), st) != cudaSuccess) return QLORA_ERR_CUDA;
-            if (cudaMemsetAsync(dB, 0, (size_t)N * r * sizeof(float), st) != cudaSuccess) return QLORA_ERR_CUDA;
+            if (want_dA && cudaMemsetAsync(dA, 0, (size_t)r * K * sizeof(float), st) != cudaSuccess) return QLORA_ERR_CUDA;
+            if (want_dB && cudaMemsetAsync(dB, 0, (size_t)N * r * sizeof(float), st) != cudaSuccess) return QLORA_ERR_CUDA;
         }
         return QLORA_OK;
     }
-    const int cols = (N > K ? N : K);
+    const int n_sides = (want_dB ? 1 : 0) + (want_dA ? 1 : 0);
+    const int cols = want_dB && want_dA ? (N > K ? N : K) : (want_dB ? N : K);
     const int col_blocks = (cols + LG_COLS - 1) / LG_COLS;
     const int rt = (r + 15) / 16;
     cudaError_t err = cudaSuccess;
@@ -387,11 +392,12 @@ int launch_lora_grads(int M, int K, int N, int r, float s, const void* X, const 
     while (cl > 1 && M <= 64 * (cl / 2)) cl /= 2;
     const int rows_cl = ((M + cl - 1) / cl + 63) / 64 * 64;
     if (M <= 256) {
-        GradSide sB{(const __nv_bfloat16*)dY, H, nullptr, dB, N, nullptr, s};
-        GradSide sA{(const __nv_bfloat16*)X, G, nullptr, dA, K, x_mask, x_mask ? s * keep_scale : s};
+        GradSide sB{(const __nv_bfloat16*)dY, H, nullptr, dB, N, nullptr, s, 1};
+        GradSide sA{(const __nv_bfloat16*)X, G, nullptr, dA, K, x_mask, x_mask ? s * keep_scale : s, 0};
+        if (!want_dB) sB = sA;                                  // one side only: it is the first (and only) z-slice of the grid
         const size_t pt_bytes = (size_t)rt * 16 * (rows_cl + 8) * sizeof(__nv_bfloat16), tile_bytes = (size_t)LG_COLS * rt * 16 * sizeof(float);
         const size_t smem = pt_bytes > tile_bytes ? pt_bytes : tile_bytes;
-        const dim3 grid((unsigned)(col_blocks * cl), 1, 2);
+        const dim3 grid((unsigned)(col_blocks * cl), 1, (unsigned)n_sides);
 #define QLORA_LGC(RTV, CLV)                                                                                    \
     do {                                                                                                       \
         static SmemLimit limit;                                                                                \
@@ -415,12 +421,26 @@ int launch_lora_grads(int M, int K, int N, int r, float s, const void* X, const 
         return err == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
     }
     // More tokens: partial sums per row slice to scratch, then a reduction launch.
-    const GradPlan plan = lora_grad_plan(M, K, N);
+    GradPlan plan = lora_grad_plan(M, K, N);
+    if (n_sides == 1) {
+        // one gradient only: its column blocks alone would leave most SMs without a block, so the rows are cut finer -- as
+        // fine as the scratch sized for both gradients allows
+        const size_t room = (size_t)plan.slices * (size_t)(K + N);
+        const int C1 = want_dB ? N : K;
+        GradPlan one = lora_grad_plan(M, want_dB ? 0 : K, want_dB ? N : 0);
+        while ((size_t)one.slices * C1 > room && one.rows_per_slice < 1024) {
+            one.rows_per_slice += 64;
+            one.slices = (M + one.rows_per_slice - 1) / one.rows_per_slice;
+        }
+        if ((size_t)one.slices * C1 <= room) plan = one;
+    }
     float* part_dB = (float*)scratch;
-    float* part_dA = part_dB + (size_t)plan.slices * N * r;
-    GradSide sB{(const __nv_bfloat16*)dY, H, part_dB, dB, N, nullptr, s};
-    GradSide sA{(const __nv_bfloat16*)X, G, part_dA, dA, K, x_mask, x_mask ? s * keep_scale : s};
-    dim3 grid(col_blocks, plan.slices, 2);
+    float* part_dA = n_sides == 1 ? part_dB : part_dB + (size_t)plan.slices * N * r;   // (alone, it starts at the base)
+    GradSide sB{(const __nv_bfloat16*)dY, H, part_dB, dB, N, nullptr, s, 1};
+    GradSide sA{(const __nv_bfloat16*)X, G, part_dA, dA, K, x_mask, x_mask ? s * keep_scale : s, 0};
+    GradSide none{};                                         // C = 0: no elements for the reduction
+    if (!want_dB) sB = sA;
+    dim3 grid(col_blocks, plan.slices, (unsigned)n_sides);
     const size_t smem = (size_t)rt * 16 * (plan.rows_per_slice + 8) * sizeof(__nv_bfloat16);
 #define QLORA_LG(RTV)                                                                                          \
     do {                                                                                                       \
@@ -436,8 +456,10 @@ int launch_lora_grads(int M, int K, int N, int r, float s, const void* X, const 
     }
 #undef QLORA_LG
     if (err != cudaSuccess) return QLORA_ERR_CUDA;
-    const size_t total = (size_t)(N + K) * r;
-    err = launch_pdl(lora_grad_reduce_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st, 1, r, plan.slices, accumulate, sB, sA);
+    const GradSide& rB = want_dB ? sB : none;
+    const GradSide& rA = want_dA ? sA : none;
+    const size_t total = (size_t)(rB.C + rA.C) * r;
+    err = launch_pdl(lora_grad_reduce_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st, 1, r, plan.slices, accumulate, rB, rA);
     return err == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
 }
 

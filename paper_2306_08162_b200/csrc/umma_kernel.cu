@@ -720,10 +720,20 @@ size_t umma_split_scratch_bytes(const qlora_desc& d, int M) {
     return (size_t)(rem_f > rem_b ? rem_f : rem_b) * kSplitTileBytes;
 }
 
+// Workspace with which a backward call of this shape can compute dB on its producer clusters: one [N, r] fp32 part per
+// producer CTA, for as many producers as the shape could ever get (0: the CTA-pair kernel would not take dB on).
+size_t umma_db_part_bytes(const qlora_desc& d, int M) {
+    if (M <= 256 || !umma_supported(d, M) || d.r == 0 || d.r > 8) return 0;
+    const int pairs = sm_count() / 2, n_blocks = (M + 15) / 16;
+    int n_prod = (n_blocks + 3) / 4;
+    if (n_prod > pairs) n_prod = pairs;
+    return (size_t)2 * n_prod * (size_t)d.N * d.r * sizeof(float);
+}
+
 // CTA-pair kernel: 512 tokens x 256 weight rows per pair of SMs (see prefer_pair_kernel for when it is used).
 static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
                             const void* zeros, const void* L, float* Pmat, void* Out, cudaStream_t st, const void* Ldown,
-                            unsigned int* sync, void* split_buf, size_t split_bytes) {
+                            unsigned int* sync, void* split_buf, size_t split_bytes, DbFuse* db) {
     PairParams p{};
     p.M = M; p.N = d.N; p.K = d.K; p.bits = d.bits; p.g = d.group_size; p.r = d.r; p.r_pad = (d.r + 15) / 16 * 16;
     p.C = transposed ? d.K : d.N;
@@ -802,6 +812,13 @@ static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const v
             if (rc != QLORA_OK) return rc;
         }
     }
+    // dB on the producers' pass over dY (backward, one rank tile): every producer CTA leaves its part in the workspace
+    p.with_db = 0;
+    if (db != nullptr && transposed && p.n_prod > 0 && d.r <= 8 && db->H != nullptr && db->dB != nullptr && db->part != nullptr &&
+        (size_t)2 * p.n_prod * (size_t)T * d.r * sizeof(float) <= db->part_bytes) {
+        p.with_db = 1; p.db_accumulate = db->accumulate; p.Hmat = db->H; p.db_part = db->part; p.db_out = db->dB;
+        db->done = true;
+    }
     if (p.n_prod > 0 || p.nsplit > 1) {                      // the counters in the workspace are in use: zero them in stream order
         p.sync = sync;
         const int rc = zero_sync_pair(sync, st);
@@ -844,9 +861,9 @@ static bool prefer_pair_kernel(const qlora_desc& d, int M, bool transposed) {
 
 int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
                      const void* zeros, const void* L, float* Pmat, void* Out, cudaStream_t st, const void* Ldown,
-                     unsigned int* sync, void* split_buf, size_t split_bytes) {
+                     unsigned int* sync, void* split_buf, size_t split_bytes, DbFuse* db) {
     if (prefer_pair_kernel(d, M, transposed))
-        return launch_umma_pair(d, M, transposed, In, Q, scales, zeros, L, Pmat, Out, st, Ldown, sync, split_buf, split_bytes);
+        return launch_umma_pair(d, M, transposed, In, Q, scales, zeros, L, Pmat, Out, st, Ldown, sync, split_buf, split_bytes, db);
     Params p{};
     p.M = M; p.N = d.N; p.K = d.K; p.bits = d.bits; p.g = d.group_size; p.r = d.r; p.r_pad = (d.r + 15) / 16 * 16;
     p.C = transposed ? d.K : d.N;

@@ -60,6 +60,11 @@ struct PairParams {
     const __nv_bfloat16* In;     // [M, T]
     const __nv_bfloat16* Ldown;  // A [r, K] (forward) or B [N, r] (backward)
     float* Pout;
+    // backward with producer clusters only: dB = s dY^T H computed on the producers' pass over dY (with_db)
+    int with_db, db_accumulate;
+    const float* Hmat;           // H fp32 [M, r]
+    float* db_part;              // [2 n_prod][N][r] fp32, one part per producer CTA (workspace)
+    float* db_out;               // dB fp32 [N, r]
 };
 
 
@@ -212,11 +217,48 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         // ------------------------------------------------------------------ producer cluster: LoRA down-projection first
         // (this CTA's row blocks: blockIdx.x, blockIdx.x + 2 n_prod, ...; the ring takes the operand area, below the barriers)
         pdl_wait();
-        if (p.r <= 8) lora_down_stream<!TRANSPOSED, 1>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, 2 * p.n_prod, smem_gen, p.lds_stages, abort_flag);
-        else          lora_down_stream<!TRANSPOSED, 2>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, 2 * p.n_prod, smem_gen, p.lds_stages, abort_flag);
-        __threadfence();       // every thread's rows of P are visible device-wide before the CTA is counted
+        bool db_here = false;
+        if constexpr (TRANSPOSED) {
+            if (p.with_db) {       // the same pass over dY also gives this CTA's part of dB
+                db_here = true;
+                float* part = p.db_part + (size_t)blockIdx.x * p.T * p.r;
+                lora_down_stream<false, 1, true>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, 2 * p.n_prod, smem_gen, p.lds_stages, abort_flag, p.Hmat, part);   // (the host asks for this with r <= 8 only: two rank tiles would not fit the registers)
+            }
+        }
+        if (!db_here) {
+            if (p.r <= 8) lora_down_stream<!TRANSPOSED, 1>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, 2 * p.n_prod, smem_gen, p.lds_stages, abort_flag);
+            else          lora_down_stream<!TRANSPOSED, 2>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, 2 * p.n_prod, smem_gen, p.lds_stages, abort_flag);
+        }
+        __threadfence();       // every thread's rows of P (and of its part of dB) are visible device-wide before the CTA is counted
         __syncthreads();
         if (threadIdx.x == 0) atomicAdd(&p.sync[0], 1u);
+        if (db_here) {
+            // The producers meet at a counter of their own (all of them are resident: they are the first clusters of a grid of
+            // at most one CTA per SM), then producer CTA i adds the parts, in CTA order, for its share of the columns.
+            const unsigned n_ctas = 2u * (unsigned)p.n_prod;
+            if (threadIdx.x == 0) {
+                atomicAdd(&p.sync[kSyncWords - 1], 1u);
+                wait_counter(&p.sync[kSyncWords - 1], n_ctas, abort_flag);
+            }
+            __syncthreads();
+            if (!*abort_flag) {
+                const int n_blocks = (p.M + 15) >> 4;
+                const int n_src = (int)n_ctas < n_blocks ? (int)n_ctas : n_blocks;      // CTAs beyond the row blocks wrote nothing
+                const size_t part_elems = (size_t)p.T * p.r;
+                const size_t e_lo = (size_t)p.T * blockIdx.x / n_ctas * p.r / 4, e_hi = (size_t)p.T * (blockIdx.x + 1) / n_ctas * p.r / 4;
+                for (size_t e4 = e_lo + threadIdx.x; e4 < e_hi; e4 += blockDim.x) {
+                    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int src = 0; src < n_src; ++src) {
+                        const float4 x = __ldcg(reinterpret_cast<const float4*>(p.db_part + (size_t)src * part_elems) + e4);
+                        v.x += x.x; v.y += x.y; v.z += x.z; v.w += x.w;
+                    }
+                    v.x *= p.s; v.y *= p.s; v.z *= p.s; v.w *= p.s;
+                    float4* dst = reinterpret_cast<float4*>(p.db_out) + e4;
+                    if (p.db_accumulate) { const float4 o = *dst; v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w; }
+                    *dst = v;
+                }
+            }
+        }
         fence_proxy_async();   // the shared memory just used goes to the TMA / tensor-core side for this cluster's tiles, if any
         __syncthreads();
     }
