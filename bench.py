@@ -63,7 +63,7 @@ def weight_bytes(w):
 
 # DRAM traffic (read + write) per launch of the dominant kernel of the default workload, from one ncu capture of that
 # kernel (dram__bytes_read.sum + dram__bytes_write.sum).  Set back to None whenever that kernel changes.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 26.03e6
+NCU_TRAFFIC_BYTES_PER_LAUNCH = (26.13e6, 26.56e6)   # forward, backward-input (with dB)
 
 
 def layer_flops(M, K, N, r):
@@ -582,7 +582,7 @@ def run_ours(args):
                          "frac": achieved / peak,
                          "frac_sustained": ((achieved * total_ms / sus_ms) / peaks["bf16_sustained"]
                                             if (sustained and bound == "tensor" and sus_ms > 0) else None),
-                         "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if args.workload == "config2" else None,
+                         "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH[dom] if args.workload == "config2" and NCU_TRAFFIC_BYTES_PER_LAUNCH else None,
                          "peak_kind": peak_kind,
                          "step_frac_of_peak": (value / world / peak) if bound == "tensor" else None},
             "sustained": (None if not sustained else {
