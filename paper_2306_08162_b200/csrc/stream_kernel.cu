@@ -1024,6 +1024,15 @@ bool stream_supported(const qlora_desc& d, int M, bool transposed) {
     return d.group_size % fwd_kb(d.bits) == 0;
 }
 
+// The frozen tensors of a layer asked into L2 by a handful of small CTAs that run under the preceding kernel of the stream
+// (see stream_prefetch_kernel); the kernel launched behind it is ordered after everything before it.
+int launch_weight_prefetch(const qlora_desc& d, const int32_t* Q, const void* scales, const void* zeros, cudaStream_t st) {
+    const size_t q_bytes = (size_t)d.K * d.bits / 8 * d.N, sz_bytes = (size_t)(d.K / d.group_size) * d.N * 2;
+    const unsigned blocks = (unsigned)((q_bytes / ST_PF_CHUNK + 127) / 128 + 1);
+    return launch_pdl(stream_prefetch_kernel, dim3(blocks), dim3(128), 0, st, 1, (const char*)Q, q_bytes, (const char*)scales,
+                      (const char*)zeros, sz_bytes) == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
+}
+
 int launch_stream_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
                        const void* zeros, const void* Ldown, const void* Lup, float* P, bool p_is_input, void* Out,
                        cudaStream_t st) {
@@ -1090,11 +1099,8 @@ int launch_stream_gemm(const qlora_desc& d, int M, bool transposed, const void* 
     }
     if (smem > 227 * 1024) return QLORA_ERR_UNSUPPORTED;
     {   // the frozen tensors on their way into L2 while the preceding call computes
-        const size_t q_bytes = (size_t)d.K * d.bits / 8 * d.N, sz_bytes = (size_t)(d.K / d.group_size) * d.N * 2;
-        const unsigned blocks = (unsigned)((q_bytes / ST_PF_CHUNK + 127) / 128 + 1);
-        if (launch_pdl(stream_prefetch_kernel, dim3(blocks), dim3(128), 0, st, 1, (const char*)Q, q_bytes, (const char*)scales, (const char*)zeros,
-                       sz_bytes) != cudaSuccess)
-            return QLORA_ERR_CUDA;
+        const int rc = launch_weight_prefetch(d, Q, scales, zeros, st);
+        if (rc != QLORA_OK) return rc;
     }
 #define QLORA_ST(B, NT)                                                                                   \
     return transposed ? st_launch<B, NT, true>(p, nw, tiles, smem, st) : st_launch<B, NT, false>(p, nw, tiles, smem, st)
