@@ -408,7 +408,7 @@ def run_ours(args):
 
     # With many tokens dB rides on the backward call (qlora_bwd_input_db: dY is read once) and the gradient call computes
     # dA alone; with few tokens the three plain calls.  Either way a step produces Y, H, dX, G, dA and dB.
-    fused_db = M > 256 and r > 0
+    fused_db = M > 256 and 0 < r <= 8     # (two rank tiles: the backward call would hand dB to the gradient kernels anyway)
     bwd_name = "qlora_bwd_input_db" if fused_db else "qlora_bwd_input"
 
     def bwd_input_call(L):
