@@ -408,7 +408,7 @@ def run_ours(args):
 
     # With many tokens dB rides on the backward call (qlora_bwd_input_db: dY is read once) and the gradient call computes
     # dA alone; with few tokens the three plain calls.  Either way a step produces Y, H, dX, G, dA and dB.
-    fused_db = M > 256 and 0 < r <= 8     # (two rank tiles: the backward call would hand dB to the gradient kernels anyway)
+    fused_db = ql.qlora_bwd_input_db_on_producers(d, M)    # (else the backward call would hand dB to the gradient kernels anyway)
     bwd_name = "qlora_bwd_input_db" if fused_db else "qlora_bwd_input"
 
     def bwd_input_call(L):
@@ -628,7 +628,7 @@ def run_chain(args):
         for name, K, N in shapes:
             d = ql.desc(bits, g, K, N, r, alpha)
             ws_bytes = max(ws_bytes, ql.qlora_workspace_bytes(d, M))
-            row[name] = dict(d=d, K=K, N=N,
+            row[name] = dict(d=d, K=K, N=N, db_on_producers=ql.qlora_bwd_input_db_on_producers(d, M),
                              Q=torch.randint(-2**31, 2**31 - 1, (K * bits // 32, N), dtype=torch.int32, device=dev, generator=gen),
                              s=torch.full((K // g, N), 0.85 / float(np.sqrt(1.25 * K)), dtype=torch.float16, device=dev),
                              z=torch.randint(1, 3, (K // g, N), device=dev, generator=gen).half(),
@@ -658,8 +658,12 @@ def run_chain(args):
                 dY = {"down": grad, "up": seed_grad[11008], "v": seed_grad[4096], "k": seed_grad[4096]}.get(name)
                 if dY is None:
                     dY = row[{"gate": "down", "o": "gate", "q": "o"}[name]]["dX"]
-                ql.qlora_bwd_input_db(P["d"], M, dY, P["Q"], P["s"], P["z"], P["A"], P["B"], P["H"], P["dX"], P["G"], P["dB"], 0, ws)
-                ql.qlora_bwd_lora(P["d"], M, P["X"], None, P["A"], P["B"], None, P["G"], P["dA"], None, 0, ws)
+                if P["db_on_producers"]:
+                    ql.qlora_bwd_input_db(P["d"], M, dY, P["Q"], P["s"], P["z"], P["A"], P["B"], P["H"], P["dX"], P["G"], P["dB"], 0, ws)
+                    ql.qlora_bwd_lora(P["d"], M, P["X"], None, P["A"], P["B"], None, P["G"], P["dA"], None, 0, ws)
+                else:
+                    ql.qlora_bwd_input(P["d"], M, dY, P["Q"], P["s"], P["z"], P["A"], P["B"], P["dX"], P["G"], ws)
+                    ql.qlora_bwd_lora(P["d"], M, P["X"], dY, P["A"], P["B"], P["H"], P["G"], P["dA"], P["dB"], 0, ws)
             grad = row["q"]["dX"]
 
     def barrier():

@@ -109,7 +109,7 @@ int qlora_bwd_input(const qlora_desc* desc, int M, const void* dY, const int32_t
 
 /* qlora_bwd_input that also produces dB = s dY^T H (Figure 1: the backward arrow into the second LoRA block leaves the
  * same dY that flows back through the frozen weight), so that dY is read once for both.  H: fp32 [M, r], the forward's
- * H_out (required when r > 0); dB: fp32 [N, r]; accumulate as in qlora_bwd_lora.  With many tokens and r <= 8 the SMs
+ * H_out (required when r > 0); dB: fp32 [N, r]; accumulate as in qlora_bwd_lora.  With many tokens and r <= 16 the SMs
  * that stream dY to form G inside the backward kernel form dB on the same pass (each leaves a part in the workspace,
  * they add the parts in a fixed order before they go on); for other shapes dB comes from the gradient kernels after
  * the backward kernel.  Either way dB is complete when the call's work is, and the same inputs give the same bits on a
@@ -118,6 +118,12 @@ int qlora_bwd_input(const qlora_desc* desc, int M, const void* dY, const int32_t
 int qlora_bwd_input_db(const qlora_desc* desc, int M, const void* dY, const int32_t* Q, const void* scales,
                        const void* zeros, const void* A, const void* B, const float* H, void* dX, float* G_out, float* dB,
                        int accumulate, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Which way qlora_bwd_input_db goes for this shape on the current device, given the whole workspace: 1 = dB is formed
+ * on the backward kernel's pass over dY (then qlora_bwd_input_db + qlora_bwd_lora(dB = NULL) is the cheaper pair of
+ * calls), 0 = dB is handed to the gradient kernels (then qlora_bwd_input + qlora_bwd_lora is: one gradient launch
+ * instead of two); negative: a QLORA_ERR_* code.  Launches nothing.  The paper has no counterpart. */
+int qlora_bwd_input_db_on_producers(const qlora_desc* desc, int M);
 
 /* Gradients of the trainable pair (Section 3.1: only theta_l is updated; Figure 1, arrows into the LoRA blocks):
  *   dA = s (dY B)^T X  fp32 [r, K],     dB = s dY^T (X A^T)  fp32 [N, r].

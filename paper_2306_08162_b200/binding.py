@@ -47,6 +47,8 @@ def library() -> ctypes.CDLL:
     lib.qlora_fwd.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.qlora_bwd_input.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.qlora_bwd_lora.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
+    lib.qlora_bwd_input_db_on_producers.argtypes = [dp, i32]
+    lib.qlora_bwd_input_db_on_producers.restype = i32
     lib.qlora_bwd_input_db.argtypes = [dp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]
     f32 = ctypes.c_float
     lib.qlora_fwd_dropout.argtypes = [dp, i32, vp, vp, f32, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -126,6 +128,13 @@ def qlora_bwd_input_db(d, M, dY, Q, scales, zeros, A, B, H, dX, G_out, dB, accum
     _check(library().qlora_bwd_input_db(ctypes.byref(d), int(M), _ptr(dY), _ptr(Q), _ptr(scales), _ptr(zeros), _ptr(A),
                                         _ptr(B), _ptr(H), _ptr(dX), _ptr(G_out), _ptr(dB), int(accumulate), _ptr(workspace), wb,
                                         _stream(stream)), "qlora_bwd_input_db")
+
+
+def qlora_bwd_input_db_on_producers(d, M) -> bool:
+    rc = library().qlora_bwd_input_db_on_producers(ctypes.byref(d), int(M))
+    if rc < 0:
+        _check(rc, "qlora_bwd_input_db_on_producers")
+    return rc == 1
 
 
 def qlora_bwd_lora(d, M, X, dY, A, B, H, G, dA, dB, accumulate, workspace, stream=None, workspace_bytes=None):

@@ -326,6 +326,13 @@ int qlora_bwd_input_db(const qlora_desc* desc, int M, const void* dY, const int3
                              static_cast<char*>(workspace) + w.grad_off, (cudaStream_t)cuda_stream, nullptr, 1.0f, 1);
 }
 
+int qlora_bwd_input_db_on_producers(const qlora_desc* desc, int M) {
+    const int rc = check_desc(desc, true);
+    if (rc != QLORA_OK) return rc;
+    if (M < 0) return QLORA_ERR_INVALID_ARG;
+    return umma_db_on_producers(*desc, M) > 0 ? 1 : 0;
+}
+
 int qlora_bwd_lora(const qlora_desc* desc, int M, const void* X, const void* dY, const void* A, const void* B,
                    const float* H, const float* G, float* dA, float* dB, int accumulate, void* workspace,
                    size_t workspace_bytes, void* cuda_stream) {

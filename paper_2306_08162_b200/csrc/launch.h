@@ -63,6 +63,8 @@ struct DbFuse {
 };
 // Workspace bytes with which any backward call of this shape can take dB on (0: none can).
 size_t umma_db_part_bytes(const qlora_desc& d, int M);
+// The number of producer pairs on which such a call, given its whole workspace, forms dB on the current device; else 0.
+int umma_db_on_producers(const qlora_desc& d, int M);
 int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q,
                      const void* scales, const void* zeros, const void* L, float* P, void* Out,
                      cudaStream_t st, const void* Ldown = nullptr, unsigned int* sync = nullptr, void* split_buf = nullptr,

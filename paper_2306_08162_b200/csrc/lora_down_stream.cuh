@@ -37,7 +37,7 @@ constexpr int LDS_MIN_STAGES = (LDS_CWARPS * LDS_MAXB * 2 * 128 * 4 + LDS_STAGE_
 // transposed across the warp (movmatrix) into the 16-row operand and H supplies the 8-column one.  A warp owns the columns
 // n of its own contraction steps, so nothing is summed across warps; its accumulators live for one chunk and are then
 // written to dBpart [T, r] (fp32, this CTA's own: every n below T is written exactly once, provided the CTA has a row block).
-template <bool L_IS_A, int NT, bool WITH_DB = false>
+template <bool L_IS_A, int NT, bool WITH_DB = false, int MAXB = LDS_MAXB>   // MAXB: row blocks this instantiation keeps accumulators for
 __device__ __forceinline__ void lora_down_stream(int M, int T, int r, const __nv_bfloat16* __restrict__ In,
                                                  const __nv_bfloat16* __restrict__ L, float* __restrict__ P, int first_block,
                                                  int block_stride, uint8_t* smem, int stages, volatile int* abort_flag,
@@ -50,7 +50,7 @@ __device__ __forceinline__ void lora_down_stream(int M, int T, int r, const __nv
     const uint32_t bar_empty = bar_full + 8u * (uint32_t)stages;
     const int n_blocks = (M + 15) / 16;
     int nb = first_block < n_blocks ? (n_blocks - first_block + block_stride - 1) / block_stride : 0;
-    if (nb > LDS_MAXB) nb = LDS_MAXB;
+    if (nb > MAXB) nb = MAXB;
     const int n_chunks = (T + LDS_TC - 1) / LDS_TC;
 
     if (threadIdx.x == 0) {
@@ -62,9 +62,9 @@ __device__ __forceinline__ void lora_down_stream(int M, int T, int r, const __nv
     }
     __syncthreads();
 
-    float acc[LDS_MAXB][NT][4];
+    float acc[MAXB][NT][4];
 #pragma unroll
-    for (int b = 0; b < LDS_MAXB; ++b)
+    for (int b = 0; b < MAXB; ++b)
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) acc[b][nt][0] = acc[b][nt][1] = acc[b][nt][2] = acc[b][nt][3] = 0.f;
 
@@ -139,7 +139,7 @@ __device__ __forceinline__ void lora_down_stream(int M, int T, int r, const __nv
                         for (int nt = 0; nt < NT; ++nt) dbacc[i][h][nt][0] = dbacc[i][h][nt][1] = dbacc[i][h][nt][2] = dbacc[i][h][nt][3] = 0.f;
             }
 #pragma unroll
-            for (int b = 0; b < LDS_MAXB; ++b) {
+            for (int b = 0; b < MAXB; ++b) {
                 if (b < nb && live) {
                     uint32_t hb[NT][2];                                    // H rows of the block as the 8-column operand (tokens = contraction)
                     if constexpr (WITH_DB) {
@@ -221,7 +221,7 @@ __device__ __forceinline__ void lora_down_stream(int M, int T, int r, const __nv
     float* red = reinterpret_cast<float*>(smem);   // [warp][b][nt][c][lane]
     if (warp < LDS_CWARPS) {
 #pragma unroll
-        for (int b = 0; b < LDS_MAXB; ++b)
+        for (int b = 0; b < MAXB; ++b)
             if (b < nb)
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt)

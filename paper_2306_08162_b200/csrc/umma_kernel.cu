@@ -721,19 +721,17 @@ size_t umma_split_scratch_bytes(const qlora_desc& d, int M) {
 }
 
 // Workspace with which a backward call of this shape can compute dB on its producer clusters: one [N, r] fp32 part per
-// producer CTA, for as many producers as the shape could ever get (0: the CTA-pair kernel would not take dB on).
+// producer CTA (0: the CTA-pair kernel would not take dB on).
 size_t umma_db_part_bytes(const qlora_desc& d, int M) {
-    if (M <= 256 || !umma_supported(d, M) || d.r == 0 || d.r > 8) return 0;
-    const int pairs = sm_count() / 2, n_blocks = (M + 15) / 16;
-    int n_prod = (n_blocks + 3) / 4;
-    if (n_prod > pairs) n_prod = pairs;
-    return (size_t)2 * n_prod * (size_t)d.N * d.r * sizeof(float);
+    return (size_t)2 * umma_db_on_producers(d, M) * (size_t)d.N * d.r * sizeof(float);
 }
 
 // CTA-pair kernel: 512 tokens x 256 weight rows per pair of SMs (see prefer_pair_kernel for when it is used).
 static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
                             const void* zeros, const void* L, float* Pmat, void* Out, cudaStream_t st, const void* Ldown,
-                            unsigned int* sync, void* split_buf, size_t split_bytes, DbFuse* db) {
+                            unsigned int* sync, void* split_buf, size_t split_bytes, DbFuse* db, bool plan_only = false) {
+    // plan_only: nothing is launched and no pointer is looked at; the return value is the number of producer pairs when a
+    // backward call with every optional workspace area would form dB on them, else 0
     PairParams p{};
     p.M = M; p.N = d.N; p.K = d.K; p.bits = d.bits; p.g = d.group_size; p.r = d.r; p.r_pad = (d.r + 15) / 16 * 16;
     p.C = transposed ? d.K : d.N;
@@ -769,13 +767,6 @@ static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const v
     p.off_bar = (p.off_lora_p + lora_p + 127u) / 128u * 128u;
     const size_t smem_bytes = (size_t)p.off_bar + 512 + 1024;
 
-    CUtensorMap ta, tq, ts, tz;
-    if (!make_map_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, In, (uint64_t)T, (uint64_t)M, 64, (uint32_t)kPairTok, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_map_2d(&tq, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, Q, (uint64_t)d.N, (uint64_t)(d.K * d.bits / 32), (uint32_t)p.packed_cols, (uint32_t)p.packed_rows, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-        !make_map_2d(&ts, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, scales, (uint64_t)d.N, (uint64_t)(d.K / d.group_size), (uint32_t)p.packed_cols, (uint32_t)p.scale_rows, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-        !make_map_2d(&tz, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, zeros, (uint64_t)d.N, (uint64_t)(d.K / d.group_size), (uint32_t)p.packed_cols, (uint32_t)p.scale_rows, CU_TENSOR_MAP_SWIZZLE_NONE))
-        return QLORA_ERR_CUDA;
-
     const int pairs = sm_count() / 2;
     p.n_prod = 0; p.T = T; p.sync = nullptr; p.wait_limit_us = kWaitLimitUs;
     p.In = (const __nv_bfloat16*)In; p.Ldown = (const __nv_bfloat16*)Ldown; p.Pout = Pmat;
@@ -784,7 +775,8 @@ static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const v
     // P = In * Ldown still to be computed (Ldown given): on SM pairs the tiles leave idle when those can take all row
     // blocks (they are then done well before the tiles' contractions are), else by a launch ahead of this one.  Both sum
     // in the same order.  producers(last) = how many pairs would do it when the last wave has `last` items (0: none can).
-    const bool want_p = Ldown != nullptr && d.r > 0;
+    const bool want_p = (Ldown != nullptr || plan_only) && d.r > 0;
+    if (plan_only) { sync = reinterpret_cast<unsigned int*>(sizeof(unsigned int)); split_buf = sync; split_bytes = ~(size_t)0; }   // (never dereferenced)
     const int n_blocks = (M + 15) / 16;
     auto producers = [&](int last) {
         // pairs with less to do: no tile at all, or one item fewer than the rest when the last wave is partly filled
@@ -805,19 +797,29 @@ static int launch_umma_pair(const qlora_desc& d, int M, bool transposed, const v
         !(want_p && producers(2 * rem) == 0 && producers(p.n_tiles % pairs) > 0)) {
         p.n_full = p.n_tiles - rem; p.nsplit = 2; p.split_buf = static_cast<float4*>(split_buf);
     }
-    if (want_p) {
-        p.n_prod = producers(p.nsplit > 1 ? 2 * rem : p.n_tiles % pairs);
-        if (p.n_prod == 0) {
-            const int rc = launch_lora_down(M, T, d.r, !transposed, In, Ldown, Pmat, st);
-            if (rc != QLORA_OK) return rc;
-        }
-    }
-    // dB on the producers' pass over dY (backward, one rank tile): every producer CTA leaves its part in the workspace
+    if (want_p) p.n_prod = producers(p.nsplit > 1 ? 2 * rem : p.n_tiles % pairs);
+    // dB on the producers' pass over dY (backward, ranks up to 16): every producer CTA leaves its part in the workspace
+    // -- where the producers have a whole tile's time to spare: with a split last wave they are only half a tile ahead of
+    // the others, and the extra work then lengthens the kernel (down_proj backward, r = 16: 159 against 140 us)
+    const bool db_fits = transposed && p.n_prod > 0 && p.nsplit == 1 &&
+                         p.n_prod * 2 * (d.r <= 8 ? LDS_MAXB : 3) >= n_blocks;   // (two rank tiles: three row blocks per producer CTA at most)
+    if (plan_only) return db_fits ? p.n_prod : 0;
     p.with_db = 0;
-    if (db != nullptr && transposed && p.n_prod > 0 && d.r <= 8 && db->H != nullptr && db->dB != nullptr && db->part != nullptr &&
+    if (db != nullptr && db_fits && db->H != nullptr && db->dB != nullptr && db->part != nullptr &&
         (size_t)2 * p.n_prod * (size_t)T * d.r * sizeof(float) <= db->part_bytes) {
         p.with_db = 1; p.db_accumulate = db->accumulate; p.Hmat = db->H; p.db_part = db->part; p.db_out = db->dB;
         db->done = true;
+    }
+    CUtensorMap ta, tq, ts, tz;
+    if (!make_map_2d(&ta, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, In, (uint64_t)T, (uint64_t)M, 64, (uint32_t)kPairTok, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_2d(&tq, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, Q, (uint64_t)d.N, (uint64_t)(d.K * d.bits / 32), (uint32_t)p.packed_cols, (uint32_t)p.packed_rows, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_map_2d(&ts, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, scales, (uint64_t)d.N, (uint64_t)(d.K / d.group_size), (uint32_t)p.packed_cols, (uint32_t)p.scale_rows, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_map_2d(&tz, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, zeros, (uint64_t)d.N, (uint64_t)(d.K / d.group_size), (uint32_t)p.packed_cols, (uint32_t)p.scale_rows, CU_TENSOR_MAP_SWIZZLE_NONE))
+        return QLORA_ERR_CUDA;
+
+    if (want_p && p.n_prod == 0) {
+        const int rc = launch_lora_down(M, T, d.r, !transposed, In, Ldown, Pmat, st);
+        if (rc != QLORA_OK) return rc;
     }
     if (p.n_prod > 0 || p.nsplit > 1) {                      // the counters in the workspace are in use: zero them in stream order
         p.sync = sync;
@@ -857,6 +859,15 @@ static bool prefer_pair_kernel(const qlora_desc& d, int M, bool transposed) {
     const int waves_pair = (tiles_pair + sms / 2 - 1) / (sms / 2);
     const float pair_us = (float)waves_pair * ((float)steps * 0.62f + 4.0f);
     return pair_us < mid_us;
+}
+
+// The number of producer pairs on which the backward call of this shape, given its whole workspace, forms dB (on the current
+// device: its SM count decides how many pairs the tiles leave idle); 0 when dB goes to the gradient kernels.
+int umma_db_on_producers(const qlora_desc& d, int M) {
+    if (M <= 256 || d.r == 0 || d.r > 16 || !umma_supported(d, M) || !prefer_pair_kernel(d, M, true)) return 0;
+    const int rc = launch_umma_pair(d, M, true, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
+                                    nullptr, 0, nullptr, true);
+    return rc > 0 ? rc : 0;
 }
 
 int launch_umma_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,

@@ -222,7 +222,8 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             if (p.with_db) {       // the same pass over dY also gives this CTA's part of dB
                 db_here = true;
                 float* part = p.db_part + (size_t)blockIdx.x * p.T * p.r;
-                lora_down_stream<false, 1, true>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, 2 * p.n_prod, smem_gen, p.lds_stages, abort_flag, p.Hmat, part);   // (the host asks for this with r <= 8 only: two rank tiles would not fit the registers)
+                if (p.r <= 8) lora_down_stream<false, 1, true>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, 2 * p.n_prod, smem_gen, p.lds_stages, abort_flag, p.Hmat, part);
+                else          lora_down_stream<false, 2, true, 3>(p.M, p.T, p.r, p.In, p.Ldown, p.Pout, (int)blockIdx.x, 2 * p.n_prod, smem_gen, p.lds_stages, abort_flag, p.Hmat, part);   // (two rank tiles: registers for three row blocks per CTA only; the host sees to it)
             }
         }
         if (!db_here) {

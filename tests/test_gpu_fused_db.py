@@ -41,8 +41,11 @@ def run_db(gl, accumulate=0, dB0=None):
 @pytest.mark.parametrize("K,N,M,bits,g,r", [
     (1024, 1024, 1536, 4, 128, 8),      # CTA-pair kernel, 12 tiles on 74 pairs: producer clusters take dB on
     (1024, 6656, 1536, 2, 64, 8),       # 78 tiles in the forward, 12 in the backward
-    (6656, 1024, 1400, 3, 128, 8),      # backward with a split last wave and ragged token rows
-    (1024, 1024, 1536, 4, 128, 16),     # two rank tiles: falls back to the gradient kernels
+    (6656, 1024, 1400, 3, 128, 8),      # backward with a split last wave (producers half a tile ahead only: falls back), ragged rows
+    (1024, 1024, 1400, 3, 128, 8),      # producers with ragged token rows
+    (1024, 1024, 1536, 4, 128, 16),     # two rank tiles: three row blocks per producer CTA
+    (1024, 1024, 4096, 4, 128, 16),     # ... which 32 tiles leave too few idle pairs for: falls back to the gradient kernels
+    (2048, 1024, 2000, 8, 128, 24),     # three rank tiles: falls back
     (512, 768, 64, 4, 128, 8),          # single-CTA tensor-core kernel: falls back
     (512, 768, 9, 8, 128, 8),           # few-token kernels: falls back
     (96, 40, 300, 4, 32, 8),            # CUDA-core kernel: falls back
@@ -86,3 +89,29 @@ def test_config2_shape_db_and_step_outputs():
     assert rel_err(to_f64(out["db"]["dB"]), ref["dB"]) <= REL_TOL
     assert rel_err(to_f64(out["db"]["dA"]), ref["dA"]) <= REL_TOL
     assert torch.equal(out["plain"]["dX"].view(torch.int16), out["db"]["dX"].view(torch.int16))
+
+
+@pytest.mark.parametrize("r", [8, 16])
+def test_producer_route_is_the_one_that_runs(r):
+    """With the whole workspace the producer clusters form dB; with a workspace one byte short of the optional area for
+    their parts the same call hands dB to the gradient kernels.  Both are right, and they group the sum over tokens
+    differently, so their bits differ: equal bits would mean the producer route never ran."""
+    layer = qi.random_codes_layer(K=1024, N=1024, bits=4, group_size=128, r=r, alpha=2.0 * r, M=1536, seed=90 + r)
+    gl = GpuLayer(layer)
+    ref = orc.layer_reference(layer)
+    M, dev = gl.M, gl.X.device
+    Y = torch.empty((M, gl.N), dtype=torch.bfloat16, device=dev)
+    H = torch.empty((M, gl.r), dtype=torch.float32, device=dev)
+    ql.qlora_fwd(gl.desc, M, gl.X, gl.Q, gl.scales, gl.zeros, gl.A, gl.B, Y, H, gl.ws)
+    need = ql.qlora_workspace_bytes(gl.desc, M)
+    got = {}
+    for name, nbytes in (("producers", need), ("gradient kernels", need - 1)):
+        dX = torch.empty((M, gl.K), dtype=torch.bfloat16, device=dev)
+        G = torch.empty((M, gl.r), dtype=torch.float32, device=dev)
+        dB = torch.empty((gl.N, gl.r), dtype=torch.float32, device=dev)
+        ql.qlora_bwd_input_db(gl.desc, M, gl.dY, gl.Q, gl.scales, gl.zeros, gl.A, gl.B, H, dX, G, dB, 0, gl.ws, workspace_bytes=nbytes)
+        torch.cuda.synchronize()
+        assert rel_err(to_f64(dB), ref["dB"]) <= REL_TOL, name
+        got[name] = dB
+    assert ql.qlora_device_status() == 0
+    assert not torch.equal(got["producers"], got["gradient kernels"])
