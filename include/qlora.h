@@ -42,7 +42,7 @@
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = the legacy default stream) of
  *     the current device.  No call synchronises the device; outputs are valid in stream order.
  *   - Calls given the same workspace must be ordered one after the other (same stream, or events): they share
- *     its contents, which include two counters through which CTAs of one launch signal each other (set to zero in
+ *     its contents, which include a few counters through which CTAs of one launch signal each other (set to zero in
  *     stream order ahead of the launch, so the workspace needs no initialisation).  Calls with different workspaces may
  *     overlap freely.
  *   - Return value: QLORA_OK or a negative QLORA_ERR_* code.  Arguments are validated before anything is

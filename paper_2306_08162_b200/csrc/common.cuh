@@ -29,7 +29,7 @@ __device__ __forceinline__ __nv_bfloat16 dequant_one(uint32_t q, __half scale, _
 // it may be scheduled while its predecessor in the stream is still running, does its own set-up (barriers, tensor memory,
 // descriptor fetches), and then blocks in pdl_wait() until the predecessor has completed and its writes are visible.
 // Nothing may read or write global memory before pdl_wait().  pdl_launch_dependents() at the top lets the successor be
-// scheduled as soon as every CTA of this grid has started.  This hides the launch latency between the six kernels of a step.
+// scheduled as soon as every CTA of this grid has started.  This hides the launch latency between the kernels of a step.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
