@@ -254,18 +254,26 @@ lora_grad_partial_kernel(int M, int r, int rows_per_slice, GradSide side0, GradS
         for (int c = 0; c < 4; ++c) acc[rt][c][0] = acc[rt][c][1] = acc[rt][c][2] = acc[rt][c][3] = 0.f;
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
     const int m_stop = min(M, m_begin + rows_per_slice);
-    for (int mm = m_begin; mm < m_stop; mm += 16 * LG_UNROLL) {
-        uint4 x0[LG_UNROLL], x1[LG_UNROLL];
+    // two register sets: the loads of the next round of 16-row steps are in flight while this round is transposed and multiplied
+    uint4 n0[LG_UNROLL], n1[LG_UNROLL];
+    auto load_round = [&](int mm) {
 #pragma unroll
         for (int u = 0; u < LG_UNROLL; ++u) {
             const int ma = mm + 16 * u + g, mb = ma + 8;
-            x0[u] = (live && ma < m_stop) ? *reinterpret_cast<const uint4*>(src + (size_t)ma * C) : zero4;
-            x1[u] = (live && mb < m_stop) ? *reinterpret_cast<const uint4*>(src + (size_t)mb * C) : zero4;
+            n0[u] = (live && ma < m_stop) ? *reinterpret_cast<const uint4*>(src + (size_t)ma * C) : zero4;
+            n1[u] = (live && mb < m_stop) ? *reinterpret_cast<const uint4*>(src + (size_t)mb * C) : zero4;
             if (sd.mask != nullptr) {
-                if (live && ma < m_stop) x0[u] = mask_eight(x0[u], __ldg(reinterpret_cast<const uint2*>(sd.mask + (size_t)ma * C + c0)));
-                if (live && mb < m_stop) x1[u] = mask_eight(x1[u], __ldg(reinterpret_cast<const uint2*>(sd.mask + (size_t)mb * C + c0)));
+                if (live && ma < m_stop) n0[u] = mask_eight(n0[u], __ldg(reinterpret_cast<const uint2*>(sd.mask + (size_t)ma * C + c0)));
+                if (live && mb < m_stop) n1[u] = mask_eight(n1[u], __ldg(reinterpret_cast<const uint2*>(sd.mask + (size_t)mb * C + c0)));
             }
         }
+    };
+    load_round(m_begin);
+    for (int mm = m_begin; mm < m_stop; mm += 16 * LG_UNROLL) {
+        uint4 x0[LG_UNROLL], x1[LG_UNROLL];
+#pragma unroll
+        for (int u = 0; u < LG_UNROLL; ++u) { x0[u] = n0[u]; x1[u] = n1[u]; }
+        if (mm + 16 * LG_UNROLL < m_stop) load_round(mm + 16 * LG_UNROLL);
 #pragma unroll
         for (int u = 0; u < LG_UNROLL; ++u) {
             const int ml = mm + 16 * u - m_begin;              // warp-uniform
