@@ -249,7 +249,15 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                 const size_t e_lo = (size_t)p.T * blockIdx.x / n_ctas * p.r / 4, e_hi = (size_t)p.T * (blockIdx.x + 1) / n_ctas * p.r / 4;
                 for (size_t e4 = e_lo + threadIdx.x; e4 < e_hi; e4 += blockDim.x) {
                     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int src = 0; src < n_src; ++src) {
+                    int src = 0;
+                    for (; src + 4 <= n_src; src += 4) {       // four parts in flight, added in CTA order
+                        float4 x[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) x[i] = __ldcg(reinterpret_cast<const float4*>(p.db_part + (size_t)(src + i) * part_elems) + e4);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) { v.x += x[i].x; v.y += x[i].y; v.z += x[i].z; v.w += x[i].w; }
+                    }
+                    for (; src < n_src; ++src) {
                         const float4 x = __ldcg(reinterpret_cast<const float4*>(p.db_part + (size_t)src * part_elems) + e4);
                         v.x += x.x; v.y += x.y; v.z += x.z; v.w += x.w;
                     }
