@@ -63,7 +63,7 @@ def weight_bytes(w):
 
 # DRAM traffic (read + write) per launch of the dominant kernel of the default workload, from one ncu capture of that
 # kernel (dram__bytes_read.sum + dram__bytes_write.sum).  Set back to None whenever that kernel changes.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = (26.13e6, 26.56e6)   # forward, backward-input (with dB)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = (26.03e6, 26.09e6)   # forward, backward-input (with dB)
 
 
 def layer_flops(M, K, N, r):
@@ -475,12 +475,14 @@ def run_ours(args):
             s_ms, s_reps, s_region, s_clocks = gt.region(1000.0, local)
             sustained = dict(ms_per_step=s_ms / args.steps, replays=s_reps, timed_region_ms=s_region, clocks=s_clocks)
         del gt
-        call_ms = []
-        for call in (lambda L: ql.qlora_fwd(d, M, L["X"], L["Q"], L["scales"], L["zeros"], L["A"], L["B"], L["Y"], L["H"], ws),
-                     bwd_input_call, bwd_lora_call):
-            gtc = GraphTimer(steps_body(call), barrier)
-            call_ms.append(gtc.region(20.0)[0] / args.steps)
-            del gtc
+        # per-call split: one graph per kind of call, their regions taken in rotation (three rounds, median) so that no call
+        # is always the one timed on the warmest GPU
+        timers = [GraphTimer(steps_body(call), barrier)
+                  for call in (lambda L: ql.qlora_fwd(d, M, L["X"], L["Q"], L["scales"], L["zeros"], L["A"], L["B"], L["Y"], L["H"], ws),
+                               bwd_input_call, bwd_lora_call)]
+        rounds = [[gtc.region(10.0)[0] / args.steps for gtc in timers] for _ in range(3)]
+        call_ms = [float(np.median([rd[i] for rd in rounds])) for i in range(3)]
+        del timers
     else:
         replays, region_ms = 1, total_ms
 
