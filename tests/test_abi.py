@@ -147,3 +147,26 @@ def test_host_state_is_per_device_and_nothing_is_keyed_by_caller_pointers():
     assert "size_t done[kMaxDevices]" in ds and "int cached[kMaxDevices]" in ds and "cudaGetDevice" in ds
     assert "max_clusters_dev[kMaxDevices]" in text["umma_kernel.cu"]
     assert "DeviceFacts facts[ST_MAX_DEVICES]" in text["stream_kernel.cu"]
+
+
+def test_which_way_db_goes_is_a_host_side_plan(ql):
+    """qlora_bwd_input_db_on_producers launches nothing: it replays the backward call's plan (tiles against SM pairs,
+    idle pairs against row blocks).  Without a GPU the library plans for 148 SMs, so the LLaMA-7B answers are fixed."""
+    yes = [(4096, 4096, 8, 2048), (4096, 4096, 8, 8192), (4096, 4096, 8, 4096), (1024, 1024, 16, 1536)]
+    no = [(4096, 4096, 8, 128),        # single-CTA tensor-core kernel: no producer pairs
+          (4096, 4096, 8, 16),         # few-token kernels
+          (4096, 4096, 24, 2048),      # three rank tiles
+          (4096, 11008, 16, 2048),     # 64 tiles leave ten idle pairs: too few for 128 row blocks at three per CTA
+          (11008, 4096, 16, 2048)]     # split last wave: the producers are only half a tile ahead
+    for K, N, r, M in yes:
+        assert ql.qlora_bwd_input_db_on_producers(ql.desc(2, 64, K, N, r, 16.0), M) is True, (K, N, r, M)
+    for K, N, r, M in no:
+        assert ql.qlora_bwd_input_db_on_producers(ql.desc(2, 64, K, N, r, 16.0), M) is False, (K, N, r, M)
+    # the optional workspace areas exist exactly where they can be used
+    d = ql.desc(4, 128, 4096, 4096, 8, 16.0)
+    assert ql.qlora_workspace_bytes(d, 2048) >= 2 * 10 * 4096 * 8 * 4 + 11 * 8192 * 8 * 4      # the parts of dB of 20 producer CTAs + gradient partial sums
+    assert ql.qlora_workspace_bytes(d, 128) < 2**20                                            # nothing optional with few tokens
+    gate = ql.desc(2, 64, 4096, 11008, 16, 32.0)
+    assert ql.qlora_workspace_bytes(gate, 2048) >= 24 * 512 * 1024      # 24 split tiles of the forward
+    with pytest.raises(ql.QloraError):
+        ql.qlora_bwd_input_db_on_producers(ql.desc(5, 64, 4096, 4096, 8, 16.0), 2048)
