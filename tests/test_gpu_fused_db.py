@@ -115,3 +115,47 @@ def test_producer_route_is_the_one_that_runs(r):
         got[name] = dB
     assert ql.qlora_device_status() == 0
     assert not torch.equal(got["producers"], got["gradient kernels"])
+
+
+@pytest.mark.parametrize("K,N,M,bits,g,r", [(1024, 1024, 1536, 4, 128, 8),      # dB on the producers
+                                            (1024, 6656, 1536, 4, 128, 8),      # ... with a split last wave in the forward
+                                            (6656, 1024, 1536, 2, 64, 16)])     # split last wave in the backward, dB by the gradient kernels
+def test_replayed_graph_gives_the_eager_bits(K, N, M, bits, g, r):
+    """A whole step (forward, backward with dB, gradient call for dA) captured in a CUDA graph and replayed three times:
+    the counters in the workspace are zeroed by a captured launch, so every replay must reproduce the eager results bit
+    for bit, split tiles and producer clusters included."""
+    layer = qi.random_codes_layer(K=K, N=N, bits=bits, group_size=g, r=r, alpha=2.0 * r, M=M, seed=K + N + r)
+    gl = GpuLayer(layer)
+    dev = gl.X.device
+
+    def buffers():
+        return dict(Y=torch.empty((M, N), dtype=torch.bfloat16, device=dev), H=torch.empty((M, r), dtype=torch.float32, device=dev),
+                    dX=torch.empty((M, K), dtype=torch.bfloat16, device=dev), G=torch.empty((M, r), dtype=torch.float32, device=dev),
+                    dA=torch.empty((r, K), dtype=torch.float32, device=dev), dB=torch.empty((N, r), dtype=torch.float32, device=dev))
+
+    def step(b):
+        ql.qlora_fwd(gl.desc, M, gl.X, gl.Q, gl.scales, gl.zeros, gl.A, gl.B, b["Y"], b["H"], gl.ws)
+        ql.qlora_bwd_input_db(gl.desc, M, gl.dY, gl.Q, gl.scales, gl.zeros, gl.A, gl.B, b["H"], b["dX"], b["G"], b["dB"], 0, gl.ws)
+        ql.qlora_bwd_lora(gl.desc, M, gl.X, None, gl.A, gl.B, None, b["G"], b["dA"], None, 0, gl.ws)
+
+    eager = buffers()
+    step(eager)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    captured = buffers()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            step(captured)
+    for _ in range(3):
+        for t in captured.values():
+            t.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        for key in eager:
+            a, b = eager[key], captured[key]
+            assert torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a, b.view(torch.int16) if b.dtype == torch.bfloat16 else b), key
+    assert ql.qlora_device_status() == 0
+    ref = orc.layer_reference(layer, rows=[0, 1, M - 1])
+    assert rel_err(to_f64(captured["dB"]), ref["dB"]) <= REL_TOL and rel_err(to_f64(captured["dA"]), ref["dA"]) <= REL_TOL
