@@ -45,6 +45,11 @@
  *     its contents, which include a few counters through which CTAs of one launch signal each other (set to zero in
  *     stream order ahead of the launch, so the workspace needs no initialisation).  Calls with different workspaces may
  *     overlap freely.
+ *     (With many tokens a launch coordinates its CTAs through those counters: tiles wait for the CTAs that form H / G,
+ *     the finishing half of a split tile for the giving half.  These waits point to CTAs dispatched earlier, so a launch
+ *     never waits for itself; where the forming CTAs also own tiles -- more tiles than SM pairs -- two such launches
+ *     running at the same time on different streams can still hold each other's SMs.  Every wait is bounded: after
+ *     250 ms the call gives up and qlora_device_status reports QLORA_ERR_TIMEOUT.)
  *   - Return value: QLORA_OK or a negative QLORA_ERR_* code.  Arguments are validated before anything is
  *     launched; on error nothing has been enqueued.  Nothing is printed, nothing throws.
  *   - Same inputs give bitwise the same outputs on every run (fixed-order reductions, no floating-point atomics).
@@ -111,7 +116,7 @@ int qlora_bwd_input(const qlora_desc* desc, int M, const void* dY, const int32_t
  * same dY that flows back through the frozen weight), so that dY is read once for both.  H: fp32 [M, r], the forward's
  * H_out (required when r > 0); dB: fp32 [N, r]; accumulate as in qlora_bwd_lora.  With many tokens and r <= 16 the SMs
  * that stream dY to form G inside the backward kernel form dB on the same pass (each leaves a part in the workspace,
- * they add the parts in a fixed order before they go on); for other shapes dB comes from the gradient kernels after
+ * the CTAs that own tiles add the parts in a fixed order while their main loops run); for other shapes dB comes from the gradient kernels after
  * the backward kernel.  Either way dB is complete when the call's work is, and the same inputs give the same bits on a
  * given device; the two routes group the sum over tokens differently, so their bits differ from each other (and from
  * qlora_bwd_lora's) in the last places.  Follow it with qlora_bwd_lora(..., dB = NULL) for dA. */

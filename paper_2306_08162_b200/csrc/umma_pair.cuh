@@ -26,11 +26,11 @@
 
 //
 // When the tiles make more than one wave and at most half a wave is left over (172 tiles on 74 pairs: 24), each left-over
-// tile is worked on by two pairs, one half of the contraction steps each, as the last thing both do.  Their epilogues
-// then trade halves of the fp32 result through the caller's workspace -- each writes the eight 32-column chunks it does
-// not finish, both count themselves in at the tile's counter and wait for the other (bounded), each adds the peer's
-// part to the chunks it keeps -- so the third wave costs about two thirds of a tile instead of a whole one.  Nothing can
-// wait in a circle: the split item is every worker's last, and all workers are resident (one CTA per SM).
+// tile is worked on by two pairs, one half of the contraction steps each, as the last thing both do.  The pair with the
+// lower block indices then gives its half of the fp32 result away through the caller's workspace and is done; the other
+// waits for it (bounded), adds the two halves and stores the tile -- so the third wave costs about three quarters of a tile
+// instead of a whole one.  Every wait in this kernel points from higher block indices to lower ones (tiles wait for producer
+// clusters, the finishing half of a split tile for the giving half), i.e. to CTAs that were dispatched earlier.
 
 constexpr int kPairTok = 128;                          // token rows per CTA per accumulator
 constexpr int kPairW = 128;                            // weight rows per CTA (256 per pair tile)
@@ -144,7 +144,10 @@ __device__ __forceinline__ PairItem pair_item(const PairParams& p, int w, int W,
     if (it < full) { r.tile = w + it * W; r.s0 = 0; r.s1 = p.steps; r.part = 0; r.nparts = 1; }
     else {
         r.tile = p.n_full + w / p.nsplit; r.part = w % p.nsplit; r.nparts = p.nsplit;
-        r.s0 = p.steps * r.part / p.nsplit; r.s1 = p.steps * (r.part + 1) / p.nsplit;
+        // (the giving half, part 0, takes 29 of 64 steps: it has its result to write out before the other half, which waits
+        // for it, can begin to add)
+        const int cut = p.steps * 29 / 64;
+        r.s0 = r.part == 0 ? 0 : cut; r.s1 = r.part == 0 ? cut : p.steps;
     }
     return r;
 }
@@ -217,7 +220,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         // ------------------------------------------------------------------ producer cluster: LoRA down-projection first
         // (this CTA's row blocks: blockIdx.x, blockIdx.x + 2 n_prod, ...; the ring takes the operand area, below the barriers)
         pdl_wait();
-        bool db_here = false;
+        bool db_here = false;                // (the parts are added up by the tile CTAs, see the epilogue)
         if constexpr (TRANSPOSED) {
             if (p.with_db) {       // the same pass over dY also gives this CTA's part of dB
                 db_here = true;
@@ -233,41 +236,6 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         __threadfence();       // every thread's rows of P (and of its part of dB) are visible device-wide before the CTA is counted
         __syncthreads();
         if (threadIdx.x == 0) atomicAdd(&p.sync[0], 1u);
-        if (db_here) {
-            // The producers meet at a counter of their own (all of them are resident: they are the first clusters of a grid of
-            // at most one CTA per SM), then producer CTA i adds the parts, in CTA order, for its share of the columns.
-            const unsigned n_ctas = 2u * (unsigned)p.n_prod;
-            if (threadIdx.x == 0) {
-                atomicAdd(&p.sync[kSyncWords - 1], 1u);
-                wait_counter(&p.sync[kSyncWords - 1], n_ctas, abort_flag);
-            }
-            __syncthreads();
-            if (!*abort_flag) {
-                const int n_blocks = (p.M + 15) >> 4;
-                const int n_src = (int)n_ctas < n_blocks ? (int)n_ctas : n_blocks;      // CTAs beyond the row blocks wrote nothing
-                const size_t part_elems = (size_t)p.T * p.r;
-                const size_t e_lo = (size_t)p.T * blockIdx.x / n_ctas * p.r / 4, e_hi = (size_t)p.T * (blockIdx.x + 1) / n_ctas * p.r / 4;
-                for (size_t e4 = e_lo + threadIdx.x; e4 < e_hi; e4 += blockDim.x) {
-                    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                    int src = 0;
-                    for (; src + 4 <= n_src; src += 4) {       // four parts in flight, added in CTA order
-                        float4 x[4];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) x[i] = __ldcg(reinterpret_cast<const float4*>(p.db_part + (size_t)(src + i) * part_elems) + e4);
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) { v.x += x[i].x; v.y += x[i].y; v.z += x[i].z; v.w += x[i].w; }
-                    }
-                    for (; src < n_src; ++src) {
-                        const float4 x = __ldcg(reinterpret_cast<const float4*>(p.db_part + (size_t)src * part_elems) + e4);
-                        v.x += x.x; v.y += x.y; v.z += x.z; v.w += x.w;
-                    }
-                    v.x *= p.s; v.y *= p.s; v.z *= p.s; v.w *= p.s;
-                    float4* dst = reinterpret_cast<float4*>(p.db_out) + e4;
-                    if (p.db_accumulate) { const float4 o = *dst; v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w; }
-                    *dst = v;
-                }
-            }
-        }
         fence_proxy_async();   // the shared memory just used goes to the TMA / tensor-core side for this cluster's tiles, if any
         __syncthreads();
     }
@@ -396,6 +364,39 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                 }
                 asm volatile("bar.sync 2, %0;" ::"r"(kEpiWarps * 32) : "memory");
                 if (*abort_flag) break;
+                if constexpr (TRANSPOSED) {
+                    if (p.with_db) {
+                        // dB: every producer CTA has left its part of s dY^T H in the workspace.  The CTAs that have a tile share
+                        // the columns; each adds the parts in producer order for its share, scales and writes dB -- here, while
+                        // its main loop still runs and these warps would only wait for it.  (A wait of producers for one
+                        // another would point from low block indices to high ones; this one points the safe way.)
+                        const int n_cons = 2 * (p.n_tiles < tile_stride ? p.n_tiles : tile_stride);
+                        const int me = 2 * first_tile + (int)cta;
+                        const int n_blocks = (p.M + 15) >> 4, n_ctas = 2 * p.n_prod;
+                        const int n_src = n_ctas < n_blocks ? n_ctas : n_blocks;            // producer CTAs beyond the row blocks wrote nothing
+                        const size_t part_elems = (size_t)p.T * p.r, total4 = part_elems / 4;
+                        const size_t e_lo = total4 * me / n_cons, e_hi = total4 * (me + 1) / n_cons;
+                        for (size_t e4 = e_lo + et; e4 < e_hi; e4 += kEpiWarps * 32) {
+                            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                            int src = 0;
+                            for (; src + 4 <= n_src; src += 4) {       // four parts in flight, added in producer order
+                                float4 x[4];
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) x[i] = __ldcg(reinterpret_cast<const float4*>(p.db_part + (size_t)(src + i) * part_elems) + e4);
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) { v.x += x[i].x; v.y += x[i].y; v.z += x[i].z; v.w += x[i].w; }
+                            }
+                            for (; src < n_src; ++src) {
+                                const float4 x = __ldcg(reinterpret_cast<const float4*>(p.db_part + (size_t)src * part_elems) + e4);
+                                v.x += x.x; v.y += x.y; v.z += x.z; v.w += x.w;
+                            }
+                            v.x *= p.s; v.y *= p.s; v.z *= p.s; v.w *= p.s;
+                            float4* dst = reinterpret_cast<float4*>(p.db_out) + e4;
+                            if (p.db_accumulate) { const float4 o = *dst; v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w; }
+                            *dst = v;
+                        }
+                    }
+                }
             }
             if (p.r > 0 && item.part == 0) {
                 // (the previous tile's LoRA MMA has completed: its accumulator-full barrier was observed below)
@@ -476,48 +477,45 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                 }
             };
             if (item.nparts > 1) {
-                // A split tile: this pair holds the sum over its half of the contraction.  The two pairs exchange halves of
-                // the tile through the workspace: each gives away the eight 32-column chunks it does not finish (fp32,
-                // laid out so that a warp's stores and the peer's loads are contiguous), counts itself in at the tile's
-                // counter, waits for all four CTAs, then adds the peer's part to the chunks it keeps and stores them.
-                // (a + b is the same in either order, so both halves of the tile see one summation order.)
+                // A split tile: this pair holds the sum over its half of the contraction.  The pair with the lower block indices
+                // (part 0, whose sum also carries the LoRA update) gives its whole half away -- fp32 through the workspace, laid out
+                // so that a warp's stores and the reader's loads are contiguous -- counts its two CTAs in at the tile's counter
+                // and is done; the other pair waits for that count (bounded), adds the peer's part to its own chunk by chunk, and
+                // stores the tile.  The wait points from high block indices to low ones only: the pair waited for was dispatched
+                // first and waits for nobody, whatever else shares the GPU.  (a + b is the same in either order.)
                 const int slot = tile - p.n_full;
-                float4* mine = p.split_buf + (size_t)((slot * 2 + item.part) * 2 + (int)cta) * (8 * 8 * 128);
-                const float4* peer = p.split_buf + (size_t)((slot * 2 + (1 - item.part)) * 2 + (int)cta) * (8 * 8 * 128);
+                float4* buf = p.split_buf + (size_t)(slot * 2 + (int)cta) * (16 * 8 * 128);     // [chunk][j4][thread]
                 auto chunk_addr = [&](int idx) { return taddr + (uint32_t)((idx >> 3) * kAccStride + (idx & 7) * 32); };
-                auto give = [&](const uint32_t (&v)[32], int k) {
+                if (item.part == 0) {
+                    auto give = [&](const uint32_t (&v)[32], int idx) {
 #pragma unroll
-                    for (int j4 = 0; j4 < 8; ++j4)
-                        mine[(k * 8 + j4) * 128 + et] = make_float4(__uint_as_float(v[4 * j4]), __uint_as_float(v[4 * j4 + 1]),
-                                                                    __uint_as_float(v[4 * j4 + 2]), __uint_as_float(v[4 * j4 + 3]));
-                };
-                {   // the chunks given away: the tensor-memory load of the next one is in flight while this one is stored
-                    uint32_t va[32], vb[32];
-                    tc_ld32(chunk_addr(1 - item.part), va);
+                        for (int j4 = 0; j4 < 8; ++j4)
+                            buf[(idx * 8 + j4) * 128 + et] = make_float4(__uint_as_float(v[4 * j4]), __uint_as_float(v[4 * j4 + 1]),
+                                                                         __uint_as_float(v[4 * j4 + 2]), __uint_as_float(v[4 * j4 + 3]));
+                    };
+                    uint32_t va[32], vb[32];                 // the tensor-memory load of the next chunk is in flight while this one is stored
+                    tc_ld32(chunk_addr(0), va);
 #pragma unroll 1
-                    for (int k = 0; k < 8; k += 2) {
+                    for (int idx = 0; idx < 16; idx += 2) {
                         tc_wait_ld();
-                        tc_ld32(chunk_addr(2 * (k + 1) + (1 - item.part)), vb);
-                        give(va, k);
+                        tc_ld32(chunk_addr(idx + 1), vb);
+                        give(va, idx);
                         tc_wait_ld();
-                        if (k + 2 < 8) tc_ld32(chunk_addr(2 * (k + 2) + (1 - item.part)), va);
-                        give(vb, k + 1);
+                        if (idx + 2 < 16) tc_ld32(chunk_addr(idx + 2), va);
+                        give(vb, idx + 1);
                     }
-                }
-                __threadfence();
-                asm volatile("bar.sync 2, %0;" ::"r"(kEpiWarps * 32) : "memory");
-                if (et == 0) {
-                    atomicAdd(&p.sync[2 + slot], 1u);
-                    wait_counter(&p.sync[2 + slot], 4u, abort_flag);
-                }
-                asm volatile("bar.sync 2, %0;" ::"r"(kEpiWarps * 32) : "memory");
-                if (*abort_flag) break;
-                {   // the chunks kept: the peer's part of the next one is requested before this one is added and stored
+                    __threadfence();
+                    asm volatile("bar.sync 2, %0;" ::"r"(kEpiWarps * 32) : "memory");
+                    if (et == 0) atomicAdd(&p.sync[2 + slot], 1u);
+                } else {
+                    if (et == 0) wait_counter(&p.sync[2 + slot], 2u, abort_flag);
+                    asm volatile("bar.sync 2, %0;" ::"r"(kEpiWarps * 32) : "memory");
+                    if (*abort_flag) break;
                     uint32_t va[32];
-                    float4 pa[8], pb[8];
-                    auto take = [&](float4 (&pv)[8], int k) {
+                    float4 pa[8], pb[8];                     // the peer's part of the next chunk is requested before this one is added and stored
+                    auto take = [&](float4 (&pv)[8], int idx) {
 #pragma unroll
-                        for (int j4 = 0; j4 < 8; ++j4) pv[j4] = __ldcg(peer + (k * 8 + j4) * 128 + et);
+                        for (int j4 = 0; j4 < 8; ++j4) pv[j4] = __ldcg(buf + (idx * 8 + j4) * 128 + et);
                     };
                     auto add = [&](uint32_t (&v)[32], const float4 (&pv)[8]) {
 #pragma unroll
@@ -530,17 +528,17 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                     };
                     take(pa, 0);
 #pragma unroll 1
-                    for (int k = 0; k < 8; k += 2) {
-                        tc_ld32(chunk_addr(2 * k + item.part), va);
-                        take(pb, k + 1);
+                    for (int idx = 0; idx < 16; idx += 2) {
+                        tc_ld32(chunk_addr(idx), va);
+                        take(pb, idx + 1);
                         tc_wait_ld();
                         add(va, pa);
-                        store_chunk(va, 2 * k + item.part);
-                        tc_ld32(chunk_addr(2 * (k + 1) + item.part), va);
-                        if (k + 2 < 8) take(pa, k + 2);
+                        store_chunk(va, idx);
+                        tc_ld32(chunk_addr(idx + 1), va);
+                        if (idx + 2 < 16) take(pa, idx + 2);
                         tc_wait_ld();
                         add(va, pb);
-                        store_chunk(va, 2 * (k + 1) + item.part);
+                        store_chunk(va, idx + 1);
                     }
                 }
             } else {
