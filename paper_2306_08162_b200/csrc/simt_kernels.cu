@@ -170,7 +170,7 @@ struct GradPlan { int slices, rows_per_slice; };
 
 static GradPlan lora_grad_plan(int M, int K, int N) {
     const int col_blocks = (K + LG_COLS - 1) / LG_COLS + (N + LG_COLS - 1) / LG_COLS;
-    int slices = (3 * 148 + col_blocks - 1) / col_blocks;        // aim for ~3 blocks per SM
+    int slices = (2 * 148) / col_blocks;                         // two blocks fit an SM (registers): aim for one wave of a 148-SM part
     if (slices > LG_MAX_SLICES) slices = LG_MAX_SLICES;
     if (slices < 1) slices = 1;
     int rows = (M + slices - 1) / slices;
