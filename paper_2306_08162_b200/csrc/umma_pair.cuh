@@ -144,9 +144,9 @@ __device__ __forceinline__ PairItem pair_item(const PairParams& p, int w, int W,
     if (it < full) { r.tile = w + it * W; r.s0 = 0; r.s1 = p.steps; r.part = 0; r.nparts = 1; }
     else {
         r.tile = p.n_full + w / p.nsplit; r.part = w % p.nsplit; r.nparts = p.nsplit;
-        // (the giving half, part 0, takes 29 of 64 steps: it has its result to write out before the other half, which waits
-        // for it, can begin to add)
-        const int cut = p.steps * 29 / 64;
+        // (the giving half, part 0, takes 27 of 64 steps: it has its result to write out before the other half, which waits
+        // for it, can begin to add; 25 .. 33 were timed, 27 is the shallow minimum)
+        const int cut = p.steps * 27 / 64;
         r.s0 = r.part == 0 ? 0 : cut; r.s1 = r.part == 0 ? cut : p.steps;
     }
     return r;
