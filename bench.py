@@ -63,7 +63,7 @@ def weight_bytes(w):
 
 # DRAM traffic (read + write) per launch of the dominant kernel of the default workload, from one ncu capture of that
 # kernel (dram__bytes_read.sum + dram__bytes_write.sum).  Set back to None whenever that kernel changes.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = (26.03e6, 26.06e6)   # forward, backward-input (with dB)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = (26.08e6, 26.17e6)   # forward, backward-input (with dB)
 
 
 def layer_flops(M, K, N, r):
