@@ -78,7 +78,6 @@ size_t required_workspace_bytes(const qlora_desc& d, int M);
 // cluster.  Ldown / Lup: the adapter applied first / second (forward A, B; backward B, A).  P = H or G, fp32 [M, r]: read
 // when p_is_input, otherwise computed inside the kernel (ranks up to 16) and written out.
 bool stream_supported(const qlora_desc& d, int M, bool transposed);
-int launch_weight_prefetch(const qlora_desc& d, const int32_t* Q, const void* scales, const void* zeros, cudaStream_t st);
 int launch_stream_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
                        const void* zeros, const void* Ldown, const void* Lup, float* P, bool p_is_input, void* Out,
                        cudaStream_t st);

@@ -899,35 +899,6 @@ __global__ void __launch_bounds__(512, 1) stream_bwd_kernel(const StreamParams p
     st_finish<true, TOKS>(p, recv_part, recv_h, hfull, lup, tile_c, rank);
 }
 
-// ------------------------------------------------------------------------------------------------------------
-// Weight prefetch.  A streaming kernel owns its SM (sixteen warps, most of the registers and shared memory), so the CTAs
-// of the next call cannot move in beside it and start their copies early.  This small kernel goes in front of every
-// streaming kernel instead: its CTAs need almost nothing, so they run while the preceding call is still computing
-// (programmatic dependent launch), ask the call's packed words, scales and zeros into L2 with bulk prefetches, and then
-// wait for the preceding grid -- the streaming kernel behind it waits for THIS grid, hence for everything before it.
-// Only the frozen tensors are touched.
-// ------------------------------------------------------------------------------------------------------------
-constexpr int ST_PF_CHUNK = 8192;   // bytes per bulk prefetch
-
-__device__ __forceinline__ void st_bulk_prefetch(const char* base, size_t bytes, size_t first, size_t stride) {
-    for (size_t off = first * ST_PF_CHUNK; off < bytes; off += stride * ST_PF_CHUNK) {
-        const size_t left = bytes - off;
-        const uint32_t n = (uint32_t)(left < ST_PF_CHUNK ? left : ST_PF_CHUNK) & ~15u;
-        if (n) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + off), "r"(n) : "memory");
-    }
-}
-
-__global__ void __launch_bounds__(128) stream_prefetch_kernel(const char* Q, size_t q_bytes, const char* scales, const char* zeros, size_t sz_bytes) {
-    pdl_launch_dependents();
-    const size_t me = (size_t)blockIdx.x * blockDim.x + threadIdx.x, all = (size_t)gridDim.x * blockDim.x;
-    st_bulk_prefetch(Q, q_bytes, me, all);
-    st_bulk_prefetch(scales, sz_bytes, me, all);
-    st_bulk_prefetch(zeros, sz_bytes, me, all);
-    pdl_wait();
-}
-
-// Raising a kernel's dynamic shared-memory limit is a per-function AND per-device setting: `done` belongs to one kernel
-// instantiation and holds, per device ordinal, the limit already set there.
 template <typename Kern>
 bool st_configure(Kern kern, size_t smem_bytes, size_t (&done)[ST_MAX_DEVICES], std::mutex& mu) {
     int dev = 0;
@@ -1024,15 +995,6 @@ bool stream_supported(const qlora_desc& d, int M, bool transposed) {
     return d.group_size % fwd_kb(d.bits) == 0;
 }
 
-// The frozen tensors of a layer asked into L2 by a handful of small CTAs that run under the preceding kernel of the stream
-// (see stream_prefetch_kernel); the kernel launched behind it is ordered after everything before it.
-int launch_weight_prefetch(const qlora_desc& d, const int32_t* Q, const void* scales, const void* zeros, cudaStream_t st) {
-    const size_t q_bytes = (size_t)d.K * d.bits / 8 * d.N, sz_bytes = (size_t)(d.K / d.group_size) * d.N * 2;
-    const unsigned blocks = (unsigned)((q_bytes / ST_PF_CHUNK + 127) / 128 + 1);
-    return launch_pdl(stream_prefetch_kernel, dim3(blocks), dim3(128), 0, st, 1, (const char*)Q, q_bytes, (const char*)scales,
-                      (const char*)zeros, sz_bytes) == cudaSuccess ? QLORA_OK : QLORA_ERR_CUDA;
-}
-
 int launch_stream_gemm(const qlora_desc& d, int M, bool transposed, const void* In, const int32_t* Q, const void* scales,
                        const void* zeros, const void* Ldown, const void* Lup, float* P, bool p_is_input, void* Out,
                        cudaStream_t st) {
@@ -1098,10 +1060,6 @@ int launch_stream_gemm(const qlora_desc& d, int M, bool transposed, const void* 
         case 8: smem = st_smem_bytes<8>(transposed, nw, toks, p.xc, p.copies, KH, ks, tile_c); break;
     }
     if (smem > 227 * 1024) return QLORA_ERR_UNSUPPORTED;
-    {   // the frozen tensors on their way into L2 while the preceding call computes
-        const int rc = launch_weight_prefetch(d, Q, scales, zeros, st);
-        if (rc != QLORA_OK) return rc;
-    }
 #define QLORA_ST(B, NT)                                                                                   \
     return transposed ? st_launch<B, NT, true>(p, nw, tiles, smem, st) : st_launch<B, NT, false>(p, nw, tiles, smem, st)
 #define QLORA_ST_BITS(NT)           \
